@@ -1,0 +1,146 @@
+"""CPU oracle for the GPTQ int4 matmul - TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes loader around ``gptq_oracle.c`` (plain C, OpenMP).  Only tests,
+the smoke check and the CPU-baseline leg of the benchmark may import this
+package; the CUDA product path never does, and this package never imports
+the CUDA package.  See the header of ``gptq_oracle.c`` for what is computed
+and which passage of the paper it follows.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gptq_oracle.c")
+_LIB = os.path.join(_HERE, "libgptq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.oracle_half_to_float.restype = ctypes.c_float
+        lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
+        lib.oracle_num_threads.restype = ctypes.c_int
+        for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
+                     "oracle_gemm_f64", "oracle_gemm_f64_at"):
+            getattr(lib, name).restype = None
+        _lib = lib
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i32(a, shape=None):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    if shape is not None:
+        assert a.shape == shape, (a.shape, shape)
+    return a
+
+
+def _f16(a, shape=None):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float16, a.dtype
+    if shape is not None:
+        assert a.shape == shape, (a.shape, shape)
+    return a
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def half_to_float(bits: int) -> float:
+    return float(_load().oracle_half_to_float(ctypes.c_uint16(bits)))
+
+
+def unpack_q(qweight: np.ndarray) -> np.ndarray:
+    """int32[K/8, N] -> uint8[K, N]."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    out = np.empty((R * 8, N), dtype=np.uint8)
+    _load().oracle_unpack_q(_p(qweight), ctypes.c_int(R * 8), ctypes.c_int(N), _p(out))
+    return out
+
+
+def unpack_z(qzeros: np.ndarray) -> np.ndarray:
+    """int32[G, N/8] -> uint8[G, N]."""
+    qzeros = _i32(qzeros)
+    G, C = qzeros.shape
+    out = np.empty((G, C * 8), dtype=np.uint8)
+    _load().oracle_unpack_z(_p(qzeros), ctypes.c_int(G), ctypes.c_int(C * 8), _p(out))
+    return out
+
+
+def dequant_f32(qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
+    """fp32[K, N] dequantised weights; ``g_idx`` None means no act-order."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales = _f16(scales, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    out = np.empty((K, N), dtype=np.float32)
+    _load().oracle_dequant_f32(_p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(K),
+                               ctypes.c_int(N), ctypes.c_int(group_size), _p(out))
+    return out
+
+
+def gemm_f64(x, qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
+    """fp64[M, N] = x[M, K] . dequant(W)[K, N], k ascending."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    x = _f16(x)
+    M = x.shape[0]
+    assert x.shape == (M, K)
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales = _f16(scales, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    out = np.empty((M, N), dtype=np.float64)
+    _load().oracle_gemm_f64(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M),
+                            ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size), _p(out))
+    return out
+
+
+def gemm_f64_at(x, qweight, qzeros, scales, g_idx, group_size: int, rows, cols) -> np.ndarray:
+    """The same sum as :func:`gemm_f64` for chosen (row, col) outputs only."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    x = _f16(x)
+    M = x.shape[0]
+    assert x.shape == (M, K)
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales = _f16(scales, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    rows = _i32(rows)
+    cols = _i32(cols)
+    assert rows.shape == cols.shape and rows.ndim == 1
+    assert rows.min(initial=0) >= 0 and rows.max(initial=0) < M
+    assert cols.min(initial=0) >= 0 and cols.max(initial=0) < N
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _load().oracle_gemm_f64_at(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M),
+                               ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size),
+                               _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
+    return out

@@ -1,0 +1,154 @@
+/*
+ * CPU oracle for the GPTQ 4-bit weight-only matmul  y[M,N] = x[M,K] . dequant(W)[K,N].
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+ * CUDA library is checked against.  It shares no code, header, table or helper
+ * with the CUDA path and must never be linked into or called from it.
+ *
+ * What it follows.  The paper (Opt4GPTQ, Section 1 and Section 4.2) accelerates
+ * the 4-bit GPTQ linear layer with fp16 activations and states (Section 4.4,
+ * last paragraph) that its kernels equal plain GPTQ up to floating-point
+ * summation order.  So the oracle is the plain definition itself:
+ *
+ *   q[k][n]  = nibble (k mod 8) of qweight[k/8][n]     (LSB first, word as uint32)
+ *   z[g][n]  = nibble (n mod 8) of qzeros[g][n/8]
+ *   g(k)     = g_idx[k] if act-order else k / group_size
+ *   w32[k][n]= float(q[k][n] - z[g(k)][n]) * float(scales[g(k)][n])   one fp32 multiply
+ *   y[m][n]  = sum_{k ascending} double(x[m][k]) * double(w32[k][n])  fp64
+ *
+ * The paper never spells the storage format out; the reading above (LSB-first
+ * nibbles, stored zero point used as is, unsigned shifts) is the one the tests
+ * pin with hand-packed words.  The fp32 product is exact (|q-z| <= 15 needs 4
+ * bits, an fp16 significand 11), so there is one right dequantised value.
+ *
+ * Parity with numbers printed in the paper: unpinned - the paper prints no value
+ * for this computation.  Each function is pinned by the mathematics instead
+ * (hand-packed words, brute force, closed forms, special cases); see tests/.
+ */
+#include <stdint.h>
+#include <stddef.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* IEEE-754 binary16 -> binary32, written from the format definition:
+ * 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+float oracle_half_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    uint32_t exp = (uint32_t)(h >> 10) & 0x1Fu;
+    uint32_t frac = (uint32_t)h & 0x3FFu;
+    uint32_t bits;
+    if (exp == 0) {
+        if (frac == 0) {
+            bits = sign << 31;                           /* signed zero */
+        } else {                                         /* subnormal: frac * 2^-24 */
+            int e = -1;
+            do { frac <<= 1; e++; } while ((frac & 0x400u) == 0);
+            frac &= 0x3FFu;
+            bits = (sign << 31) | ((uint32_t)(127 - 15 - e) << 23) | (frac << 13);
+        }
+    } else if (exp == 31) {
+        bits = (sign << 31) | 0x7F800000u | (frac << 13); /* inf / nan */
+    } else {
+        bits = (sign << 31) | ((exp + 127 - 15) << 23) | (frac << 13);
+    }
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+static inline unsigned nibble(int32_t word, int i)
+{
+    return ((uint32_t)word >> (4 * i)) & 15u;
+}
+
+/* Step 1: q[k][n] for all k < K, n < N. */
+void oracle_unpack_q(const int32_t *qweight, int K, int N, uint8_t *q_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            q_out[(size_t)k * N + n] = (uint8_t)nibble(qweight[(size_t)(k >> 3) * N + n], k & 7);
+}
+
+/* Step 2: z[g][n] for all g < G, n < N. */
+void oracle_unpack_z(const int32_t *qzeros, int G, int N, uint8_t *z_out)
+{
+    for (int g = 0; g < G; g++)
+        for (int n = 0; n < N; n++)
+            z_out[(size_t)g * N + n] = (uint8_t)nibble(qzeros[(size_t)g * (N / 8) + (n >> 3)], n & 7);
+}
+
+static inline int group_of(const int32_t *g_idx, int k, int group_size)
+{
+    return g_idx ? g_idx[k] : k / group_size;
+}
+
+static inline float dequant_one(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                                const int32_t *g_idx, int N, int group_size, int k, int n)
+{
+    int g = group_of(g_idx, k, group_size);
+    int q = (int)nibble(qweight[(size_t)(k >> 3) * N + n], k & 7);
+    int z = (int)nibble(qzeros[(size_t)g * (N / 8) + (n >> 3)], n & 7);
+    float s = oracle_half_to_float(scales[(size_t)g * N + n]);
+    return (float)(q - z) * s;
+}
+
+/* Steps 3-4: w32[k][n].  g_idx may be NULL (no act-order). */
+void oracle_dequant_f32(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                        const int32_t *g_idx, int K, int N, int group_size, float *w_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            w_out[(size_t)k * N + n] = dequant_one(qweight, qzeros, scales, g_idx, N, group_size, k, n);
+}
+
+/* Step 5: y[m][n] in fp64, k ascending. */
+void oracle_gemm_f64(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                     const uint16_t *scales, const int32_t *g_idx,
+                     int M, int N, int K, int group_size, double *y_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; n++) {
+        for (int m = 0; m < M; m++) {
+            double acc = 0.0;
+            for (int k = 0; k < K; k++) {
+                float w = dequant_one(qweight, qzeros, scales, g_idx, N, group_size, k, n);
+                acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+            }
+            y_out[(size_t)m * N + n] = acc;
+        }
+    }
+}
+
+/* Step 5 on chosen outputs only: y_out[i] = y[rows[i]][cols[i]], the same sum,
+ * for spot checks at sizes where the full product would take too long. */
+void oracle_gemm_f64_at(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                        const uint16_t *scales, const int32_t *g_idx,
+                        int M, int N, int K, int group_size,
+                        const int32_t *rows, const int32_t *cols, int count, double *y_out)
+{
+    (void)M;
+    #pragma omp parallel for schedule(static)
+    for (int i = 0; i < count; i++) {
+        int m = rows[i], n = cols[i];
+        double acc = 0.0;
+        for (int k = 0; k < K; k++) {
+            float w = dequant_one(qweight, qzeros, scales, g_idx, N, group_size, k, n);
+            acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+        }
+        y_out[i] = acc;
+    }
+}

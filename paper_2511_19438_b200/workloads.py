@@ -1,0 +1,155 @@
+"""Seeded synthetic inputs for the GPTQ int4 matmul path.
+
+This module only *draws and encodes* inputs (random nibbles, scales, zero
+points, activations, act-order permutations) and names the workload shapes.
+It holds none of the method's arithmetic: no unpacking, no dequantisation,
+no matmul.  Both the CUDA path and the CPU oracle are fed from here, so the
+two never share anything but their inputs.
+
+Storage format produced (the GPTQ checkpoint convention the path consumes):
+
+* ``qweight int32[K/8, N]`` - nibble ``i`` (bits ``4i..4i+3``, LSB first) of
+  word ``(r, n)`` is ``q[8r+i, n]`` in ``0..15``.
+* ``qzeros int32[G, N/8]``  - nibble ``j`` of word ``(g, c)`` is ``z[g, 8c+j]``.
+* ``scales fp16[G, N]``, ``G = K / group_size``.
+* ``g_idx int32[K]`` (act-order only) - row ``k`` uses scale/zero row
+  ``g_idx[k]``; here ``g_idx[k] = perm[k] // group_size`` for a seeded
+  uniform permutation, so every group has exactly ``group_size`` rows.
+
+Value distributions: ``x ~ fp16(N(0,1))``, ``q, z ~ U{0..15}``,
+``scales = fp16(0.002 + |N(0, sigma=0.01)|)``.
+"""
+from __future__ import annotations
+
+import zlib
+from dataclasses import dataclass
+
+import numpy as np
+
+GROUP_SIZE = 128
+SCALE_FLOOR = 0.002
+SCALE_SIGMA = 0.01
+
+# (K, N) of the decoder linears.  Llama-2-7B: hidden 4096, ffn 11008.
+SHAPES_7B = {
+    "qkv": (4096, 12288),
+    "o": (4096, 4096),
+    "gate_up": (4096, 22016),
+    "down": (11008, 4096),
+}
+# Llama-2-13B: hidden 5120, ffn 13824 (the act-order configuration).
+SHAPES_13B = {
+    "qkv": (5120, 15360),
+    "gate_up": (5120, 27648),
+    "down": (13824, 5120),
+}
+LAYERS_7B = 32
+DECODE_M = (1, 4, 8, 16)
+ACT_ORDER_M = (1, 8)
+PREFILL_M = (512, 1024, 2048, 4096)
+STEP_M = (1, 8, 32, 64)
+
+
+def seed_for(*parts) -> int:
+    """Stable 32-bit seed from a tuple of names/numbers (printed in logs)."""
+    return zlib.crc32("/".join(str(p) for p in parts).encode()) & 0xFFFFFFFF
+
+
+def _rng(seed: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def pack_along_k(q: np.ndarray) -> np.ndarray:
+    """uint8[K, N] nibbles -> int32[K/8, N], nibble i of a word = row 8r+i."""
+    K, N = q.shape
+    assert K % 8 == 0
+    q32 = q.astype(np.uint32).reshape(K // 8, 8, N)
+    w = np.zeros((K // 8, N), dtype=np.uint32)
+    for i in range(8):
+        w |= q32[:, i, :] << np.uint32(4 * i)
+    return w.view(np.int32)
+
+
+def pack_along_n(z: np.ndarray) -> np.ndarray:
+    """uint8[G, N] nibbles -> int32[G, N/8], nibble j of a word = column 8c+j."""
+    G, N = z.shape
+    assert N % 8 == 0
+    z32 = z.astype(np.uint32).reshape(G, N // 8, 8)
+    w = np.zeros((G, N // 8), dtype=np.uint32)
+    for j in range(8):
+        w |= z32[:, :, j] << np.uint32(4 * j)
+    return w.view(np.int32)
+
+
+@dataclass
+class QuantLinear:
+    """One GPTQ linear layer in checkpoint (canonical) layout, host arrays."""
+    K: int
+    N: int
+    group_size: int
+    qweight: np.ndarray          # int32[K/8, N]
+    qzeros: np.ndarray           # int32[G, N/8]
+    scales: np.ndarray           # float16[G, N]
+    g_idx: np.ndarray | None     # int32[K] or None
+    seed: int
+
+    @property
+    def act_order(self) -> bool:
+        return self.g_idx is not None
+
+    @property
+    def G(self) -> int:
+        return self.K // self.group_size
+
+
+def make_scales(G: int, N: int, seed: int) -> np.ndarray:
+    r = _rng(seed)
+    s = SCALE_FLOOR + np.abs(r.standard_normal((G, N), dtype=np.float32) * SCALE_SIGMA)
+    return s.astype(np.float16)
+
+
+def make_g_idx(K: int, group_size: int, seed: int) -> np.ndarray:
+    perm = _rng(seed).permutation(K)
+    return (perm // group_size).astype(np.int32)
+
+
+def make_linear(K: int, N: int, seed: int, group_size: int = GROUP_SIZE,
+                act_order: bool = False) -> QuantLinear:
+    """Random GPTQ layer.  Packed words are drawn directly as uniform 32-bit
+    integers, which makes every nibble uniform on 0..15 and independent."""
+    assert K % 8 == 0 and N % 8 == 0 and K % group_size == 0
+    G = K // group_size
+    r = _rng(seed)
+    qweight = r.integers(0, 1 << 32, size=(K // 8, N), dtype=np.uint32).view(np.int32)
+    qzeros = r.integers(0, 1 << 32, size=(G, N // 8), dtype=np.uint32).view(np.int32)
+    scales = make_scales(G, N, seed ^ 0x5CA1E5)
+    g_idx = make_g_idx(K, group_size, seed ^ 0x61D7) if act_order else None
+    return QuantLinear(K, N, group_size, qweight, qzeros, scales, g_idx, seed)
+
+
+def make_linear_from_values(q: np.ndarray, z: np.ndarray, scales: np.ndarray,
+                            group_size: int, g_idx: np.ndarray | None = None) -> QuantLinear:
+    """Encode caller-chosen nibbles (tests use this for hand-built cases)."""
+    K, N = q.shape
+    return QuantLinear(K, N, group_size, pack_along_k(q), pack_along_n(z),
+                       np.ascontiguousarray(scales, dtype=np.float16),
+                       None if g_idx is None else np.ascontiguousarray(g_idx, dtype=np.int32), 0)
+
+
+def make_x(M: int, K: int, seed: int) -> np.ndarray:
+    return _rng(seed).standard_normal((M, K), dtype=np.float32).astype(np.float16)
+
+
+def algorithmic_bytes(M: int, K: int, N: int, group_size: int = GROUP_SIZE,
+                      act_order: bool = False) -> int:
+    """Bytes the matmul must move: packed weights, scales, packed zeros,
+    x, y and (act-order) the row permutation."""
+    G = K // group_size
+    b = K * N // 2 + G * N * 2 + G * N // 2 + M * K * 2 + M * N * 2
+    if act_order:
+        b += 4 * K
+    return b
+
+
+def matmul_flops(M: int, K: int, N: int) -> int:
+    return 2 * M * K * N

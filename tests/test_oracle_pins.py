@@ -1,0 +1,278 @@
+"""Pins for the CPU oracle (no GPU needed).
+
+The oracle is what every CUDA result is compared with, so it is checked here
+against things that are not itself: a hand-packed layer decoded by hand,
+brute force with exact rational arithmetic, closed forms, and special cases
+that reduce to textbook results.  The paper (Opt4GPTQ) prints no value for the
+matmul, so none of these is a printed example; they pin the definition.
+"""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2511_19438_b200 import workloads as wl
+from tests.golden.loader import hex_words, load_fixture, numbers
+
+
+# --------------------------------------------------------------------------- helpers
+def local_pack_words(nibbles_8):
+    """Test-local packer, written independently of the generator module: builds the
+    32-bit word digit by digit from Python ints (nibble 0 is the least significant)."""
+    word = 0
+    for i, v in enumerate(nibbles_8):
+        assert 0 <= int(v) <= 15
+        word += int(v) * (16 ** i)
+    return word
+
+
+def local_pack_k(q):
+    K, N = q.shape
+    out = np.zeros((K // 8, N), dtype=np.uint32)
+    for r in range(K // 8):
+        for n in range(N):
+            out[r, n] = local_pack_words(q[8 * r:8 * r + 8, n])
+    return out.view(np.int32)
+
+
+def local_pack_n(z):
+    G, N = z.shape
+    out = np.zeros((G, N // 8), dtype=np.uint32)
+    for g in range(G):
+        for c in range(N // 8):
+            out[g, c] = local_pack_words(z[g, 8 * c:8 * c + 8])
+    return out.view(np.int32)
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    f = load_fixture("tiny_k16_n8.txt")
+    return dict(
+        K=f["K"], N=f["N"], gs=f["group_size"],
+        qweight=hex_words(f["qweight"]), qzeros=hex_words(f["qzeros"]),
+        q=numbers(f["q"], np.int64), z=numbers(f["z"], np.int64),
+        scales=numbers(f["scales"], np.float16), g_idx=numbers(f["g_idx"], np.int32)[0],
+        x=numbers(f["x"], np.float16),
+    )
+
+
+# --------------------------------------------------------------------------- fp16 decode
+def test_half_to_float_all_bit_patterns():
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.half_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+
+
+# --------------------------------------------------------------------------- hand-packed layer
+def test_fixture_shapes(tiny):
+    assert tiny["qweight"].shape == (2, 8) and tiny["qzeros"].shape == (2, 1)
+    assert tiny["q"].shape == (16, 8) and tiny["z"].shape == (2, 8)
+
+
+def test_unpack_matches_hand_decoded_nibbles(tiny):
+    assert np.array_equal(oracle.unpack_q(tiny["qweight"]), tiny["q"].astype(np.uint8))
+    assert np.array_equal(oracle.unpack_z(tiny["qzeros"]), tiny["z"].astype(np.uint8))
+
+
+def test_dequant_matches_hand_tables(tiny):
+    q, z, s, gs = tiny["q"], tiny["z"], tiny["scales"].astype(np.float64), tiny["gs"]
+    w = oracle.dequant_f32(tiny["qweight"], tiny["qzeros"], tiny["scales"], None, gs)
+    for k in range(16):
+        for n in range(8):
+            assert float(w[k, n]) == float((q[k, n] - z[k // gs, n]) * s[k // gs, n]), (k, n)
+    # a few entries written out literally: (q - z) * s
+    assert w[0, 0] == -1.0          # (0 - 1) * 1
+    assert w[7, 5] == 1.125         # (15 - 6) * 0.125
+    assert w[15, 7] == -0.125       # (13 - 15) * 0.0625
+    assert w[8, 3] == 4.0           # (15 - 13) * 2
+    assert w[3, 6] == 8.0           # (9 - 7) * 4
+
+
+def test_dequant_act_order_matches_hand_tables(tiny):
+    q, z, s, g_idx = tiny["q"], tiny["z"], tiny["scales"].astype(np.float64), tiny["g_idx"]
+    w = oracle.dequant_f32(tiny["qweight"], tiny["qzeros"], tiny["scales"], g_idx, tiny["gs"])
+    for k in range(16):
+        g = int(g_idx[k])
+        for n in range(8):
+            assert float(w[k, n]) == float((q[k, n] - z[g, n]) * s[g, n]), (k, n)
+    assert w[1, 0] == -1.0          # row 1 is in group 1: (1 - 3) * 0.5
+    assert w[9, 7] == 6.0           # row 9 is in group 0: (14 - 8) * 1
+
+
+def brute_force_y(x, q, z, s, groups):
+    """Exact rational y[m][n] from the hand tables."""
+    M, K = x.shape
+    N = q.shape[1]
+    y = [[Fraction(0) for _ in range(N)] for _ in range(M)]
+    for m in range(M):
+        for n in range(N):
+            acc = Fraction(0)
+            for k in range(K):
+                g = groups[k]
+                acc += Fraction(float(x[m, k])) * (int(q[k, n]) - int(z[g, n])) * Fraction(float(s[g, n]))
+            y[m][n] = acc
+    return y
+
+
+@pytest.mark.parametrize("act_order", [False, True])
+def test_gemm_matches_rational_brute_force(tiny, act_order):
+    g_idx = tiny["g_idx"] if act_order else None
+    groups = [int(g) for g in tiny["g_idx"]] if act_order else [k // tiny["gs"] for k in range(16)]
+    want = brute_force_y(tiny["x"], tiny["q"], tiny["z"], tiny["scales"], groups)
+    got = oracle.gemm_f64(tiny["x"], tiny["qweight"], tiny["qzeros"], tiny["scales"], g_idx, tiny["gs"])
+    for m in range(2):
+        for n in range(8):
+            assert Fraction(float(got[m, n])) == want[m][n], (m, n)
+    if not act_order:
+        # column 0, x = ones: group 0 gives (0+..+7 - 8*1)*1 = 20, group 1 gives (28 - 8*3)*0.5 = 2
+        assert got[0, 0] == 22.0
+
+
+# --------------------------------------------------------------------------- invariants
+@pytest.mark.parametrize("K,N,gs,seed", [(32, 16, 8, 1), (256, 24, 128, 2), (384, 40, 128, 3)])
+def test_dequant_of_pack_reproduces_q_minus_z_times_s(K, N, gs, seed):
+    r = np.random.default_rng(seed)
+    G = K // gs
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    z = r.integers(0, 16, (G, N), dtype=np.uint8)
+    s = wl.make_scales(G, N, seed)
+    qw, qz = local_pack_k(q), local_pack_n(z)
+    # the generator's packer must agree with the digit-by-digit one
+    assert np.array_equal(qw, wl.pack_along_k(q)) and np.array_equal(qz, wl.pack_along_n(z))
+    assert np.array_equal(oracle.unpack_q(qw), q) and np.array_equal(oracle.unpack_z(qz), z)
+    w = oracle.dequant_f32(qw, qz, s, None, gs)
+    grp = np.arange(K) // gs
+    want64 = (q.astype(np.int64) - z[grp].astype(np.int64)).astype(np.float64) * s[grp].astype(np.float64)
+    # <= 4 significant bits times <= 11 significant bits: the fp32 product is the exact real product
+    assert np.array_equal(w.astype(np.float64), want64)
+    assert np.array_equal(w, want64.astype(np.float32))
+
+
+def test_act_order_with_trivial_g_idx_is_bit_identical():
+    L = wl.make_linear(512, 64, seed=11)
+    g_idx = (np.arange(512) // 128).astype(np.int32)
+    a = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, None, 128)
+    b = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, g_idx, 128)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+    x = wl.make_x(3, 512, 12)
+    ya = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128)
+    yb = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, g_idx, 128)
+    assert np.array_equal(ya, yb)
+
+
+def test_row_permutation_leaves_y_unchanged():
+    """Permuting (rows of q, entries of g_idx, columns of x) by the same permutation
+    is a reordering of the sum over k only."""
+    K, N, gs = 512, 48, 128
+    L = wl.make_linear(K, N, seed=21, act_order=True)
+    x = wl.make_x(4, K, 22)
+    y0 = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs)
+    p = np.random.default_rng(23).permutation(K)
+    q = oracle.unpack_q(L.qweight)
+    qw_p = local_pack_k(q[p])
+    y1 = oracle.gemm_f64(np.ascontiguousarray(x[:, p]), qw_p, L.qzeros, L.scales, L.g_idx[p], gs)
+    assert np.allclose(y0, y1, rtol=1e-12, atol=1e-12)
+    assert not np.allclose(y0, oracle.gemm_f64(x, qw_p, L.qzeros, L.scales, L.g_idx[p], gs), atol=1e-3)
+
+
+# --------------------------------------------------------------------------- GEMM special cases
+def test_one_hot_x_selects_a_row_of_w():
+    L = wl.make_linear(256, 32, seed=31, act_order=True)
+    w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    for k in (0, 7, 8, 129, 255):
+        x = np.zeros((1, 256), dtype=np.float16)
+        x[0, k] = 1.0
+        y = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+        assert np.array_equal(y[0], w[k].astype(np.float64))
+
+
+def test_all_ones_x_gives_column_sums():
+    L = wl.make_linear(384, 24, seed=41)
+    w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, None, 128).astype(np.float64)
+    y = oracle.gemm_f64(np.ones((1, 384), dtype=np.float16), L.qweight, L.qzeros, L.scales, None, 128)
+    for n in range(24):
+        assert abs(y[0, n] - math.fsum(w[:, n])) <= 1e-12 * max(1.0, abs(y[0, n]))
+
+
+def test_integer_case_is_an_exact_integer_matrix_product():
+    """z = 8, s = 1, small-integer x: y is the integer product x . (q - 8), exact in fp64."""
+    K, N, M, gs = 256, 40, 5, 128
+    r = np.random.default_rng(51)
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    z = np.full((K // gs, N), 8, dtype=np.uint8)
+    s = np.ones((K // gs, N), dtype=np.float16)
+    xi = r.integers(-4, 5, (M, K))
+    L = wl.make_linear_from_values(q, z, s, gs)
+    y = oracle.gemm_f64(xi.astype(np.float16), L.qweight, L.qzeros, L.scales, None, gs)
+    want = xi.astype(np.int64) @ (q.astype(np.int64) - 8)
+    assert np.array_equal(y, want.astype(np.float64))
+
+
+def test_transposed_or_swapped_operands_would_be_caught():
+    """A non-square, non-symmetric case: the result has shape [M, N] and differs from
+    what x^T or W^T conventions would give."""
+    K, N, M, gs = 128, 8, 2, 128
+    q = np.zeros((K, N), dtype=np.uint8)
+    q[5, 3] = 9                       # the only non-zero weight after z = 0
+    z = np.zeros((1, N), dtype=np.uint8)
+    s = np.full((1, N), 0.5, dtype=np.float16)
+    x = np.zeros((M, K), dtype=np.float16)
+    x[1, 5] = 2.0
+    L = wl.make_linear_from_values(q, z, s, gs)
+    y = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, gs)
+    want = np.zeros((M, N))
+    want[1, 3] = 9.0                  # 2 * (9 - 0) * 0.5
+    assert np.array_equal(y, want)
+
+
+def numpy_unpack(qweight, qzeros):
+    K8, N = qweight.shape
+    sh = (4 * np.arange(8, dtype=np.uint32))
+    q = ((qweight.view(np.uint32)[:, None, :] >> sh[None, :, None]) & 15).reshape(K8 * 8, N)
+    z = ((qzeros.view(np.uint32)[:, :, None] >> sh[None, None, :]) & 15).reshape(qzeros.shape[0], N)
+    return q.astype(np.int64), z.astype(np.int64)
+
+
+@pytest.mark.parametrize("K,N,act", [(4096, 4096, False), (5120, 1024, True)])
+def test_against_library_fp64_matmul(K, N, act):
+    """Config-1 shape (and one act-order shape) against numpy's fp64 matmul over a
+    vectorised unpack: a different summation routine over the same definition."""
+    L = wl.make_linear(K, N, seed=wl.seed_for("pin", K, N, act), act_order=act)
+    x = wl.make_x(2, K, wl.seed_for("pin-x", K))
+    q, z = numpy_unpack(L.qweight, L.qzeros)
+    grp = L.g_idx if act else np.arange(K) // 128
+    w = (q - z[grp]).astype(np.float64) * L.scales[grp].astype(np.float64)
+    want = x.astype(np.float64) @ w
+    got = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert np.allclose(got, want, rtol=1e-11, atol=1e-10)
+    # closed-form spread: var(q - z) = 2 * (16^2 - 1) / 12 = 42.5, E[s^2] from the half-normal
+    # scale recipe = 0.002^2 + 2*0.002*0.01*sqrt(2/pi) + 0.01^2, var(x) = 1
+    es2 = wl.SCALE_FLOOR ** 2 + 2 * wl.SCALE_FLOOR * wl.SCALE_SIGMA * math.sqrt(2 / math.pi) + wl.SCALE_SIGMA ** 2
+    std_want = math.sqrt(K * 42.5 * es2)
+    assert abs(got.std() / std_want - 1) < 0.04
+
+
+def test_sampled_outputs_equal_full_product():
+    L = wl.make_linear(256, 64, seed=61, act_order=True)
+    x = wl.make_x(6, 256, 62)
+    full = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    rows = np.array([0, 5, 3, 3, 1], dtype=np.int32)
+    cols = np.array([63, 0, 17, 18, 40], dtype=np.int32)
+    at = oracle.gemm_f64_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128, rows, cols)
+    assert np.array_equal(at, full[rows, cols])
+
+
+def test_generator_distributions():
+    L = wl.make_linear(1024, 512, seed=71, act_order=True)
+    q = oracle.unpack_q(L.qweight)
+    z = oracle.unpack_z(L.qzeros)
+    assert abs(q.mean() - 7.5) < 0.05 and abs(z.mean() - 7.5) < 0.2
+    assert np.bincount(q.ravel(), minlength=16).min() > 0.9 * q.size / 16
+    assert np.array_equal(np.bincount(L.g_idx, minlength=8), np.full(8, 128))
+    s = L.scales.astype(np.float64)
+    assert s.min() >= 0.002 - 1e-5 and abs(s.mean() - (0.002 + 0.01 * math.sqrt(2 / math.pi))) < 2e-4
