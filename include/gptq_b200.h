@@ -1,0 +1,149 @@
+/*
+ * gptq_b200 - GPTQ 4-bit weight-only quantized matmul for NVIDIA B200 (sm_100a).
+ *
+ *     y[M,N] = x[M,K] . dequant(W)[K,N]
+ *
+ * This is the linear-layer product that the Opt4GPTQ paper accelerates (Section 1:
+ * 4-bit GPTQ weights inside every linear layer of the served model; Section 4.2: fp16
+ * activations and fp16 weights after dequantisation).  The paper's three kernel-level
+ * ideas map onto this library as follows: vectorised loads (Section 3.2, Algorithm 2)
+ * become 16-byte-granular bulk copies of re-tiled weights; native packed-half arithmetic
+ * (Section 3.3, Algorithm 3) becomes lop3/sub.f16x2 dequantisation feeding tensor-core
+ * MMAs; block-level pre-reduction with one committing thread (Section 3.1, Algorithm 1)
+ * becomes an fp32 partial-tile workspace reduced in a fixed order by the last-arriving
+ * block, with one plain fp16 store and no global atomics on the output.
+ *
+ * Storage format ("canonical", what checkpoints hold):
+ *   qweight int32[K/8, N]  nibble i (bits 4i..4i+3, word read as unsigned) of word (r,n)
+ *                          is q[8r+i, n] in 0..15
+ *   qzeros  int32[G, N/8]  nibble j of word (g,c) is z[g, 8c+j]; the stored nibble IS the
+ *                          zero point (no +1 offset);  G = K / group_size
+ *   scales  fp16 [G, N]
+ *   g_idx   int32[K]       act-order only: row k uses scale/zero row g_idx[k]
+ *   w[k,n] = (q[k,n] - z[g(k),n]) * scales[g(k),n],  g(k) = g_idx[k] or k / group_size
+ *
+ * All pointers are DEVICE pointers unless a parameter name ends in _host.  The caller owns
+ * every buffer; the library allocates no device memory.  All launches are asynchronous on
+ * the given stream (a cudaStream_t passed as void*; NULL = the default stream).
+ * Every function returns a gptq_status (0 = OK, negative = error); nothing throws, aborts
+ * or traps.  Arguments are validated on the host before any launch.
+ */
+#ifndef GPTQ_B200_H
+#define GPTQ_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GPTQ_OK = 0,
+    GPTQ_ERR_NULL = -1,        /* a required pointer is NULL */
+    GPTQ_ERR_SHAPE = -2,       /* M<1, K%8, N%8, K%group_size, group_size<=0 ... */
+    GPTQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned */
+    GPTQ_ERR_UNSUPPORTED = -4, /* valid GPTQ shape outside the tiled fast path */
+    GPTQ_ERR_LAYOUT = -5,      /* bad `which`/flag argument */
+    GPTQ_ERR_GIDX = -6,        /* g_idx out of range or groups of unequal size */
+    GPTQ_ERR_WORKSPACE = -7,   /* workspace missing or too small for this call */
+    GPTQ_ERR_CUDA = -8,        /* a CUDA runtime call failed (see gptq_last_cuda_error) */
+    GPTQ_ERR_TIMEOUT = -9      /* a bounded device-side wait gave up (see gptq_check_status) */
+} gptq_status;
+
+/* Static description of a status code. */
+const char *gptq_status_string(int status);
+/* cudaError_t of the most recent failing runtime call in this process (0 if none). */
+int gptq_last_cuda_error(void);
+
+/* ---- bit-exact building blocks on the canonical layout (the format reading) -------- */
+
+/* q_out uint8[K,N] and z_out uint8[G,N] (either may be NULL to skip it). */
+int gptq_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out,
+                   int N, int K, int group_size, void *stream);
+
+/* w_out fp32[K,N] = float(q - z) * float(scale), one fp32 multiply (the product is exact).
+ * repacked = 0: inputs are canonical; g_idx is the checkpoint's g_idx when act_order != 0.
+ * repacked = 1: inputs are the buffers written by gptq_repack and g_idx is its perm_out;
+ *               rows are written back in ORIGINAL order, so both modes give identical bits. */
+int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                     float *w_out, int N, int K, int group_size, int act_order, int repacked,
+                     void *stream);
+
+/* ---- one-time repack into the tiled layout the matmul kernels stream ---------------- */
+
+/* Byte size of each gptq_repack output: which = 0 qweight_out, 1 qzeros_out, 2 scales_out,
+ * 3 perm_out (0 bytes unless act_order).  Sizes equal the canonical ones.  Returns 0 for an
+ * invalid argument. */
+size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order);
+
+/* Re-tiles a canonical layer.  Fast-path requirements: group_size == 128, K % 128 == 0,
+ * N % 128 == 0 (else GPTQ_ERR_UNSUPPORTED).  With act_order != 0 the rows are stably sorted
+ * by g_idx so that each group's rows are contiguous; perm_out[i] = original index of sorted
+ * row i (int32[K]).  g_idx is range-checked on the device and every group must have exactly
+ * group_size rows; this one-time call synchronises the stream to report GPTQ_ERR_GIDX.
+ * Outputs must not alias inputs. */
+int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out,
+                int N, int K, int group_size, int act_order, void *stream);
+
+/* ---- the matmul ---------------------------------------------------------------------- */
+
+/* Scratch the matmul may need for this problem (split-K partial tiles and tickets; with
+ * act_order a gathered copy of x).  0 means none. */
+size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order);
+
+/* Registers caller-owned device scratch for later gptq_gemm calls on the current device and
+ * zeroes its ticket area on `stream`.  The workspace is shared by all calls: calls that may
+ * overlap on the GPU (different streams) must not share one.  ptr = NULL unregisters. */
+int gptq_set_workspace(void *ptr, size_t bytes, void *stream);
+
+/* y fp16[M,N] = x fp16[M,K] . dequant(W).  qweight/qzeros/scales are the REPACKED buffers from
+ * gptq_repack; with act_order != 0, g_idx is gptq_repack's perm_out (else it may be NULL).
+ * fp32 accumulation, one round-to-nearest-even conversion to fp16.  Any M >= 1.
+ * The kernels begin fetching weights before earlier work on the stream has finished
+ * (programmatic dependent launch); x, y and the workspace are only touched afterwards.  The
+ * weight buffers must therefore not be written by a kernel launched immediately before this
+ * call on the same stream (gptq_repack itself is safe). */
+int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales,
+              const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
+              void *stream);
+
+/* The same product for callers whose activations live in host memory: copies x_host (pinned
+ * for true asynchrony) to x_stage, runs gptq_gemm, copies y_stage to y_host, all on `stream`.
+ * x_stage (M*K fp16) and y_stage (M*N fp16) are caller-owned device buffers. */
+int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, const void *scales,
+                   const int32_t *g_idx, void *y_host, void *x_stage, void *y_stage,
+                   int M, int N, int K, int group_size, int act_order, void *stream);
+
+/* Synchronises `stream` and returns GPTQ_ERR_TIMEOUT if any kernel's bounded wait gave up
+ * since the last check (the flag is then cleared), GPTQ_ERR_CUDA on a runtime error, else OK. */
+int gptq_check_status(void *stream);
+
+/* ---- host-only: how a problem would be launched (no CUDA call; usable without a GPU) -- */
+
+typedef struct {
+    int kernel;       /* 1 = streaming mma.sync kernel (decode / small batch), 2 = tcgen05 prefill */
+    int m_tile;       /* tokens per CTA tile */
+    int m_chunks;     /* launches along M */
+    int stages;       /* pipeline depth */
+    int ctas;         /* grid size of one launch */
+    int items;        /* (128-column panel, 128-row group) work items of one launch */
+    int split_panels; /* panels whose K range is shared by several CTAs (need the workspace) */
+    int smem_bytes;   /* dynamic shared memory per CTA */
+    size_t workspace_bytes;
+} gptq_plan_t;
+
+int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out);
+
+/* The stream-K partition the kernel uses, from the same arithmetic: CTA `cta` of `ctas` works
+ * through items [*first_item, *end_item) of `items`; the K range of panel `panel` (its `groups`
+ * consecutive items) is shared by CTAs *first_cta .. *last_cta, whose partial tiles are summed
+ * in that order. */
+int gptq_plan_cta_range(int items, int ctas, int cta, int *first_item, int *end_item);
+int gptq_plan_panel_owners(int items, int ctas, int groups, int panel, int *first_cta, int *last_cta);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPTQ_B200_H */

@@ -1,0 +1,173 @@
+"""Thin ctypes binding over libgptq_b200.so - argument marshalling only.
+
+Every function has the name and argument order of its C-ABI entry point
+(``include/gptq_b200.h``).  Device buffers are passed as torch CUDA tensors
+(or raw integer addresses); torch is used for device memory and streams only.
+Nothing here computes: if the compiled library is missing the import of this
+module fails, there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgptq_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2511_19438_b200.build` "
+        "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the GPTQ matmul.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+GPTQ_OK = 0
+GPTQ_ERR_NULL = -1
+GPTQ_ERR_SHAPE = -2
+GPTQ_ERR_ALIGN = -3
+GPTQ_ERR_UNSUPPORTED = -4
+GPTQ_ERR_LAYOUT = -5
+GPTQ_ERR_GIDX = -6
+GPTQ_ERR_WORKSPACE = -7
+GPTQ_ERR_CUDA = -8
+GPTQ_ERR_TIMEOUT = -9
+
+
+class gptq_plan_t(ctypes.Structure):
+    _fields_ = [
+        ("kernel", ctypes.c_int), ("m_tile", ctypes.c_int), ("m_chunks", ctypes.c_int),
+        ("stages", ctypes.c_int), ("ctas", ctypes.c_int), ("items", ctypes.c_int),
+        ("split_panels", ctypes.c_int), ("smem_bytes", ctypes.c_int),
+        ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+_SIGNATURES = {
+    "gptq_status_string": (ctypes.c_char_p, [_i]),
+    "gptq_last_cuda_error": (_i, []),
+    "gptq_unpack_u8": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "gptq_dequant_f32": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "gptq_repack_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "gptq_repack": (_i, [_vp] * 8 + [_i, _i, _i, _i, _vp]),
+    "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "gptq_set_workspace": (_i, [_vp, _sz, _vp]),
+    "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_check_status": (_i, [_vp]),
+    "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
+    "gptq_plan_cta_range": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
+    "gptq_plan_panel_owners": (_i, [_i, _i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+EXPORTED = tuple(_SIGNATURES)
+
+
+class GptqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {gptq_status_string(status)} (status {status})")
+
+
+def _ptr(t):
+    """Address of a torch tensor / numpy array / raw int (None -> NULL)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def check(status: int, where: str) -> None:
+    if status != GPTQ_OK:
+        raise GptqError(status, where)
+
+
+def gptq_status_string(status: int) -> str:
+    return _lib.gptq_status_string(status).decode()
+
+
+def gptq_last_cuda_error() -> int:
+    return _lib.gptq_last_cuda_error()
+
+
+def gptq_unpack_u8(qweight, qzeros, q_out, z_out, N, K, group_size, stream=None) -> int:
+    return _lib.gptq_unpack_u8(_ptr(qweight), _ptr(qzeros), _ptr(q_out), _ptr(z_out), N, K, group_size,
+                               _stream(stream))
+
+
+def gptq_dequant_f32(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked,
+                     stream=None) -> int:
+    return _lib.gptq_dequant_f32(_ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(w_out), N, K,
+                                 group_size, int(act_order), int(repacked), _stream(stream))
+
+
+def gptq_repack_bytes(which, N, K, group_size, act_order) -> int:
+    return _lib.gptq_repack_bytes(which, N, K, group_size, int(act_order))
+
+
+def gptq_repack(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
+                group_size, act_order, stream=None) -> int:
+    return _lib.gptq_repack(_ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(qweight_out),
+                            _ptr(qzeros_out), _ptr(scales_out), _ptr(perm_out), N, K, group_size,
+                            int(act_order), _stream(stream))
+
+
+def gptq_workspace_bytes(M, N, K, group_size, act_order) -> int:
+    return _lib.gptq_workspace_bytes(M, N, K, group_size, int(act_order))
+
+
+def gptq_set_workspace(ptr, nbytes, stream=None) -> int:
+    return _lib.gptq_set_workspace(_ptr(ptr), nbytes, _stream(stream))
+
+
+def gptq_gemm(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
+    return _lib.gptq_gemm(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N, K,
+                          group_size, int(act_order), _stream(stream))
+
+
+def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_stage, M, N, K, group_size,
+                   act_order, stream=None) -> int:
+    return _lib.gptq_gemm_host(_ptr(x_host), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx),
+                               _ptr(y_host), _ptr(x_stage), _ptr(y_stage), M, N, K, group_size,
+                               int(act_order), _stream(stream))
+
+
+def gptq_check_status(stream=None) -> int:
+    return _lib.gptq_check_status(_stream(stream))
+
+
+def gptq_plan(M, N, K, group_size, act_order, sm_count):
+    """Returns (status, gptq_plan_t).  Host-only: makes no CUDA call."""
+    out = gptq_plan_t()
+    st = _lib.gptq_plan(M, N, K, group_size, int(act_order), sm_count, ctypes.byref(out))
+    return st, out
+
+
+def gptq_plan_cta_range(items, ctas, cta):
+    """Returns (status, first_item, end_item)."""
+    a, b = ctypes.c_int(), ctypes.c_int()
+    st = _lib.gptq_plan_cta_range(items, ctas, cta, ctypes.byref(a), ctypes.byref(b))
+    return st, a.value, b.value
+
+
+def gptq_plan_panel_owners(items, ctas, groups, panel):
+    """Returns (status, first_cta, last_cta)."""
+    a, b = ctypes.c_int(), ctypes.c_int()
+    st = _lib.gptq_plan_panel_owners(items, ctas, groups, panel, ctypes.byref(a), ctypes.byref(b))
+    return st, a.value, b.value

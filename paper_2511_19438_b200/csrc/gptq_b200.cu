@@ -1,0 +1,303 @@
+// C ABI of the gptq_b200 library: argument validation, workspace bookkeeping, dispatch.
+// The library is one translation unit; the kernels live in the headers included below.
+#include "gptq_common.cuh"
+#include "gptq_layout.cuh"
+#include "gptq_streamk.cuh"
+
+#include <atomic>
+#include <mutex>
+
+namespace gptq {
+
+static std::atomic<int> g_last_cuda_error{0};
+
+int record_cuda_error(cudaError_t e)
+{
+    if (e == cudaSuccess) return GPTQ_OK;
+    g_last_cuda_error.store((int)e);
+    return GPTQ_ERR_CUDA;
+}
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kTicketAreaBytes = 16384;   // 4096 panels
+constexpr int kStreamKMaxRows = 64;          // tokens per stream-K launch
+
+static Workspace g_workspace[kMaxDevices];
+static int g_sm_count[kMaxDevices];
+static std::mutex g_mutex;
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_shape(int M, int N, int K, int group_size)
+{
+    if (M < 1 || N < 8 || K < 8 || group_size < 1) return GPTQ_ERR_SHAPE;
+    if (K % 8 || N % 8 || K % group_size) return GPTQ_ERR_SHAPE;
+    return GPTQ_OK;
+}
+static int check_fast_path(int N, int K, int group_size)
+{
+    if (group_size != kGroup || N % kPanel || K % kGroup) return GPTQ_ERR_UNSUPPORTED;
+    if (N / kPanel > (int)(kTicketAreaBytes / sizeof(int))) return GPTQ_ERR_UNSUPPORTED;
+    return GPTQ_OK;
+}
+
+static int current_device_sms(int *dev_out, int *sms_out)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= kMaxDevices) return GPTQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_sm_count[dev] == 0) {
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        g_sm_count[dev] = sms;
+    }
+    *dev_out = dev;
+    *sms_out = g_sm_count[dev];
+    return GPTQ_OK;
+}
+
+struct GemmPlan {
+    StreamKPlan sk;          // plan of one launch (for the largest chunk)
+    int m_chunks;
+    size_t x_perm_bytes;     // gathered activations (act-order)
+    size_t workspace_bytes;  // 0 if nothing is needed
+};
+
+static GemmPlan make_plan(int M, int N, int K, int act_order, int sm_count)
+{
+    GemmPlan gp{};
+    const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
+    gp.sk = plan_streamk(rows, N, K, sm_count);
+    gp.m_chunks = (M + kStreamKMaxRows - 1) / kStreamKMaxRows;
+    gp.x_perm_bytes = act_order ? (((size_t)M * K * sizeof(__half) + 255) & ~(size_t)255) : 0;
+    const size_t need = gp.sk.partial_bytes + gp.x_perm_bytes;
+    gp.workspace_bytes = need ? kTicketAreaBytes + need : 0;
+    return gp;
+}
+
+}  // namespace gptq
+
+using namespace gptq;
+
+extern "C" {
+
+const char *gptq_status_string(int status)
+{
+    switch (status) {
+    case GPTQ_OK: return "ok";
+    case GPTQ_ERR_NULL: return "a required pointer is NULL";
+    case GPTQ_ERR_SHAPE: return "invalid shape (need M>=1, K%8==0, N%8==0, K%group_size==0)";
+    case GPTQ_ERR_ALIGN: return "a pointer is not 16-byte aligned";
+    case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 128, N%128==0, K%128==0, equal groups)";
+    case GPTQ_ERR_LAYOUT: return "invalid layout selector or flag";
+    case GPTQ_ERR_GIDX: return "g_idx entry out of range";
+    case GPTQ_ERR_WORKSPACE: return "workspace missing or too small (see gptq_workspace_bytes)";
+    case GPTQ_ERR_CUDA: return "a CUDA runtime call failed (see gptq_last_cuda_error)";
+    case GPTQ_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown status";
+    }
+}
+
+int gptq_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+int gptq_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out, int N, int K,
+                   int group_size, void *stream)
+{
+    if ((q_out && !qweight) || (z_out && !qzeros) || (!q_out && !z_out)) return GPTQ_ERR_NULL;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    return launch_unpack_u8(qweight, qzeros, q_out, z_out, N, K, K / group_size, (cudaStream_t)stream);
+}
+
+int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                     float *w_out, int N, int K, int group_size, int act_order, int repacked, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !w_out || (act_order && !g_idx)) return GPTQ_ERR_NULL;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    if (repacked != 0 && repacked != 1) return GPTQ_ERR_LAYOUT;
+    if (repacked) {
+        st = check_fast_path(N, K, group_size);
+        if (st) return st;
+    }
+    return launch_dequant_f32(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked,
+                              (cudaStream_t)stream);
+}
+
+size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order)
+{
+    if (check_shape(1, N, K, group_size) != GPTQ_OK) return 0;
+    const size_t G = (size_t)(K / group_size);
+    switch (which) {
+    case 0: return (size_t)K / 8 * N * 4;
+    case 1: return G * (N / 8) * 4;
+    case 2: return G * N * 2;
+    case 3: return act_order ? (size_t)K * 4 : 0;
+    default: return 0;
+    }
+}
+
+int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
+                int group_size, int act_order, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out) return GPTQ_ERR_NULL;
+    if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    st = check_fast_path(N, K, group_size);
+    if (st) return st;
+    if (!aligned16(qweight_out) || !aligned16(qzeros_out) || !aligned16(scales_out)) return GPTQ_ERR_ALIGN;
+    if (qweight_out == (const void *)qweight || qzeros_out == (const void *)qzeros || scales_out == scales)
+        return GPTQ_ERR_LAYOUT;
+    return launch_repack(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
+                         act_order, (cudaStream_t)stream);
+}
+
+int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out)
+{
+    if (!out) return GPTQ_ERR_NULL;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    st = check_fast_path(N, K, group_size);
+    if (st) return st;
+    if (sm_count < 1) return GPTQ_ERR_SHAPE;
+    const GemmPlan gp = make_plan(M, N, K, act_order, sm_count);
+    out->kernel = 1;
+    out->m_tile = gp.sk.m_tile;
+    out->m_chunks = gp.m_chunks;
+    out->stages = gp.sk.stages;
+    out->ctas = gp.sk.ctas;
+    out->items = gp.sk.items;
+    out->split_panels = gp.sk.split_panels;
+    out->smem_bytes = gp.sk.smem_bytes;
+    out->workspace_bytes = gp.workspace_bytes;
+    return GPTQ_OK;
+}
+
+int gptq_plan_cta_range(int items, int ctas, int cta, int *first_item, int *end_item)
+{
+    if (!first_item || !end_item) return GPTQ_ERR_NULL;
+    if (items < 1 || ctas < 1 || ctas > items || cta < 0 || cta >= ctas) return GPTQ_ERR_SHAPE;
+    *first_item = sk_range_begin(items, ctas, cta);
+    *end_item = sk_range_begin(items, ctas, cta + 1);
+    return GPTQ_OK;
+}
+
+int gptq_plan_panel_owners(int items, int ctas, int groups, int panel, int *first_cta, int *last_cta)
+{
+    if (!first_cta || !last_cta) return GPTQ_ERR_NULL;
+    if (items < 1 || ctas < 1 || ctas > items || groups < 1 || items % groups || panel < 0 ||
+        panel >= items / groups)
+        return GPTQ_ERR_SHAPE;
+    const long long first_item = (long long)panel * groups;
+    *first_cta = sk_owner(items, ctas, first_item);
+    *last_cta = sk_owner(items, ctas, first_item + groups - 1);
+    return GPTQ_OK;
+}
+
+size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order)
+{
+    if (check_shape(M, N, K, group_size) != GPTQ_OK || check_fast_path(N, K, group_size) != GPTQ_OK) return 0;
+    int dev, sms;
+    if (current_device_sms(&dev, &sms) != GPTQ_OK) return 0;
+    return make_plan(M, N, K, act_order, sms).workspace_bytes;
+}
+
+int gptq_set_workspace(void *ptr, size_t bytes, void *stream)
+{
+    int dev, sms;
+    int st = current_device_sms(&dev, &sms);
+    if (st) return st;
+    if (ptr == nullptr) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        g_workspace[dev] = Workspace{};
+        return GPTQ_OK;
+    }
+    if (!aligned16(ptr)) return GPTQ_ERR_ALIGN;
+    if (bytes < kTicketAreaBytes) return GPTQ_ERR_WORKSPACE;
+    st = record_cuda_error(cudaMemsetAsync(ptr, 0, kTicketAreaBytes, (cudaStream_t)stream));
+    if (st) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_workspace[dev].ptr = ptr;
+    g_workspace[dev].bytes = bytes;
+    return GPTQ_OK;
+}
+
+int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+              void *y, int M, int N, int K, int group_size, int act_order, void *stream)
+{
+    if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
+        return GPTQ_ERR_ALIGN;
+    st = check_fast_path(N, K, group_size);
+    if (st) return st;
+
+    int dev, sms;
+    st = current_device_sms(&dev, &sms);
+    if (st) return st;
+    const GemmPlan gp = make_plan(M, N, K, act_order, sms);
+    Workspace ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace[dev];
+    }
+    if (gp.workspace_bytes > 0 && (ws.ptr == nullptr || ws.bytes < gp.workspace_bytes)) return GPTQ_ERR_WORKSPACE;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t *wsb = (uint8_t *)ws.ptr;
+    int *tickets = (int *)wsb;
+    float *partials = gp.workspace_bytes ? (float *)(wsb + kTicketAreaBytes) : nullptr;
+    const __half *xin = (const __half *)x;
+    if (act_order) {
+        __half *x_perm = (__half *)(wsb + kTicketAreaBytes + gp.sk.partial_bytes);
+        st = launch_gather_x((const __half *)x, g_idx, x_perm, M, K, s);
+        if (st) return st;
+        xin = x_perm;
+    }
+    for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
+        const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
+        const StreamKPlan pl = plan_streamk(rows, N, K, sms);
+        st = launch_streamk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
+                            pl, partials, tickets, s);
+        if (st) return st;
+    }
+    return GPTQ_OK;
+}
+
+int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, const void *scales,
+                   const int32_t *g_idx, void *y_host, void *x_stage, void *y_stage, int M, int N, int K,
+                   int group_size, int act_order, void *stream)
+{
+    if (!x_host || !y_host || !x_stage || !y_stage) return GPTQ_ERR_NULL;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    st = record_cuda_error(cudaMemcpyAsync(x_stage, x_host, (size_t)M * K * sizeof(__half), cudaMemcpyHostToDevice, s));
+    if (st) return st;
+    st = gptq_gemm(x_stage, qweight, qzeros, scales, g_idx, y_stage, M, N, K, group_size, act_order, stream);
+    if (st) return st;
+    return record_cuda_error(cudaMemcpyAsync(y_host, y_stage, (size_t)M * N * sizeof(__half), cudaMemcpyDeviceToHost, s));
+}
+
+int gptq_check_status(void *stream)
+{
+    cudaStream_t s = (cudaStream_t)stream;
+    int status = 0;
+    cudaError_t e = cudaMemcpyFromSymbolAsync(&status, g_device_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (status == kStatusOk) return GPTQ_OK;
+    int zero = 0;
+    e = cudaMemcpyToSymbolAsync(g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    return status == kStatusWaitTimeout ? GPTQ_ERR_TIMEOUT : GPTQ_ERR_GIDX;
+}
+
+}  // extern "C"

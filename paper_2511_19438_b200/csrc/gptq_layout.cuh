@@ -1,0 +1,243 @@
+// Format kernels: nibble unpack, fp32 dequantisation (canonical and tiled layouts), the
+// one-time repack into the tiled layout, and the activation gather used with act-order.
+// All of them are plain element-per-thread kernels; none is on the per-token path except
+// gather_x (act-order only).
+#pragma once
+#include "gptq_common.cuh"
+
+namespace gptq {
+
+// ------------------------------------------------------------------------------ unpack
+__global__ void unpack_q_kernel(const int32_t *__restrict__ qweight, uint8_t *__restrict__ q_out, int N, int K)
+{
+    // one thread per packed word: writes its 8 rows of one column
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t words = (size_t)(K / 8) * N;
+    if (idx >= words) return;
+    int r = (int)(idx / N), n = (int)(idx % N);
+    uint32_t w = (uint32_t)qweight[idx];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q_out[(size_t)(8 * r + i) * N + n] = (uint8_t)((w >> (4 * i)) & 15u);
+}
+
+__global__ void unpack_z_kernel(const int32_t *__restrict__ qzeros, uint8_t *__restrict__ z_out, int N, int G)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t words = (size_t)G * (N / 8);
+    if (idx >= words) return;
+    uint32_t w = (uint32_t)qzeros[idx];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) z_out[idx * 8 + j] = (uint8_t)((w >> (4 * j)) & 15u);
+}
+
+int launch_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out, int N, int K,
+                     int G, cudaStream_t s)
+{
+    const int T = 256;
+    if (q_out) {
+        size_t words = (size_t)(K / 8) * N;
+        unpack_q_kernel<<<(unsigned)((words + T - 1) / T), T, 0, s>>>(qweight, q_out, N, K);
+    }
+    if (z_out) {
+        size_t words = (size_t)G * (N / 8);
+        unpack_z_kernel<<<(unsigned)((words + T - 1) / T), T, 0, s>>>(qzeros, z_out, N, G);
+    }
+    return record_cuda_error(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------ dequant fp32
+// One thread per (k, n).  float(q - z) * float(s): a single fp32 multiply whose result is exact.
+__global__ void dequant_canonical_kernel(const int32_t *__restrict__ qweight, const int32_t *__restrict__ qzeros,
+                                         const __half *__restrict__ scales, const int32_t *__restrict__ g_idx,
+                                         float *__restrict__ w_out, int N, int K, int group_size)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)K * N) return;
+    int k = (int)(idx / N), n = (int)(idx % N);
+    int g = g_idx ? g_idx[k] : k / group_size;
+    int q = (int)(((uint32_t)qweight[(size_t)(k >> 3) * N + n] >> (4 * (k & 7))) & 15u);
+    int z = (int)(((uint32_t)qzeros[(size_t)g * (N / 8) + (n >> 3)] >> (4 * (n & 7))) & 15u);
+    w_out[idx] = __fmul_rn((float)(q - z), __half2float(scales[(size_t)g * N + n]));
+}
+
+// Tiled layout: thread per (sorted row i, column n); the row goes back to its original index.
+__global__ void dequant_tiled_kernel(const uint8_t *__restrict__ qweight, const uint8_t *__restrict__ qzeros,
+                                     const __half *__restrict__ scales, const int32_t *__restrict__ perm,
+                                     float *__restrict__ w_out, int N, int K)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)K * N) return;
+    int i = (int)(idx / N), n = (int)(idx % N);
+    int G = K / kGroup, grp = i / kGroup;
+    int slot, hi;
+    size_t off = repacked_word_offset(i, n, G, &slot);
+    uint32_t word = *reinterpret_cast<const uint32_t *>(qweight + off);
+    int q = (int)((word >> (4 * slot)) & 15u);
+    uint8_t zb = qzeros[repacked_zero_byte(grp, n, G, &hi)];
+    int z = hi ? (zb >> 4) : (zb & 15);
+    float s = __half2float(scales[repacked_scale_index(grp, n, G)]);
+    int k = perm ? perm[i] : i;
+    w_out[(size_t)k * N + n] = __fmul_rn((float)(q - z), s);
+}
+
+int launch_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                       float *w_out, int N, int K, int group_size, int act_order, int repacked, cudaStream_t s)
+{
+    const int T = 256;
+    size_t total = (size_t)K * N;
+    unsigned blocks = (unsigned)((total + T - 1) / T);
+    if (repacked)
+        dequant_tiled_kernel<<<blocks, T, 0, s>>>((const uint8_t *)qweight, (const uint8_t *)qzeros,
+                                                  (const __half *)scales, act_order ? g_idx : nullptr, w_out, N, K);
+    else
+        dequant_canonical_kernel<<<blocks, T, 0, s>>>((const int32_t *)qweight, (const int32_t *)qzeros,
+                                                      (const __half *)scales, act_order ? g_idx : nullptr, w_out,
+                                                      N, K, group_size);
+    return record_cuda_error(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------ act-order sort
+// perm = stable argsort(g_idx).  Thread k counts the keys that sort before its own:
+// rank(k) = #{k' : g[k'] < g[k]} + #{k' < k : g[k'] == g[k]}.  O(K^2) compares, one-time, K <= ~16k.
+// Also checks 0 <= g[k] < G and that every group has exactly 128 rows.
+__global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *__restrict__ perm, int K, int G)
+{
+    extern __shared__ int32_t tile[];
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    int mine = (k < K) ? g_idx[k] : 0;
+    bool bad = (k < K) && (mine < 0 || mine >= G);
+    int below = 0, same_before = 0, same_total = 0;
+    for (int base = 0; base < K; base += blockDim.x) {
+        int kk = base + threadIdx.x;
+        tile[threadIdx.x] = (kk < K) ? g_idx[kk] : -1;
+        __syncthreads();
+        int lim = min((int)blockDim.x, K - base);
+        for (int j = 0; j < lim; ++j) {
+            int other = tile[j];
+            below += (other < mine);
+            same_total += (other == mine);
+            same_before += (other == mine) && (base + j < k);
+        }
+        __syncthreads();
+    }
+    if (k >= K) return;
+    if (bad) {
+        atomicMax(&g_device_status, (int)kStatusBadGidx);
+        return;
+    }
+    if (same_total != kGroup) atomicMax(&g_device_status, (int)kStatusUnequalGroups);
+    int rank = below + same_before;
+    if (rank >= 0 && rank < K) perm[rank] = k;
+}
+
+// ------------------------------------------------------------------------------ repack
+// One thread per output word of the tiled layout.
+__global__ void repack_weights_kernel(const int32_t *__restrict__ qweight, const int32_t *__restrict__ perm,
+                                      uint32_t *__restrict__ out, int N, int K)
+{
+    size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t words = (size_t)(K / 8) * N;
+    if (o >= words) return;
+    int G = K / kGroup;
+    // decode the output word index: [item][blk(2)][unit(8)][lane(32)][c(4)]
+    int c = (int)(o & 3), lane = (int)((o >> 2) & 31), u = (int)((o >> 7) & 7), blk = (int)((o >> 10) & 1);
+    size_t item = o >> 11;
+    int p = (int)(item / G), grp = (int)(item % G);
+    int g = lane >> 2, t4 = lane & 3, j = c & 1, h = c >> 1;
+    int n = p * kPanel + 16 * u + g + 8 * h;
+    int i0 = grp * kGroup + blk * 64 + j * 32 + t4 * 8;
+    uint32_t word = 0;
+    if (perm == nullptr) {
+        uint32_t src = (uint32_t)qweight[(size_t)(i0 >> 3) * N + n];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) word |= ((src >> (4 * e)) & 15u) << (4 * nibble_slot(e));
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            int k = perm[i0 + e];
+            uint32_t q = ((uint32_t)qweight[(size_t)(k >> 3) * N + n] >> (4 * (k & 7))) & 15u;
+            word |= q << (4 * nibble_slot(e));
+        }
+    }
+    out[o] = word;
+}
+
+// One thread per (group, column): scale to its tiled position; thread with h == 0 also writes the
+// zero byte of its column pair.
+__global__ void repack_meta_kernel(const int32_t *__restrict__ qzeros, const __half *__restrict__ scales,
+                                   uint8_t *__restrict__ z_out, __half *__restrict__ s_out, int N, int G)
+{
+    size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)G * N) return;
+    int grp = (int)(idx / N), n = (int)(idx % N);
+    s_out[repacked_scale_index(grp, n, G)] = scales[idx];
+    if (((n % 16) >> 3) == 0) {
+        const int32_t *zrow = qzeros + (size_t)grp * (N / 8);
+        uint32_t za = ((uint32_t)zrow[n >> 3] >> (4 * (n & 7))) & 15u;
+        int nb = n + 8;
+        uint32_t zb = ((uint32_t)zrow[nb >> 3] >> (4 * (nb & 7))) & 15u;
+        int hi;
+        z_out[repacked_zero_byte(grp, n, G, &hi)] = (uint8_t)(za | (zb << 4));
+    }
+}
+
+// Ends the repack with an ordinary (fully stream-ordered) kernel boundary, so that a matmul
+// launched right after it with programmatic dependent launch cannot fetch weights early.
+__global__ void repack_fence_kernel() {}
+
+int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                  void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
+                  int act_order, cudaStream_t s)
+{
+    const int T = 256;
+    int G = K / kGroup;
+    if (act_order) {
+        int blocks = (K + T - 1) / T;
+        argsort_gidx_kernel<<<blocks, T, T * sizeof(int32_t), s>>>(g_idx, perm_out, K, G);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return record_cuda_error(e);
+        // one-time call: read the validation result before tiling with a possibly invalid perm
+        int status = 0;
+        e = cudaMemcpyFromSymbolAsync(&status, g_device_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        if (status == kStatusBadGidx || status == kStatusUnequalGroups) {
+            int zero = 0;
+            e = cudaMemcpyToSymbolAsync(g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+            if (e != cudaSuccess) return record_cuda_error(e);
+            return status == kStatusBadGidx ? GPTQ_ERR_GIDX : GPTQ_ERR_UNSUPPORTED;
+        }
+    }
+    size_t words = (size_t)(K / 8) * N;
+    repack_weights_kernel<<<(unsigned)((words + T - 1) / T), T, 0, s>>>(qweight, act_order ? perm_out : nullptr,
+                                                                        (uint32_t *)qweight_out, N, K);
+    size_t meta = (size_t)G * N;
+    repack_meta_kernel<<<(unsigned)((meta + T - 1) / T), T, 0, s>>>(qzeros, (const __half *)scales,
+                                                                    (uint8_t *)qzeros_out, (__half *)scales_out, N, G);
+    repack_fence_kernel<<<1, 32, 0, s>>>();
+    return record_cuda_error(cudaGetLastError());
+}
+
+// ------------------------------------------------------------------------------ gather x
+// x_out[m][i] = x[m][perm[i]]: puts the activations in the sorted row order of the tiled weights.
+__global__ void gather_x_kernel(const __half *__restrict__ x, const int32_t *__restrict__ perm,
+                                __half *__restrict__ x_out, int M, int K)
+{
+    pdl_launch_dependents();   // the matmul that follows may start fetching weights now
+    pdl_wait();                // x may come from the kernel just before this one
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K) return;
+    int src = perm[i];
+    for (int m = blockIdx.y; m < M; m += gridDim.y) x_out[(size_t)m * K + i] = x[(size_t)m * K + src];
+}
+
+int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, int K, cudaStream_t s)
+{
+    const int T = 256;
+    dim3 grid((K + T - 1) / T, (unsigned)min(M, 64));
+    gather_x_kernel<<<grid, T, 0, s>>>(x, perm, x_out, M, K);
+    return record_cuda_error(cudaGetLastError());
+}
+
+}  // namespace gptq

@@ -1,0 +1,78 @@
+"""Device-side plumbing for tests and the benchmark: uploads a synthetic layer,
+runs the one-time repack through the C ABI, keeps the workspace registered.
+
+torch is used only to own device memory and streams; every computation is a
+call into libgptq_b200.so through ``binding``.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import binding as B
+from .workloads import QuantLinear
+
+
+@dataclass
+class DeviceLinear:
+    """A layer resident on the GPU: canonical buffers (optional) and the tiled ones."""
+    K: int
+    N: int
+    group_size: int
+    act_order: bool
+    qweight_t: torch.Tensor      # tiled
+    qzeros_t: torch.Tensor
+    scales_t: torch.Tensor
+    perm: torch.Tensor | None    # int32[K], original index of sorted row i
+    canonical: tuple | None      # (qweight, qzeros, scales, g_idx) device tensors, if kept
+
+
+def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda") -> DeviceLinear:
+    qw = to_device(L.qweight, device)
+    qz = to_device(L.qzeros, device)
+    sc = to_device(L.scales, device)
+    gi = to_device(L.g_idx, device) if L.act_order else None
+    qw_t = torch.empty(B.gptq_repack_bytes(0, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
+    qz_t = torch.empty(B.gptq_repack_bytes(1, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
+    sc_t = torch.empty(B.gptq_repack_bytes(2, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
+    perm = torch.empty(L.K, dtype=torch.int32, device=device) if L.act_order else None
+    B.check(B.gptq_repack(qw, qz, sc, gi, qw_t, qz_t, sc_t, perm, L.N, L.K, L.group_size, L.act_order), "gptq_repack")
+    torch.cuda.current_stream().synchronize()
+    canonical = (qw, qz, sc, gi) if keep_canonical else None
+    return DeviceLinear(L.K, L.N, L.group_size, L.act_order, qw_t, qz_t, sc_t, perm, canonical)
+
+
+class WorkspaceHolder:
+    """Owns one device scratch buffer and keeps it registered with the library."""
+
+    def __init__(self, device="cuda"):
+        self.device = device
+        self.buf = None
+
+    def ensure(self, nbytes: int) -> None:
+        if nbytes <= 0:
+            return
+        if self.buf is None or self.buf.numel() < nbytes:
+            torch.cuda.synchronize()
+            self.buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        # registering is idempotent and cheap (it re-zeroes the 16 KB ticket area on the stream)
+        B.check(B.gptq_set_workspace(self.buf, self.buf.numel()), "gptq_set_workspace")
+
+    def ensure_for(self, M: int, D: DeviceLinear) -> None:
+        self.ensure(B.gptq_workspace_bytes(M, D.N, D.K, D.group_size, D.act_order))
+
+
+def gemm(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """y = x . dequant(W) through gptq_gemm (x fp16 [M, K] on the device)."""
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, D.N), dtype=torch.float16, device=x.device)
+    B.check(B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, D.N, D.K, D.group_size,
+                        D.act_order, stream), "gptq_gemm")
+    return y

@@ -1,0 +1,156 @@
+"""Host-side checks of the C-ABI library that need no GPU: the shared object loads, exports
+every symbol the header declares, validates arguments before touching CUDA, and plans the
+stream-K partition consistently (every item covered once; the contributors the reducing CTA
+expects are exactly the CTAs that write a partial tile for that panel)."""
+import os
+import re
+
+import pytest
+
+from paper_2511_19438_b200 import build as libbuild
+
+libbuild.build()
+from paper_2511_19438_b200 import binding as B  # noqa: E402
+from paper_2511_19438_b200 import workloads as wl  # noqa: E402
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "gptq_b200.h")
+A16 = 0x1000  # a fake, 16-byte aligned "device address"; validation never dereferences it
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(gptq_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(B._lib, n), f"{n} declared in the header but not exported"
+    assert set(names) == set(B.EXPORTED), set(names) ^ set(B.EXPORTED)
+
+
+def test_status_strings():
+    assert B.gptq_status_string(0) == "ok"
+    for code in range(-9, 0):
+        assert B.gptq_status_string(code) not in ("ok", "unknown status")
+    assert B.gptq_status_string(-77) == "unknown status"
+
+
+def test_gemm_validation_order_without_gpu():
+    ok = dict(M=1, N=4096, K=4096, group_size=128, act_order=0)
+
+    def call(x=A16, qw=A16, qz=A16, sc=A16, gi=None, y=A16, **kw):
+        a = dict(ok, **kw)
+        return B.gptq_gemm(x, qw, qz, sc, gi, y, a["M"], a["N"], a["K"], a["group_size"], a["act_order"], stream=0)
+
+    assert call(x=None) == B.GPTQ_ERR_NULL
+    assert call(y=None) == B.GPTQ_ERR_NULL
+    assert call(act_order=1, gi=None) == B.GPTQ_ERR_NULL
+    assert call(M=0) == B.GPTQ_ERR_SHAPE
+    assert call(K=4100) == B.GPTQ_ERR_SHAPE          # K % 8
+    assert call(N=4097) == B.GPTQ_ERR_SHAPE
+    assert call(K=4096 + 64) == B.GPTQ_ERR_SHAPE     # K % group_size
+    assert call(group_size=0) == B.GPTQ_ERR_SHAPE
+    assert call(x=A16 + 8) == B.GPTQ_ERR_ALIGN
+    assert call(qw=A16 + 4) == B.GPTQ_ERR_ALIGN
+    assert call(group_size=64) == B.GPTQ_ERR_UNSUPPORTED
+    assert call(N=4096 + 64) == B.GPTQ_ERR_UNSUPPORTED
+
+
+def test_other_entry_points_validate_without_gpu():
+    assert B.gptq_unpack_u8(None, None, None, None, 128, 128, 128, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_unpack_u8(A16, A16, A16, A16, 130, 128, 128, stream=0) == B.GPTQ_ERR_SHAPE
+    assert B.gptq_dequant_f32(A16, A16, A16, None, None, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_dequant_f32(A16, A16, A16, None, A16, 128, 128, 128, 0, 2, stream=0) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_dequant_f32(A16, A16, A16, None, A16, 64, 128, 128, 0, 1, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack(A16, A16, A16, None, A16 + 16, None, A16, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_repack(A16, A16, A16, None, A16, A16 + 16, A16 + 32, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_repack(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack(A16, A16, A16, A16, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_host(None, A16, A16, A16, None, A16, A16, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+
+
+def test_repack_bytes_equal_canonical_sizes():
+    for (K, N) in list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()):
+        G = K // 128
+        assert B.gptq_repack_bytes(0, N, K, 128, 0) == K * N // 2
+        assert B.gptq_repack_bytes(1, N, K, 128, 0) == G * N // 2
+        assert B.gptq_repack_bytes(2, N, K, 128, 0) == G * N * 2
+        assert B.gptq_repack_bytes(3, N, K, 128, 0) == 0
+        assert B.gptq_repack_bytes(3, N, K, 128, 1) == 4 * K
+    assert B.gptq_repack_bytes(7, 128, 128, 128, 0) == 0
+    assert B.gptq_repack_bytes(0, 129, 128, 128, 0) == 0
+
+
+SHAPES = list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()) + [(128, 128), (256, 384), (1024, 128)]
+
+
+@pytest.mark.parametrize("K,N", SHAPES)
+@pytest.mark.parametrize("M", [1, 8, 9, 16, 33, 64, 200])
+@pytest.mark.parametrize("sms", [148, 132, 7])
+def test_plan_is_consistent(K, N, M, sms):
+    st, pl = B.gptq_plan(M, N, K, 128, 0, sms)
+    assert st == B.GPTQ_OK
+    G, panels = K // 128, N // 128
+    assert pl.items == G * panels
+    assert 1 <= pl.ctas <= min(pl.items, 2 * sms)
+    assert pl.m_tile in (8, 16, 32, 64) and pl.m_tile >= min(M, 64)
+    assert pl.m_chunks == (M + 63) // 64
+    assert 2 <= pl.stages <= 8
+    assert pl.smem_bytes <= 227 * 1024
+    # every item is covered exactly once, ranges are contiguous and balanced within one item
+    end_prev, sizes = 0, []
+    for c in range(pl.ctas):
+        st, a, b = B.gptq_plan_cta_range(pl.items, pl.ctas, c)
+        assert st == B.GPTQ_OK and a == end_prev and b > a
+        sizes.append(b - a)
+        end_prev = b
+    assert end_prev == pl.items and max(sizes) - min(sizes) <= 1
+    # contributors per panel: the reducing CTA's view must match who actually writes partials
+    writers = {}
+    for c in range(pl.ctas):
+        _, a, b = B.gptq_plan_cta_range(pl.items, pl.ctas, c)
+        first_panel = a // G
+        for p in range(a // G, (b - 1) // G + 1):
+            lo, hi = max(a, p * G), min(b, (p + 1) * G)
+            if not (lo == p * G and hi == (p + 1) * G):     # partial segment -> slot 0 or 1
+                writers.setdefault(p, []).append((c, 0 if p == first_panel else 1))
+    split = 0
+    for p in range(panels):
+        st, cf, cl = B.gptq_plan_panel_owners(pl.items, pl.ctas, G, p)
+        assert st == B.GPTQ_OK
+        if cf == cl:
+            assert p not in writers
+            continue
+        split += 1
+        expect = []
+        for cc in range(cf, cl + 1):
+            _, a, _b = B.gptq_plan_cta_range(pl.items, pl.ctas, cc)
+            expect.append((cc, 0 if a // G == p else 1))
+        assert writers[p] == expect
+    assert split == pl.split_panels
+    # slots are never reused by two panels of one CTA
+    used = [w for ws in writers.values() for w in ws]
+    assert len(used) == len(set(used))
+    if split:
+        rows = min(M, 64)
+        assert pl.workspace_bytes >= 16384 + pl.ctas * 2 * rows * 128 * 4
+    else:
+        assert pl.workspace_bytes == 0
+
+
+def test_plan_act_order_adds_gathered_x():
+    st, a = B.gptq_plan(8, 5120, 13824, 128, 0, 148)
+    st2, b = B.gptq_plan(8, 5120, 13824, 128, 1, 148)
+    assert st == st2 == B.GPTQ_OK
+    assert b.workspace_bytes - a.workspace_bytes >= 8 * 13824 * 2 or a.workspace_bytes == 0
+
+
+def test_plan_rejects_bad_arguments():
+    assert B.gptq_plan(1, 4096, 4096, 128, 0, 0)[0] == B.GPTQ_ERR_SHAPE
+    assert B.gptq_plan(1, 4096, 4096, 32, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_plan_cta_range(10, 11, 0)[0] == B.GPTQ_ERR_SHAPE
+    assert B.gptq_plan_panel_owners(10, 5, 3, 0)[0] == B.GPTQ_ERR_SHAPE

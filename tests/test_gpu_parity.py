@@ -1,0 +1,294 @@
+"""GPU parity tests: every result of the CUDA library (called through the C ABI) against the
+CPU oracle on the same seeded inputs.
+
+Bars: unpacked nibbles and fp32 dequantised weights are bit-exact; fp16 matmul outputs are
+within rtol 1e-2 / atol 1e-2*sqrt(K/4096) of the fp64 oracle (the stated tolerance), and also
+within the much tighter bound this implementation should meet (exact integer q - z, fp32
+accumulation, one fp16 rounding: |err| <= 2^-11 |y| + 1e-4 * sqrt(K/4096))."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_19438_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2511_19438_b200 import build as libbuild
+    libbuild.build()
+    from paper_2511_19438_b200 import binding as B
+    from paper_2511_19438_b200 import harness as H
+
+
+@pytest.fixture(scope="module")
+def ws():
+    return H.WorkspaceHolder()
+
+
+def assert_close(y_gpu: np.ndarray, y64: np.ndarray, K: int):
+    y = y_gpu.astype(np.float64)
+    err = np.abs(y - y64)
+    loose = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64)
+    tight = 1e-4 * math.sqrt(K / 4096) + 2.0 ** -11 * np.abs(y64)
+    assert np.all(np.isfinite(y))
+    assert np.all(err <= loose), f"stated tolerance: {int((err > loose).sum())} violations, max err {err.max():.3e}"
+    assert np.all(err <= tight), f"implementation bound: {int((err > tight).sum())} violations, max err {err.max():.3e}"
+
+
+def run_gemm(L, x_np, ws):
+    D = H.upload_and_repack(L)
+    ws.ensure_for(x_np.shape[0], D)
+    y = H.gemm(H.to_device(x_np), D)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    return y.cpu().numpy(), D
+
+
+# ------------------------------------------------------------------------------- bit-exact parts
+@pytest.mark.parametrize("K,N,gs", [(16, 8, 8), (256, 136, 32), (384, 264, 128), (4096, 4096, 128)])
+def test_unpack_bit_exact(K, N, gs):
+    L = wl.make_linear(K, N, seed=wl.seed_for("unpack", K, N), group_size=gs)
+    q = torch.empty((K, N), dtype=torch.uint8, device="cuda")
+    z = torch.empty((K // gs, N), dtype=torch.uint8, device="cuda")
+    B.check(B.gptq_unpack_u8(H.to_device(L.qweight), H.to_device(L.qzeros), q, z, N, K, gs), "unpack")
+    assert np.array_equal(q.cpu().numpy(), oracle.unpack_q(L.qweight))
+    assert np.array_equal(z.cpu().numpy(), oracle.unpack_z(L.qzeros))
+    # either output may be skipped
+    q2 = torch.zeros_like(q)
+    B.check(B.gptq_unpack_u8(H.to_device(L.qweight), None, q2, None, N, K, gs), "unpack q only")
+    assert torch.equal(q, q2)
+
+
+@pytest.mark.parametrize("K,N,gs,act", [(64, 24, 32, False), (512, 136, 64, True), (1024, 264, 128, True),
+                                        (4096, 4096, 128, False)])
+def test_dequant_canonical_bit_exact(K, N, gs, act):
+    L = wl.make_linear(K, N, seed=wl.seed_for("dq", K, N, act), group_size=gs, act_order=act)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    gi = H.to_device(L.g_idx) if act else None
+    B.check(B.gptq_dequant_f32(H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales), gi, w,
+                               N, K, gs, act, 0), "dequant")
+    want = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs)
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("K,N,act", [(128, 128, False), (384, 256, True), (1024, 640, True), (4096, 4096, False),
+                                     (5120, 1280, True)])
+def test_repack_is_lossless_and_sorted(K, N, act):
+    L = wl.make_linear(K, N, seed=wl.seed_for("rp", K, N, act), act_order=act)
+    D = H.upload_and_repack(L)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, 128, act, 1), "dequant tiled")
+    want = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    if act:
+        assert np.array_equal(D.perm.cpu().numpy(), np.argsort(L.g_idx, kind="stable").astype(np.int32))
+
+
+def test_repack_rejects_bad_g_idx():
+    L = wl.make_linear(256, 128, seed=5, act_order=True)
+    bad = L.g_idx.copy()
+    bad[17] = 2                                   # out of range (G = 2)
+    L_bad = wl.QuantLinear(L.K, L.N, 128, L.qweight, L.qzeros, L.scales, bad, 0)
+    with pytest.raises(B.GptqError) as e:
+        H.upload_and_repack(L_bad)
+    assert e.value.status == B.GPTQ_ERR_GIDX
+    uneven = L.g_idx.copy()
+    uneven[np.argmax(uneven == 0)] = 1            # group 1 gets 129 rows
+    L_un = wl.QuantLinear(L.K, L.N, 128, L.qweight, L.qzeros, L.scales, uneven, 0)
+    with pytest.raises(B.GptqError) as e:
+        H.upload_and_repack(L_un)
+    assert e.value.status == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_check_status() == B.GPTQ_OK     # the flag was cleared
+    H.upload_and_repack(L)                        # and a valid layer still works
+
+
+# ------------------------------------------------------------------------------- matmul, small
+SMALL = [
+    (128, 128, 1, False), (256, 128, 1, False), (1024, 384, 3, False), (512, 256, 8, False),
+    (2048, 640, 9, False), (768, 128, 16, False), (1280, 1152, 17, False), (640, 384, 33, False),
+    (512, 256, 64, False), (384, 256, 65, False), (256, 384, 130, False),
+    (256, 128, 1, True), (1024, 640, 5, True), (2560, 256, 8, True), (512, 384, 40, True),
+]
+
+
+@pytest.mark.parametrize("K,N,M,act", SMALL)
+def test_gemm_small_full_compare(K, N, M, act, ws):
+    L = wl.make_linear(K, N, seed=wl.seed_for("small", K, N, M, act), act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("small-x", K, M))
+    y, _ = run_gemm(L, x, ws)
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+
+
+@pytest.mark.parametrize("M", [1, 7, 16, 24, 64])
+def test_gemm_integer_case_is_exact(M, ws):
+    """z = 8, s = 1, small-integer x: every product and partial sum is an integer below 2^24, so
+    any summation order gives the exact result, and it is exact in fp16 wherever |y| <= 2048."""
+    K, N = 1024, 256
+    r = np.random.default_rng(77)
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    L = wl.make_linear_from_values(q, np.full((K // 128, N), 8, np.uint8), np.ones((K // 128, N), np.float16), 128)
+    x = r.integers(-4, 5, (M, K)).astype(np.float16)
+    y, _ = run_gemm(L, x, ws)
+    want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128)
+    small = np.abs(want) <= 2048
+    assert small.mean() > 0.9
+    assert np.array_equal(y.astype(np.float64)[small], want[small])
+    assert_close(y, want, K)
+
+
+def test_gemm_power_of_two_scales_tight(ws):
+    K, N, M = 2048, 384, 4
+    L0 = wl.make_linear(K, N, seed=91)
+    r = np.random.default_rng(92)
+    s = (2.0 ** r.integers(-9, -5, (K // 128, N))).astype(np.float16)
+    L = wl.QuantLinear(K, N, 128, L0.qweight, L0.qzeros, s, None, 0)
+    x = wl.make_x(M, K, 93)
+    y, _ = run_gemm(L, x, ws)
+    want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128)
+    err = np.abs(y.astype(np.float64) - want)
+    assert np.all(err <= 2.0 ** -11 * np.abs(want) + 2e-5)
+
+
+def test_gemm_one_hot_rows_return_rounded_weights(ws):
+    K, N = 512, 256
+    L = wl.make_linear(K, N, seed=101, act_order=True)
+    ks = [0, 1, 9, 127, 128, 300, 511]
+    x = np.zeros((len(ks), K), dtype=np.float16)
+    for i, k in enumerate(ks):
+        x[i, k] = 1.0
+    y, _ = run_gemm(L, x, ws)
+    w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert np.array_equal(y, w[ks].astype(np.float16))
+
+
+def test_gemm_is_deterministic_and_leaves_neighbours_alone(ws):
+    K, N, M = 4096, 4096, 5
+    L = wl.make_linear(K, N, seed=111)
+    D = H.upload_and_repack(L)
+    ws.ensure_for(M, D)
+    x = H.to_device(wl.make_x(M, K, 112))
+    guard = torch.full((M + 2, N), 7.0, dtype=torch.float16, device="cuda")
+    y = guard[1:M + 1]
+    H.gemm(x, D, y)
+    first = y.clone()
+    for _ in range(3):
+        H.gemm(x, D, y)
+        assert torch.equal(first, y)
+    assert torch.all(guard[0] == 7.0) and torch.all(guard[M + 1] == 7.0)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+def test_gemm_without_workspace_is_refused_not_wrong():
+    K, N = 4096, 4096                       # split panels on any GPU with more than 32 SMs
+    L = wl.make_linear(K, N, seed=121)
+    D = H.upload_and_repack(L)
+    need = B.gptq_workspace_bytes(1, N, K, 128, 0)
+    assert need > 0
+    B.check(B.gptq_set_workspace(None, 0), "unset")
+    x = H.to_device(wl.make_x(1, K, 122))
+    y = torch.zeros((1, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 1, N, K, 128, 0) == B.GPTQ_ERR_WORKSPACE
+    small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
+    B.check(B.gptq_set_workspace(small, small.numel()), "small ws")
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 1, N, K, 128, 0) == B.GPTQ_ERR_WORKSPACE
+    B.check(B.gptq_set_workspace(None, 0), "unset")
+    assert torch.count_nonzero(y) == 0
+
+
+def test_gemm_host_round_trip(ws):
+    K, N, M = 4096, 4096, 8
+    L = wl.make_linear(K, N, seed=131)
+    D = H.upload_and_repack(L)
+    ws.buf = None
+    ws.ensure_for(M, D)
+    x_np = wl.make_x(M, K, 132)
+    x_host = torch.from_numpy(x_np).pin_memory()
+    y_host = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    xs = torch.empty((M, K), dtype=torch.float16, device="cuda")
+    ys = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    B.check(B.gptq_gemm_host(x_host, D.qweight_t, D.qzeros_t, D.scales_t, None, y_host, xs, ys, M, N, K, 128, 0),
+            "gemm_host")
+    torch.cuda.synchronize()
+    assert_close(y_host.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, None, 128), K)
+
+
+# ------------------------------------------------------------------------------- matmul, full size
+def sampled_check(L, x, y, n_samples, seed):
+    r = np.random.default_rng(seed)
+    M = x.shape[0]
+    rows = r.integers(0, M, n_samples).astype(np.int32)
+    cols = r.integers(0, L.N, n_samples).astype(np.int32)
+    # always include the corners and the last panel's last column
+    rows[:4] = [0, 0, M - 1, M - 1]
+    cols[:4] = [0, L.N - 1, 0, L.N - 1]
+    want = oracle.gemm_f64_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128, rows, cols)
+    assert_close(y[rows, cols], want, L.K)
+
+
+def test_config1_full_compare(ws):
+    K, N = 4096, 4096
+    L = wl.make_linear(K, N, seed=wl.seed_for("config1"))
+    x = wl.make_x(1, K, wl.seed_for("config1-x"))
+    y, _ = run_gemm(L, x, ws)
+    want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128)
+    assert_close(y, want, K)
+    # the spread of y matches the closed form for these input distributions
+    es2 = wl.SCALE_FLOOR ** 2 + 2 * wl.SCALE_FLOOR * wl.SCALE_SIGMA * math.sqrt(2 / math.pi) + wl.SCALE_SIGMA ** 2
+    assert abs(y.astype(np.float64).std() / math.sqrt(K * 42.5 * es2) - 1) < 0.05
+
+
+@pytest.mark.parametrize("name", list(wl.SHAPES_7B))
+def test_config2_llama7b_decode(name, ws):
+    K, N = wl.SHAPES_7B[name]
+    L = wl.make_linear(K, N, seed=wl.seed_for("config2", name))
+    D = H.upload_and_repack(L)
+    for M in wl.DECODE_M:
+        x = wl.make_x(M, K, wl.seed_for("config2-x", name, M))
+        ws.ensure_for(M, D)
+        y = H.gemm(H.to_device(x), D).cpu().numpy()
+        sampled_check(L, x, y, 3000, seed=M)
+        if M == 1 and name in ("o", "down"):
+            assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128), K)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+@pytest.mark.parametrize("name", list(wl.SHAPES_13B))
+def test_config3_act_order(name, ws):
+    K, N = wl.SHAPES_13B[name]
+    L = wl.make_linear(K, N, seed=wl.seed_for("config3", name), act_order=True)
+    D = H.upload_and_repack(L)
+    for M in wl.ACT_ORDER_M:
+        x = wl.make_x(M, K, wl.seed_for("config3-x", name, M))
+        ws.ensure_for(M, D)
+        y = H.gemm(H.to_device(x), D).cpu().numpy()
+        sampled_check(L, x, y, 3000, seed=M)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+@pytest.mark.parametrize("name,M,act", [("o", 512, False), ("qkv", 1024, False), ("down", 2048, True),
+                                        ("gate_up", 4096, False), ("o", 4096, True)])
+def test_config4_prefill_sampled(name, M, act, ws):
+    K, N = wl.SHAPES_7B[name]
+    L = wl.make_linear(K, N, seed=wl.seed_for("config4", name, act), act_order=act)
+    D = H.upload_and_repack(L)
+    x = wl.make_x(M, K, wl.seed_for("config4-x", name, M))
+    ws.ensure_for(M, D)
+    y = H.gemm(H.to_device(x), D).cpu().numpy()
+    sampled_check(L, x, y, 4000, seed=M)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+@pytest.mark.parametrize("M", wl.STEP_M)
+def test_config5_decode_step_layers(M, ws):
+    """Layers 0 and 31 of the 32-layer step (distinct seeded weights per layer)."""
+    for layer in (0, 31):
+        for name, (K, N) in wl.SHAPES_7B.items():
+            L = wl.make_linear(K, N, seed=wl.seed_for("config5", layer, name))
+            D = H.upload_and_repack(L)
+            x = wl.make_x(M, K, wl.seed_for("config5-x", layer, name, M))
+            ws.ensure_for(M, D)
+            y = H.gemm(H.to_device(x), D).cpu().numpy()
+            sampled_check(L, x, y, 1500, seed=layer * 100 + M)
+    assert B.gptq_check_status() == B.GPTQ_OK
