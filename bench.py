@@ -1,0 +1,506 @@
+#!/usr/bin/env python
+"""Benchmark of the GPTQ int4 matmul path on B200.
+
+A STEP is one pass of the whole path (stage x, stream packed weights, unpack, dequantise,
+multiply-accumulate, reduce, store fp16 y) over every matmul of the workload:
+
+  decode7b  (default)  the four Llama-2-7B decoder linears (qkv, o, gate_up, down), group 128,
+                       at M = 1, 4, 8, 16, over `--layers` distinct seeded copies of the layer so
+                       that each launch streams weights last touched ~0.8 GB ago (HBM-cold)
+  step32               32 layers x 4 linears at M = 1, 8, 32, 64 (a full decode step's linears)
+  actorder13b          Llama-2-13B shapes with act-order g_idx at M = 1, 8
+  prefill7b            the 7B shapes at M = 512 .. 4096 (metric becomes TFLOP/s)
+
+Every matmul is a gptq_gemm call through the C ABI.  The device-timed number replays CUDA graphs
+of those calls (one graph per M) with CUDA events around them; the end-to-end number calls
+gptq_gemm_host with pinned host activations and outputs, copies inside the timed region.
+One JSON line is printed by rank 0.  With --impl reference the CPU oracle is timed instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_19438_b200 import workloads as wl  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_FP16_TFLOPS = 2250.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_TFLOPS = 1590.0
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture, keyed by kernel name, with
+# the digest of the kernel sources they were taken on; reported as null once the sources change.
+NCU_TRAFFIC = {}
+
+WORKLOADS = {
+    "decode7b": dict(shapes=wl.SHAPES_7B, Ms=wl.DECODE_M, act_order=False, layers=8, kind="decode",
+                     describes="configs[1]: Llama-2-7B decoder linears, group 128, M in {1,4,8,16}"),
+    "step32": dict(shapes=wl.SHAPES_7B, Ms=wl.STEP_M, act_order=False, layers=32, kind="decode",
+                   describes="configs[4]: 32-layer Llama-2-7B decode step linears, M in {1,8,32,64}"),
+    "actorder13b": dict(shapes=wl.SHAPES_13B, Ms=wl.ACT_ORDER_M, act_order=True, layers=4, kind="decode",
+                        describes="configs[2]: Llama-2-13B shapes with act-order g_idx, M in {1,8}"),
+    "prefill7b": dict(shapes=wl.SHAPES_7B, Ms=wl.PREFILL_M, act_order=False, layers=2, kind="prefill",
+                      describes="configs[3]: Llama-2-7B shapes, M in {512,1024,2048,4096}"),
+}
+
+
+def kernel_source_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2511_19438_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), tflops_burst=float(p["bf16_tflops"]),
+                    tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, tflops_burst=FALLBACK_TFLOPS, tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) in a thread."""
+
+    REASONS = {
+        0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+        0x80: "hw_power_brake_slowdown",
+    }
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples = []
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self.max_mhz = None
+        self.error = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                tok = ids[index] if index < len(ids) else ids[0]
+                self.h = (pynvml.nvmlDeviceGetHandleByUUID(tok) if tok.startswith("GPU-")
+                          else pynvml.nvmlDeviceGetHandleByIndex(int(tok)))
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # no NVML: the clocks object says so
+            self.nv = None
+            self.error = repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception as e:
+                self.error = repr(e)
+                return
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float, note: str = ""):
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": len(inside)}
+        if inside:
+            out["sm_mhz"] = statistics.median(s[1] for s in inside)
+            mask = 0
+            for s in inside:
+                mask |= s[2]
+            out["reasons"] = sorted(name for bit, name in self.REASONS.items() if mask & bit)
+        if note:
+            out["note"] = note
+        if self.error:
+            out["error"] = self.error
+        return out
+
+
+# ------------------------------------------------------------------------------------ workload
+def build_problems(spec, layers, H, torch, device):
+    """Uploads `layers` distinct seeded copies of every shape (repacked through the C ABI) and the
+    activations; returns {M: [(D, x, y, name), ...]} in launch order (layer-major)."""
+    Ms = spec["Ms"]
+    per_m = {M: [] for M in Ms}
+    host = {}
+    for layer in range(layers):
+        for name, (K, N) in spec["shapes"].items():
+            L = wl.make_linear(K, N, seed=wl.seed_for("bench", layer, name), act_order=spec["act_order"])
+            D = H.upload_and_repack(L)
+            if layer == 0:
+                host[name] = L
+            for M in Ms:
+                if layer == 0:
+                    x = H.to_device(wl.make_x(M, K, wl.seed_for("bench-x", name, M)), device)
+                else:   # activations are tiny next to the weights: reuse layer 0's
+                    x = per_m[M][list(spec["shapes"]).index(name)][1]
+                if spec["kind"] == "prefill" and layer > 0:
+                    y = per_m[M][list(spec["shapes"]).index(name)][2]
+                else:
+                    y = torch.empty((M, N), dtype=torch.float16, device=device)
+                per_m[M].append((D, x, y, name))
+    return per_m, host
+
+
+def step_bytes_flops(spec, layers):
+    b = {M: 0 for M in spec["Ms"]}
+    f = {M: 0 for M in spec["Ms"]}
+    for M in spec["Ms"]:
+        for (K, N) in spec["shapes"].values():
+            b[M] += layers * wl.algorithmic_bytes(M, K, N, act_order=spec["act_order"])
+            f[M] += layers * wl.matmul_flops(M, K, N)
+    return b, f
+
+
+def launches_per_gemm(spec, M):
+    """Kernels one gptq_gemm call launches: one per 64-token chunk, plus the x gather with act-order."""
+    return (M + 63) // 64 + (1 if spec["act_order"] else 0)
+
+
+# ------------------------------------------------------------------------------------ reference arm
+def oracle_sample(spec, budget_s):
+    """The bounded sample of the workload the CPU oracle is timed on: layer 0 of the workload, the
+    largest of a fixed ladder of (shapes, M) subsets whose estimated time fits `budget_s` (the
+    estimate comes from a probe of the smallest shape at the smallest M)."""
+    import oracle
+    shapes = spec["shapes"]
+    small = min(shapes, key=lambda n: shapes[n][0] * shapes[n][1])
+    Ms = [M for M in spec["Ms"] if M <= 16] or [16]
+    ladder = [([small], Ms[:1]), (list(shapes), Ms[:1]), (list(shapes), Ms[:2]), (list(shapes), Ms)]
+    layer = {n: wl.make_linear(K, N, seed=wl.seed_for("bench", 0, n), act_order=spec["act_order"])
+             for n, (K, N) in shapes.items()}
+    Lp = layer[small]
+    xp = wl.make_x(Ms[0], Lp.K, wl.seed_for("bench-x", small, Ms[0]))
+    oracle.gemm_f64(xp, Lp.qweight, Lp.qzeros, Lp.scales, Lp.g_idx, Lp.group_size)   # first touch
+    t0 = time.perf_counter()
+    oracle.gemm_f64(xp, Lp.qweight, Lp.qzeros, Lp.scales, Lp.g_idx, Lp.group_size)
+    rate = Ms[0] * Lp.K * Lp.N / (time.perf_counter() - t0)
+    pick = ladder[0]
+    for names, ms in ladder:
+        macs = sum(M * shapes[n][0] * shapes[n][1] for n in names for M in ms)
+        if macs / rate <= budget_s:
+            pick = (names, ms)
+    names, ms = pick
+    items = [(layer[n], wl.make_x(M, layer[n].K, wl.seed_for("bench-x", n, M)), M) for n in names for M in ms]
+    text = f"layer 0 of the workload, shapes {names}, M in {list(ms)}, full outputs"
+    return items, text
+
+
+def run_oracle_once(items, spec):
+    import oracle
+    t0 = time.perf_counter()
+    for (L, x, M) in items:
+        oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
+    dt = time.perf_counter() - t0
+    nbytes = sum(wl.algorithmic_bytes(M, L.K, L.N, act_order=L.act_order) for (L, x, M) in items)
+    flops = sum(wl.matmul_flops(M, L.K, L.N) for (L, x, M) in items)
+    return dt, nbytes, flops
+
+
+def metric_of(spec):
+    if spec["kind"] == "prefill":
+        return "GPTQ int4 matmul: prefill TFLOPS (% fp16 peak)", "TFLOP/s"
+    return "GPTQ int4 matmul: decode HBM GB/s (% of 8 TB/s)", "GB/s"
+
+
+def to_metric(spec, nbytes, flops, seconds):
+    return (flops / seconds / 1e12) if spec["kind"] == "prefill" else (nbytes / seconds / 1e9)
+
+
+def cpu_baseline(spec):
+    import oracle
+    oracle.build()
+    items, text = oracle_sample(spec, budget_s=12.0)
+    dt, nbytes, flops = run_oracle_once(items, spec)
+    return {"value": to_metric(spec, nbytes, flops, dt), "unit": metric_of(spec)[1], "cores": oracle.num_threads(),
+            "kind": "oracle", "sample": text, "seconds": round(dt, 3)}
+
+
+def run_reference(args, spec):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    items, text = oracle_sample(spec, budget_s=min(12.0, 150.0 / max(args.steps + min(args.warmup, 1), 1)))
+    for _ in range(min(args.warmup, 1)):
+        run_oracle_once(items, spec)
+    total = 0.0
+    for _ in range(args.steps):
+        dt, nbytes, flops = run_oracle_once(items, spec)
+        total += dt
+    value = to_metric(spec, nbytes * args.steps, flops * args.steps, total)
+    metric, unit = metric_of(spec)
+    line = {
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "describes": spec["describes"], "sample": text},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": text},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ product arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode7b", choices=list(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="distinct weight copies per shape (0 = workload default)")
+    ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    spec = WORKLOADS[args.workload]
+    layers = args.layers or spec["layers"]
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GPTQ matmul has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2511_19438_b200 import build as libbuild
+    if local_rank == 0:
+        libbuild.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2511_19438_b200 import binding as B
+    from paper_2511_19438_b200 import harness as H
+
+    per_m, _host = build_problems(spec, layers, H, torch, device)
+    ws = H.WorkspaceHolder(device)
+    need = 0
+    for M, probs in per_m.items():
+        for (D, x, y, _n) in probs:
+            need = max(need, B.gptq_workspace_bytes(M, D.N, D.K, D.group_size, D.act_order))
+    ws.ensure(need)
+    bytes_m, flops_m = step_bytes_flops(spec, layers)
+
+    def run_m(M):
+        for (D, x, y, _n) in per_m[M]:
+            H.gemm(x, D, y)
+
+    # eager warm-up (configures the kernels), then one CUDA graph per M
+    stream = torch.cuda.Stream(device)
+    graphs = {}
+    with torch.cuda.stream(stream):
+        for M in spec["Ms"]:
+            run_m(M)
+        stream.synchronize()
+        B.check(B.gptq_check_status(), "warm-up")
+        for M in spec["Ms"]:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                run_m(M)
+            graphs[M] = g
+    torch.cuda.synchronize()
+
+    Ms = list(spec["Ms"])
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            for M in Ms:
+                graphs[M].replay()
+        barrier()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(Ms) + 1)] for _ in range(args.steps)]
+        t_host0 = time.perf_counter()
+        for k in range(args.steps):
+            ev[k][0].record(stream)
+            for i, M in enumerate(Ms):
+                graphs[M].replay()
+                ev[k][i + 1].record(stream)
+        barrier()
+        t_host1 = time.perf_counter()
+    total_ms = ev[0][0].elapsed_time(ev[-1][-1])
+    seg_ms = {M: sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)) for i, M in enumerate(Ms)}
+    clocks = sampler.summary(t_host0, t_host1)
+    if clocks["samples"] < 3:
+        # the timed region was too short to catch a sample: keep replaying the same step, untimed
+        t2 = time.perf_counter()
+        with torch.cuda.stream(stream):
+            while time.perf_counter() - t2 < 1.0:
+                for M in Ms:
+                    graphs[M].replay()
+                stream.synchronize()
+        clocks = sampler.summary(t2, time.perf_counter(),
+                                 note="timed region shorter than the sampling period; sampled over 1 s of the same steps right after it")
+    B.check(B.gptq_check_status(), "timed region")
+
+    # ---- end to end: host activations in, host outputs back, every call through gptq_gemm_host
+    e2e_steps = args.e2e_steps or min(args.steps, 20)
+    host_io = {}
+    h2d = d2h = 0
+    for M in Ms:
+        for (D, x, y, name) in per_m[M][:len(spec["shapes"])]:
+            xh = x.cpu().pin_memory()
+            yh = torch.empty((M, D.N), dtype=torch.float16).pin_memory()
+            host_io[(M, name)] = (xh, yh)
+    for M in Ms:
+        for (D, x, y, name) in per_m[M]:
+            h2d += M * D.K * 2
+            d2h += M * D.N * 2
+
+    def e2e_step():
+        for M in Ms:
+            for (D, x, y, name) in per_m[M]:
+                xh, yh = host_io[(M, name)]
+                B.check(B.gptq_gemm_host(xh, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, yh, x, y, M, D.N, D.K,
+                                         D.group_size, D.act_order), "gptq_gemm_host")
+        stream.synchronize()   # the step's results are on the host
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    sampler.stop()
+
+    # ---- reduce over ranks (max time), aggregate over replicas
+    times = torch.tensor([total_ms, e2e_ms] + [seg_ms[M] for M in Ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    times = times.tolist()
+    total_ms, e2e_ms = times[0], times[1]
+    seg_ms = {M: times[2 + i] for i, M in enumerate(Ms)}
+
+    if rank == 0:
+        peaks = measured_peaks()
+        metric, unit = metric_of(spec)
+        step_bytes, step_flops = sum(bytes_m.values()), sum(flops_m.values())
+        sec = total_ms / 1e3
+        value = world * to_metric(spec, step_bytes * args.steps, step_flops * args.steps, sec)
+        e2e_value = world * to_metric(spec, step_bytes * e2e_steps, step_flops * e2e_steps, e2e_ms / 1e3)
+        launches_step = sum(launches_per_gemm(spec, M) * len(per_m[M]) for M in Ms)
+        per_m_report = {}
+        for M in Ms:
+            s = seg_ms[M] / 1e3
+            per_m_report[str(M)] = {
+                "GB/s": round(bytes_m[M] * args.steps / s / 1e9, 1),
+                "TFLOP/s": round(flops_m[M] * args.steps / s / 1e12, 2),
+                "us_per_matmul": round(1e6 * s / args.steps / len(per_m[M]), 3),
+            }
+        # dominant kernel: the streaming kernel instantiation that took most of the timed region
+        if spec["kind"] == "prefill":
+            dom_Ms = Ms
+            kname = "streamk_kernel<8>"
+        else:
+            groups = {}
+            for M in Ms:
+                tile = 8 if M <= 8 else 16 if M <= 16 else 32 if M <= 32 else 64
+                groups.setdefault(tile, []).append(M)
+            tile = max(groups, key=lambda t: sum(seg_ms[M] for M in groups[t]))
+            dom_Ms = groups[tile]
+            kname = f"streamk_kernel<{tile // 8}>"
+        dom_s = sum(seg_ms[M] for M in dom_Ms) / 1e3
+        dom_launches = sum(((M + 63) // 64) * len(per_m[M]) for M in dom_Ms) * args.steps
+        if spec["kind"] == "prefill":
+            achieved = sum(flops_m[M] for M in dom_Ms) * args.steps / dom_s / 1e12
+            peak, bound, runit = peaks["tflops_sustained"], "tensor", "TFLOP/s"
+        else:
+            achieved = sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_s / 1e9
+            peak, bound, runit = peaks["hbm_gbs"], "hbm", "GB/s"
+        digest = kernel_source_digest()
+        traffic = None
+        t = NCU_TRAFFIC.get(kname)
+        if t and t.get("digest") == digest:
+            traffic = t["bytes_per_launch"]
+        roofline = {
+            "bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": runit,
+            "frac": round(achieved / peak, 4), "traffic": traffic, "kernel": kname, "peak_source": peaks["source"],
+            "avg_launch_us": round(1e6 * dom_s / dom_launches, 3),
+            "alg_bytes_per_launch": round(sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_launches),
+            "launches_timed": dom_launches, "M_covered": dom_Ms,
+            "frac_of_nominal": round(achieved / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 4),
+        }
+        line = {
+            "metric": metric, "value": round(value, 2), "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+            "config": {"workload": args.workload, "describes": spec["describes"], "layers": layers,
+                       "matmuls_per_step": sum(len(per_m[M]) for M in Ms), "group_size": 128,
+                       "act_order": spec["act_order"], "parallelism": f"{world} independent replica(s)",
+                       "l2": f"inputs larger than L2: each M pass streams {round(bytes_m[Ms[0]] / 1e6)} MB of distinct weights",
+                       "timing": "CUDA events around CUDA-graph replays of the gptq_gemm calls, one graph per M"},
+            "clocks": clocks,
+            "e2e": {"value": round(e2e_value, 2), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
+                    "api": "gptq_gemm_host per matmul, pinned host x and y"},
+            "gpu_launches": launches_step * args.steps,
+            "per_M": per_m_report,
+            "roofline": roofline,
+            "pct_of_nominal": round(100 * value / world / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 2),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(spec)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
