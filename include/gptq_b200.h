@@ -116,6 +116,30 @@ int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, 
                    const int32_t *g_idx, void *y_host, void *x_stage, void *y_stage,
                    int M, int N, int K, int group_size, int act_order, void *stream);
 
+/* (No counterpart in the paper: a packaging variant of gptq_gemm.)
+ * The same product as gptq_gemm for callers that cannot hand the library a workspace because
+ * they cannot allocate device memory at all: code hosted inside a serving process whose device
+ * memory was partitioned at start-up and where a later cudaMalloc is forbidden or would stall
+ * the whole device (cudaMalloc/cudaFree synchronise it), such as a decode loop with a latency
+ * budget.  The split-K partial tiles, their tickets and (act-order) the gathered activations
+ * live in an 8 MiB array that is part of the library image: every GPU that loads the library
+ * holds it until the process exits.  Arguments, layouts and arithmetic are those of gptq_gemm.
+ *  - Problems whose scratch need (gptq_workspace_bytes) exceeds gptq_noalloc_scratch_bytes()
+ *    are refused with GPTQ_ERR_WORKSPACE; nothing is launched.  (All decode shapes of the 7B
+ *    and 13B layers fit up to M = 16.)
+ *  - The call allocates and frees nothing, on the device or through any library.
+ *  - The first call on each device looks up the array's device address (the device must be
+ *    current, as for every call); make that first call before any stream capture begins.
+ *  - All calls share the one array, which keeps the previous call's contents; each call clears
+ *    the tickets it needs on `stream` first.  Calls that can overlap on the GPU (different
+ *    streams, several host threads) race on it: serialise them, or use gptq_gemm with
+ *    per-stream workspaces. */
+int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                      const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
+                      void *stream);
+/* Size in bytes of the built-in scratch array (host-only, no CUDA call). */
+size_t gptq_noalloc_scratch_bytes(void);
+
 /* Synchronises `stream` and returns GPTQ_ERR_TIMEOUT if any kernel's bounded wait gave up
  * since the last check (the flag is then cleared), GPTQ_ERR_CUDA on a runtime error, else OK. */
 int gptq_check_status(void *stream);

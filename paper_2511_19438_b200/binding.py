@@ -54,6 +54,8 @@ _SIGNATURES = {
     "gptq_set_workspace": (_i, [_vp, _sz, _vp]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_noalloc_scratch_bytes": (_sz, []),
     "gptq_check_status": (_i, [_vp]),
     "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_cta_range": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
@@ -146,6 +148,15 @@ def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_st
     return _lib.gptq_gemm_host(_ptr(x_host), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx),
                                _ptr(y_host), _ptr(x_stage), _ptr(y_stage), M, N, K, group_size,
                                int(act_order), _stream(stream))
+
+
+def gptq_gemm_noalloc(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
+    return _lib.gptq_gemm_noalloc(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N,
+                                  K, group_size, int(act_order), _stream(stream))
+
+
+def gptq_noalloc_scratch_bytes() -> int:
+    return _lib.gptq_noalloc_scratch_bytes()
 
 
 def gptq_check_status(stream=None) -> int:

@@ -285,6 +285,77 @@ int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, 
     return record_cuda_error(cudaMemcpyAsync(y_host, y_stage, (size_t)M * N * sizeof(__half), cudaMemcpyDeviceToHost, s));
 }
 
+// ---- matmul with built-in scratch -----------------------------------------------------------
+// Scratch for gptq_gemm_noalloc: lives in the library's device image, so every GPU that loads
+// the library holds these 8 MiB until the process exits.  Layout = the registered workspace's:
+// [tickets 16 KB][fp32 partial tiles][gathered x (act-order)].
+constexpr size_t kStaticScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+// In host code `g_static_scratch` is only a handle for the runtime, never a device address; the
+// address a kernel can use is looked up once per device and cached here.
+static void *g_static_scratch_addr[kMaxDevices];
+
+static int static_scratch_address(int dev, void **out)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);   // device `dev` is current
+        if (e != cudaSuccess) return record_cuda_error(e);
+        if (p == nullptr) return GPTQ_ERR_CUDA;
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return GPTQ_OK;
+}
+
+size_t gptq_noalloc_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                      const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
+                      void *stream)
+{
+    if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
+        return GPTQ_ERR_ALIGN;
+    st = check_fast_path(N, K, group_size);
+    if (st) return st;
+    int dev, sms;
+    st = current_device_sms(&dev, &sms);
+    if (st) return st;
+    const GemmPlan gp = make_plan(M, N, K, act_order, sms);
+    // the built-in scratch has a fixed size: larger problems must use gptq_gemm with a workspace
+    if (gp.workspace_bytes > kStaticScratchBytes) return GPTQ_ERR_WORKSPACE;
+    void *base = nullptr;
+    st = static_scratch_address(dev, &base);
+    if (st) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t *wsb = (uint8_t *)base;
+    int *tickets = (int *)wsb;
+    float *partials = (float *)(wsb + kTicketAreaBytes);
+    // the array keeps whatever the previous call left; the tickets are the only part that must be zero
+    st = record_cuda_error(cudaMemsetAsync(tickets, 0, (size_t)(N / kPanel) * sizeof(int), s));
+    if (st) return st;
+    const __half *xin = (const __half *)x;
+    if (act_order) {
+        __half *x_perm = (__half *)(wsb + kTicketAreaBytes + gp.sk.partial_bytes);
+        st = launch_gather_x((const __half *)x, g_idx, x_perm, M, K, s);
+        if (st) return st;
+        xin = x_perm;
+    }
+    for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
+        const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
+        const StreamKPlan pl = plan_streamk(rows, N, K, sms);
+        st = launch_streamk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
+                            pl, partials, tickets, s);
+        if (st) return st;
+    }
+    return GPTQ_OK;
+}
+
 int gptq_check_status(void *stream)
 {
     cudaStream_t s = (cudaStream_t)stream;
