@@ -16,18 +16,21 @@
 // tiles in CTA order (a fixed order, so results are reproducible) and writes fp16 y once.
 #pragma once
 #include "gptq_common.cuh"
+#include "gptq_tma.cuh"
 
 namespace gptq {
 
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamKThreads = kConsumerThreads + 32;
-constexpr int kXRowBytes = 320;   // 256 B of x + 64 B pad: conflict-free 128-bit fragment loads
-constexpr int kBarrierBytes = 128;
+constexpr int kRingOffset = 1024;   // barriers live below the ring; the ring is 1024-byte aligned
 
+// A ring stage: [x: two K64 tiles of MT*8 token rows x 128 B, 128-byte swizzled by the tensor-map load]
+//               [8192 B packed weights][256 B scales][64 B zeros], rounded up to 1024 B.
+__host__ __device__ constexpr int streamk_x_bytes(int MT) { return MT * 2048; }
 __host__ __device__ constexpr int streamk_stage_bytes(int MT)
 {
-    return kItemWBytes + kItemSBytes + kItemZBytes + MT * 8 * kXRowBytes;
+    return (streamk_x_bytes(MT) + kItemWBytes + kItemSBytes + kItemZBytes + 1023) & ~1023;
 }
 
 // Stream-K index arithmetic (shared by the kernel, the planner and the host-side introspection
@@ -36,8 +39,12 @@ __host__ __device__ inline int sk_range_begin(long long T, int C, int c) { retur
 // the CTA whose range contains item t
 __host__ __device__ inline int sk_owner(long long T, int C, long long t) { return (int)(((t + 1) * C - 1) / T); }
 
+// MMA token slot n (0..7) -> token row inside an 8-row tile: bit reversal.  With this choice the
+// eight lanes of a quarter warp (two token slots x four k chunks) read eight different 16-byte
+// chunks of the swizzled x tile, so the 128-bit fragment loads are bank-conflict free.
+__host__ __device__ constexpr int token_row_of_slot(int n) { return ((n & 1) << 2) | (n & 2) | ((n >> 2) & 1); }
+
 struct StreamKArgs {
-    const __half *x;        // [M, K] (already in sorted row order for act-order layers)
     const uint8_t *qweight; // tiled
     const uint8_t *scales;
     const uint8_t *qzeros;
@@ -50,21 +57,24 @@ struct StreamKArgs {
 };
 
 template <int MT>
-__global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const StreamKArgs a)
+__global__ void __launch_bounds__(kStreamKThreads, MT <= 2 ? 2 : 1)
+streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
 {
-    extern __shared__ __align__(128) uint8_t smem_raw[];
+    extern __shared__ uint8_t smem_raw[];
     constexpr int kStage = streamk_stage_bytes(MT);
-    constexpr int kOffS = kItemWBytes, kOffZ = kOffS + kItemSBytes, kOffX = kOffZ + kItemZBytes;
+    constexpr int kXTile = MT * 1024;                       // one K64 tile of x
+    constexpr int kOffW = streamk_x_bytes(MT), kOffS = kOffW + kItemWBytes, kOffZ = kOffS + kItemSBytes;
 
-    const uint32_t smem_base = smem_u32(smem_raw);
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_base;                  // stages x 8 B
     const uint32_t bar_empty = smem_base + 64;            // stages x 8 B
-    const uint32_t ring = smem_base + kBarrierBytes;
+    const uint32_t ring = smem_base + kRingOffset;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int C = gridDim.x, c = blockIdx.x;
     const long long T = a.items;
     const int t0 = sk_range_begin(T, C, c), t1 = sk_range_begin(T, C, c + 1);
     const int stages = a.stages;
+    __shared__ int s_last;
 
     if (threadIdx.x == kConsumerThreads) {
         for (int s = 0; s < stages; ++s) {
@@ -74,57 +84,41 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
         fence_barrier_init();
         fence_proxy_async();
     }
-    // token rows beyond M stay zero for the whole kernel (the bulk copies never touch them)
-    {
-        const int zero_rows = MT * 8 - a.M;   // rows a.M .. MT*8-1 of every stage
-        const int vec_per_row = kXRowBytes / 16;
-        for (int i = threadIdx.x; i < stages * zero_rows * vec_per_row; i += kStreamKThreads) {
-            int s = i / (zero_rows * vec_per_row), rem = i % (zero_rows * vec_per_row);
-            int row = a.M + rem / vec_per_row, v = rem % vec_per_row;
-            *reinterpret_cast<uint4 *>(smem_raw + kBarrierBytes + s * kStage + kOffX + row * kXRowBytes + v * 16) =
-                make_uint4(0, 0, 0, 0);
-        }
-    }
     __syncthreads();
     pdl_launch_dependents();
 
     if (warp == kConsumerWarps) {
-        // ------------------------------------------------------------------ producer warp
+        // ------------------------------------------------------------------ producer (one thread)
+        if (lane != 0) return;
         const uint64_t policy = l2_policy_evict_first();
+        tma_prefetch_descriptor(&x_map);
         const uint32_t meta_bytes = kItemWBytes + kItemSBytes + kItemZBytes;
         const int n_items = t1 - t0;
         const int n_pre = n_items < stages ? n_items : stages;
         auto issue_weights = [&](int t, int s) {
-            uint32_t dst = ring + s * kStage, bar = bar_full + 8 * s;
+            const uint32_t dst = ring + s * kStage, bar = bar_full + 8 * s;
             mbar_expect_tx(bar, meta_bytes);
-            bulk_g2s_hint(dst, a.qweight + (size_t)t * kItemWBytes, kItemWBytes, bar, policy);
+            bulk_g2s_hint(dst + kOffW, a.qweight + (size_t)t * kItemWBytes, kItemWBytes, bar, policy);
             bulk_g2s_hint(dst + kOffS, a.scales + (size_t)t * kItemSBytes, kItemSBytes, bar, policy);
             bulk_g2s_hint(dst + kOffZ, a.qzeros + (size_t)t * kItemZBytes, kItemZBytes, bar, policy);
         };
         // weights never depend on earlier work in the stream: fill the ring before waiting on it
-        if (lane == 0)
-            for (int i = 0; i < n_pre; ++i) issue_weights(t0 + i, i);
+        for (int i = 0; i < n_pre; ++i) issue_weights(t0 + i, i);
         pdl_wait();
-        int s = 0, round = 0;
-        bool ok = true;
-        for (int it = 0; it < n_items && ok; ++it) {
-            const int t = t0 + it;
+        int s = 0, round = 0, grp = t0 % a.G;
+        for (int it = 0; it < n_items; ++it) {
             const uint32_t bar = bar_full + 8 * s;
-            if (lane == 0) {
-                if (it >= stages) {
-                    ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1));
-                    if (ok) issue_weights(t, s);
-                }
-                if (ok) mbar_arrive_expect_tx(bar, (uint32_t)a.M * 256u);
+            if (it >= stages) {
+                if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
+                issue_weights(t0 + it, s);
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (ok) {
-                const int grp = t % a.G;
-                const uint32_t dst = ring + s * kStage + kOffX;
-                for (int m = lane; m < a.M; m += 32)
-                    bulk_g2s(dst + m * kXRowBytes, a.x + (size_t)m * a.K + (size_t)grp * kGroup, 256, bar);
-            }
+            // the group's activations for all token rows: two swizzled K64 tiles, rows >= M read as zero
+            mbar_arrive_expect_tx(bar, (uint32_t)streamk_x_bytes(MT));
+            const uint32_t dst = ring + s * kStage;
+            tma_load_2d(dst, &x_map, grp * kGroup, 0, bar);
+            tma_load_2d(dst + kXTile, &x_map, grp * kGroup + 64, 0, bar);
             if (++s == stages) { s = 0; ++round; }
+            if (++grp == a.G) grp = 0;
         }
         return;
     }
@@ -132,10 +126,13 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
     // -------------------------------------------------------------------- consumer warps
     pdl_wait();
     const int g = lane >> 2, t4 = lane & 3;
-    const uint32_t w_off = warp * kUnitBytes + lane * 16;
+    const int r = token_row_of_slot(g);
+    const uint32_t w_off = kOffW + warp * kUnitBytes + lane * 16;
     const uint32_t s_off = kOffS + (warp * 16 + 2 * g) * 2;
     const uint32_t z_off = kOffZ + warp * 8 + g;
-    const uint32_t x_off = kOffX + g * kXRowBytes + t4 * 16;
+    // x fragment of k chunk (4j + t4) for token slot g: row r of the swizzled tile
+    const uint32_t x_off0 = r * 128 + ((uint32_t)(t4 ^ r) << 4);          // j = 0
+    const uint32_t x_off1 = r * 128 + ((uint32_t)((4 + t4) ^ r) << 4);    // j = 1
     constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
 
     float acc[MT][4];
@@ -146,10 +143,9 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
 
     int s = 0;
     uint32_t phase = 0;
-    int p = t0 / a.G, grp = t0 % a.G;
+    int p = t0 / a.G, grp = t0 - p * a.G;
     int seg_first_grp = grp;
     const int first_panel = p;
-    __shared__ int s_last;
 
     bool ok = true;   // false after a wait gave up: keep taking part in barriers, skip the data
     for (int t = t0; t < t1; ++t) {
@@ -188,7 +184,7 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
                 const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
-                    const uint4 xb = lds128(st + x_off + mt * 8 * kXRowBytes + (blk * 64 + j * 32) * 2);
+                    const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
                     mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
                     mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
                 }
@@ -211,6 +207,8 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
         const bool seg_end = (grp == a.G - 1) || (t == t1 - 1);
         if (seg_end) {
             const int col = warp * 16 + g;
+            // accumulator i of tile mt: weight column col + 8*(i>>1), token slot 2*t4 + (i&1)
+            const int m_lo = token_row_of_slot(2 * t4), m_hi = token_row_of_slot(2 * t4 + 1);
             if (seg_first_grp == 0 && grp == a.G - 1) {
                 // this CTA saw the panel's whole K range: round once and store
                 __half *yp = a.y + (size_t)p * kPanel + col;
@@ -218,7 +216,7 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const int m = mt * 8 + 2 * t4 + (i & 1);
+                        const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                         if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
                     }
             } else {
@@ -228,7 +226,7 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const int m = mt * 8 + 2 * t4 + (i & 1);
+                        const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                         if (m < a.M) pp[(size_t)m * kPanel + 8 * (i >> 1)] = acc[mt][i];
                     }
                 __threadfence();
@@ -243,14 +241,27 @@ __global__ void __launch_bounds__(kStreamKThreads, 1) streamk_kernel(const Strea
                 named_bar_sync(1, kConsumerThreads);
                 if (s_last) {
                     __threadfence();
+                    // every contributor after the first starts inside this panel (slot 0); the first one
+                    // starts inside it only if its range begins exactly at the panel's first item
+                    const int slot_first = (sk_range_begin(T, C, c_first) >= first_item) ? 0 : 1;
+                    const int nc = c_last - c_first + 1;
+                    const size_t tile = (size_t)a.M * kPanel;
                     for (int idx = threadIdx.x; idx < a.M * kPanel; idx += kConsumerThreads) {
-                        const int m = idx / kPanel, cc_col = idx % kPanel;
+                        const float *src = a.partials + (size_t)c_first * 2 * tile + idx;
                         float sum = 0.f;
-                        for (int cc = c_first; cc <= c_last; ++cc) {
-                            const int cc_first_panel = sk_range_begin(T, C, cc) / a.G;
-                            const int cc_slot = (cc_first_panel == p) ? 0 : 1;
-                            sum += __ldcg(a.partials + ((size_t)(cc * 2 + cc_slot) * a.M + m) * kPanel + cc_col);
+                        // fixed summation order (CTA order), eight loads in flight at a time
+                        for (int c0 = 0; c0 < nc; c0 += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int ci = c0 + u;
+                                const int sl = (ci == 0) ? slot_first : 0;
+                                v[u] = (ci < nc) ? __ldcg(src + (size_t)(ci * 2 + sl) * tile) : 0.f;
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) sum += v[u];
                         }
+                        const int m = idx / kPanel, cc_col = idx % kPanel;
                         a.y[(size_t)m * a.N + (size_t)p * kPanel + cc_col] = __float2half_rn(sum);
                     }
                     if (threadIdx.x == 0) a.tickets[p] = 0;   // ready for the next launch
@@ -278,7 +289,7 @@ StreamKPlan plan_streamk(int m_rows, int N, int K, int sm_count)
     // MT <= 2 keeps two CTAs per SM (<= 113 registers per thread, ~110 KB of ring each); wider
     // token tiles need more registers, so they run one CTA per SM with a deeper ring.
     const int ctas_per_sm = MT <= 2 ? 2 : 1;
-    const int ring_budget = (ctas_per_sm == 2 ? 110 : 220) * 1024 - kBarrierBytes;
+    const int ring_budget = (ctas_per_sm == 2 ? 112 : 224) * 1024 - 2 * kRingOffset;
     int stages = ring_budget / stage;
     if (stages > 8) stages = 8;
     pl.m_tile = MT * 8;
@@ -286,7 +297,7 @@ StreamKPlan plan_streamk(int m_rows, int N, int K, int sm_count)
     pl.items = panels * G;
     const int max_ctas = sm_count * ctas_per_sm;
     pl.ctas = pl.items < max_ctas ? pl.items : max_ctas;
-    pl.smem_bytes = kBarrierBytes + stages * stage;
+    pl.smem_bytes = 2 * kRingOffset + stages * stage;   // barrier block + alignment slack + ring
     // panels that are not covered by a single CTA
     int split = 0;
     const long long T = pl.items, C = pl.ctas;
@@ -301,7 +312,8 @@ StreamKPlan plan_streamk(int m_rows, int N, int K, int sm_count)
 }
 
 template <int MT>
-static int launch_streamk_mt(const StreamKArgs &args, const StreamKPlan &plan, cudaStream_t s)
+static int launch_streamk_mt(const StreamKArgs &args, const CUtensorMap &x_map, const StreamKPlan &plan,
+                             cudaStream_t s)
 {
     static int configured_smem[64] = {};
     int dev = 0;
@@ -326,14 +338,13 @@ static int launch_streamk_mt(const StreamKArgs &args, const StreamKPlan &plan, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return record_cuda_error(cudaLaunchKernelEx(&cfg, streamk_kernel<MT>, args));
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, streamk_kernel<MT>, args, x_map));
 }
 
 int launch_streamk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
                    int M, int N, int K, const StreamKPlan &plan, float *partials, int *tickets, cudaStream_t s)
 {
     StreamKArgs args;
-    args.x = x;
     args.qweight = (const uint8_t *)qweight;
     args.scales = (const uint8_t *)scales;
     args.qzeros = (const uint8_t *)qzeros;
@@ -346,11 +357,16 @@ int launch_streamk(const __half *x, const void *qweight, const void *qzeros, con
     args.G = K / kGroup;
     args.items = plan.items;
     args.stages = plan.stages;
+    // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
+    CUtensorMap x_map;
+    int st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
+                                (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.m_tile, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st) return st;
     switch (plan.m_tile) {
-    case 8: return launch_streamk_mt<1>(args, plan, s);
-    case 16: return launch_streamk_mt<2>(args, plan, s);
-    case 32: return launch_streamk_mt<4>(args, plan, s);
-    case 64: return launch_streamk_mt<8>(args, plan, s);
+    case 8: return launch_streamk_mt<1>(args, x_map, plan, s);
+    case 16: return launch_streamk_mt<2>(args, x_map, plan, s);
+    case 32: return launch_streamk_mt<4>(args, x_map, plan, s);
+    case 64: return launch_streamk_mt<8>(args, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }
