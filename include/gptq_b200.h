@@ -89,12 +89,12 @@ int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scale
 
 /* ---- the matmul ---------------------------------------------------------------------- */
 
-/* Scratch the matmul may need for this problem (split-K partial tiles and tickets; with
- * act_order a gathered copy of x).  0 means none. */
+/* Scratch gptq_gemm needs for this problem: with act_order a gathered copy of x (M*K fp16, rounded
+ * up to 256 bytes), otherwise 0 (the split-K partial sums stay in shared memory). */
 size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order);
 
-/* Registers caller-owned device scratch for later gptq_gemm calls on the current device and
- * zeroes its ticket area on `stream`.  The workspace is shared by all calls: calls that may
+/* Registers caller-owned device scratch for later gptq_gemm calls on the current device (`stream`
+ * is unused and kept for compatibility).  The workspace is shared by all calls: calls that may
  * overlap on the GPU (different streams) must not share one.  ptr = NULL unregisters. */
 int gptq_set_workspace(void *ptr, size_t bytes, void *stream);
 
@@ -124,7 +124,7 @@ int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, 
  * budget.  The split-K partial tiles, their tickets and (act-order) the gathered activations
  * live in an 8 MiB array that is part of the library image: every GPU that loads the library
  * holds it until the process exits.  Arguments, layouts and arithmetic are those of gptq_gemm.
- *  - Problems whose scratch need (gptq_workspace_bytes) exceeds gptq_noalloc_scratch_bytes()
+ *  - Problems whose scratch need (gptq_plan_noalloc's workspace_bytes) exceeds gptq_noalloc_scratch_bytes()
  *    are refused with GPTQ_ERR_WORKSPACE; nothing is launched.  (All decode shapes of the 7B
  *    and 13B layers fit up to M = 16.)
  *  - The call allocates and frees nothing, on the device or through any library.
@@ -147,20 +147,25 @@ int gptq_check_status(void *stream);
 /* ---- host-only: how a problem would be launched (no CUDA call; usable without a GPU) -- */
 
 typedef struct {
-    int kernel;       /* 1 = streaming mma.sync kernel (decode / small batch), 2 = tcgen05 prefill */
+    int kernel;       /* 1 = cluster split-K mma.sync kernel (gptq_gemm, M <= 64 per launch),
+                         3 = stream-K mma.sync kernel (gptq_gemm_noalloc) */
     int m_tile;       /* tokens per CTA tile */
     int m_chunks;     /* launches along M */
     int stages;       /* pipeline depth */
     int ctas;         /* grid size of one launch */
     int items;        /* (128-column panel, 128-row group) work items of one launch */
-    int split_panels; /* panels whose K range is shared by several CTAs (need the workspace) */
+    int split_panels; /* panels whose K range is shared by several CTAs */
     int smem_bytes;   /* dynamic shared memory per CTA */
     size_t workspace_bytes;
+    int cluster_size; /* CTAs that share one panel (kernel 1); 1 for kernel 3 */
 } gptq_plan_t;
 
+/* How gptq_gemm would launch this problem on a GPU with sm_count SMs. */
 int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out);
+/* The same for gptq_gemm_noalloc (stream-K kernel; workspace_bytes is its need of the built-in scratch). */
+int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out);
 
-/* The stream-K partition the kernel uses, from the same arithmetic: CTA `cta` of `ctas` works
+/* The stream-K partition gptq_gemm_noalloc's kernel uses, from the same arithmetic: CTA `cta` of `ctas` works
  * through items [*first_item, *end_item) of `items`; the K range of panel `panel` (its `groups`
  * consecutive items) is shared by CTAs *first_cta .. *last_cta, whose partial tiles are summed
  * in that order. */

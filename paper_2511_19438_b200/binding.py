@@ -38,7 +38,7 @@ class gptq_plan_t(ctypes.Structure):
         ("kernel", ctypes.c_int), ("m_tile", ctypes.c_int), ("m_chunks", ctypes.c_int),
         ("stages", ctypes.c_int), ("ctas", ctypes.c_int), ("items", ctypes.c_int),
         ("split_panels", ctypes.c_int), ("smem_bytes", ctypes.c_int),
-        ("workspace_bytes", ctypes.c_size_t),
+        ("workspace_bytes", ctypes.c_size_t), ("cluster_size", ctypes.c_int),
     ]
 
 
@@ -58,6 +58,7 @@ _SIGNATURES = {
     "gptq_noalloc_scratch_bytes": (_sz, []),
     "gptq_check_status": (_i, [_vp]),
     "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
+    "gptq_plan_noalloc": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_cta_range": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
     "gptq_plan_panel_owners": (_i, [_i, _i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
 }
@@ -167,6 +168,13 @@ def gptq_plan(M, N, K, group_size, act_order, sm_count):
     """Returns (status, gptq_plan_t).  Host-only: makes no CUDA call."""
     out = gptq_plan_t()
     st = _lib.gptq_plan(M, N, K, group_size, int(act_order), sm_count, ctypes.byref(out))
+    return st, out
+
+
+def gptq_plan_noalloc(M, N, K, group_size, act_order, sm_count):
+    """Returns (status, gptq_plan_t) for gptq_gemm_noalloc.  Host-only: makes no CUDA call."""
+    out = gptq_plan_t()
+    st = _lib.gptq_plan_noalloc(M, N, K, group_size, int(act_order), sm_count, ctypes.byref(out))
     return st, out
 
 

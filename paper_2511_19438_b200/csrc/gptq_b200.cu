@@ -3,6 +3,7 @@
 #include "gptq_common.cuh"
 #include "gptq_layout.cuh"
 #include "gptq_streamk.cuh"
+#include "gptq_splitk.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -59,16 +60,17 @@ static int current_device_sms(int *dev_out, int *sms_out)
     return GPTQ_OK;
 }
 
-struct GemmPlan {
+// Stream-K launch geometry and scratch need (the kernel behind gptq_gemm_noalloc).
+struct StreamKGemmPlan {
     StreamKPlan sk;          // plan of one launch (for the largest chunk)
     int m_chunks;
     size_t x_perm_bytes;     // gathered activations (act-order)
     size_t workspace_bytes;  // 0 if nothing is needed
 };
 
-static GemmPlan make_plan(int M, int N, int K, int act_order, int sm_count)
+static StreamKGemmPlan make_streamk_plan(int M, int N, int K, int act_order, int sm_count)
 {
-    GemmPlan gp{};
+    StreamKGemmPlan gp{};
     const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
     gp.sk = plan_streamk(rows, N, K, sm_count);
     gp.m_chunks = (M + kStreamKMaxRows - 1) / kStreamKMaxRows;
@@ -76,6 +78,12 @@ static GemmPlan make_plan(int M, int N, int K, int act_order, int sm_count)
     const size_t need = gp.sk.partial_bytes + gp.x_perm_bytes;
     gp.workspace_bytes = need ? kTicketAreaBytes + need : 0;
     return gp;
+}
+
+// gptq_gemm keeps its split-K partials on chip; its only scratch is the gathered x of act-order layers.
+static size_t gemm_workspace_need(int M, int K, int act_order)
+{
+    return act_order ? (((size_t)M * K * sizeof(__half) + 255) & ~(size_t)255) : 0;
 }
 
 }  // namespace gptq
@@ -165,8 +173,31 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     st = check_fast_path(N, K, group_size);
     if (st) return st;
     if (sm_count < 1) return GPTQ_ERR_SHAPE;
-    const GemmPlan gp = make_plan(M, N, K, act_order, sm_count);
+    const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
+    const SplitKPlan pl = plan_splitk(rows, N, K, sm_count);
     out->kernel = 1;
+    out->m_tile = pl.m_tile;
+    out->m_chunks = (M + kStreamKMaxRows - 1) / kStreamKMaxRows;
+    out->stages = pl.stages;
+    out->ctas = pl.ctas;
+    out->items = (N / kPanel) * (K / kGroup);
+    out->split_panels = pl.S > 1 ? N / kPanel : 0;
+    out->smem_bytes = pl.smem_bytes;
+    out->workspace_bytes = gemm_workspace_need(M, K, act_order);
+    out->cluster_size = pl.S;
+    return GPTQ_OK;
+}
+
+int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out)
+{
+    if (!out) return GPTQ_ERR_NULL;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    st = check_fast_path(N, K, group_size);
+    if (st) return st;
+    if (sm_count < 1) return GPTQ_ERR_SHAPE;
+    const StreamKGemmPlan gp = make_streamk_plan(M, N, K, act_order, sm_count);
+    out->kernel = 3;
     out->m_tile = gp.sk.m_tile;
     out->m_chunks = gp.m_chunks;
     out->stages = gp.sk.stages;
@@ -175,6 +206,7 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     out->split_panels = gp.sk.split_panels;
     out->smem_bytes = gp.sk.smem_bytes;
     out->workspace_bytes = gp.workspace_bytes;
+    out->cluster_size = 1;
     return GPTQ_OK;
 }
 
@@ -202,28 +234,19 @@ int gptq_plan_panel_owners(int items, int ctas, int groups, int panel, int *firs
 size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order)
 {
     if (check_shape(M, N, K, group_size) != GPTQ_OK || check_fast_path(N, K, group_size) != GPTQ_OK) return 0;
-    int dev, sms;
-    if (current_device_sms(&dev, &sms) != GPTQ_OK) return 0;
-    return make_plan(M, N, K, act_order, sms).workspace_bytes;
+    return gemm_workspace_need(M, K, act_order);
 }
 
 int gptq_set_workspace(void *ptr, size_t bytes, void *stream)
 {
+    (void)stream;
     int dev, sms;
     int st = current_device_sms(&dev, &sms);
     if (st) return st;
-    if (ptr == nullptr) {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        g_workspace[dev] = Workspace{};
-        return GPTQ_OK;
-    }
-    if (!aligned16(ptr)) return GPTQ_ERR_ALIGN;
-    if (bytes < kTicketAreaBytes) return GPTQ_ERR_WORKSPACE;
-    st = record_cuda_error(cudaMemsetAsync(ptr, 0, kTicketAreaBytes, (cudaStream_t)stream));
-    if (st) return st;
+    if (ptr != nullptr && !aligned16(ptr)) return GPTQ_ERR_ALIGN;
     std::lock_guard<std::mutex> lock(g_mutex);
     g_workspace[dev].ptr = ptr;
-    g_workspace[dev].bytes = bytes;
+    g_workspace[dev].bytes = ptr ? bytes : 0;
     return GPTQ_OK;
 }
 
@@ -241,30 +264,25 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
     int dev, sms;
     st = current_device_sms(&dev, &sms);
     if (st) return st;
-    const GemmPlan gp = make_plan(M, N, K, act_order, sms);
-    Workspace ws;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        ws = g_workspace[dev];
-    }
-    if (gp.workspace_bytes > 0 && (ws.ptr == nullptr || ws.bytes < gp.workspace_bytes)) return GPTQ_ERR_WORKSPACE;
-
     cudaStream_t s = (cudaStream_t)stream;
-    uint8_t *wsb = (uint8_t *)ws.ptr;
-    int *tickets = (int *)wsb;
-    float *partials = gp.workspace_bytes ? (float *)(wsb + kTicketAreaBytes) : nullptr;
     const __half *xin = (const __half *)x;
     if (act_order) {
-        __half *x_perm = (__half *)(wsb + kTicketAreaBytes + gp.sk.partial_bytes);
+        Workspace ws;
+        {
+            std::lock_guard<std::mutex> lock(g_mutex);
+            ws = g_workspace[dev];
+        }
+        if (ws.ptr == nullptr || ws.bytes < gemm_workspace_need(M, K, act_order)) return GPTQ_ERR_WORKSPACE;
+        __half *x_perm = (__half *)ws.ptr;
         st = launch_gather_x((const __half *)x, g_idx, x_perm, M, K, s);
         if (st) return st;
         xin = x_perm;
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
-        const StreamKPlan pl = plan_streamk(rows, N, K, sms);
-        st = launch_streamk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
-                            pl, partials, tickets, s);
+        const SplitKPlan pl = plan_splitk(rows, N, K, sms);
+        st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
+                           pl, s);
         if (st) return st;
     }
     return GPTQ_OK;
@@ -325,7 +343,7 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
     int dev, sms;
     st = current_device_sms(&dev, &sms);
     if (st) return st;
-    const GemmPlan gp = make_plan(M, N, K, act_order, sms);
+    const StreamKGemmPlan gp = make_streamk_plan(M, N, K, act_order, sms);
     // the built-in scratch has a fixed size: larger problems must use gptq_gemm with a workspace
     if (gp.workspace_bytes > kStaticScratchBytes) return GPTQ_ERR_WORKSPACE;
     void *base = nullptr;

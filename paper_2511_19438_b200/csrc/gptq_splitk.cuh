@@ -1,0 +1,371 @@
+// Decode / small-batch GPTQ matmul (M <= 64 per launch): HBM-bound streaming with split-K inside a
+// thread-block cluster.
+//
+// A CTA owns one 128-column panel and a contiguous range of its K groups; the S CTAs that share a
+// panel form one cluster (S = 1..8, chosen so that panels * S fills the SMs once).  A producer
+// thread streams the CTA's items (8 KB of packed weights, 256 B of scales, 64 B of zeros, one
+// swizzled tensor-map tile of x per K64 block) through a shared-memory ring guarded by
+// mbarriers; weights are fetched before griddepcontrol.wait, so they overlap the previous kernel.
+// Eight consumer warps each own 16 columns: a lane reads its 16-byte chunk, turns nibbles into
+// fp16 pairs with lop3 (1024+q or 64+q, exact), subtracts the zero as packed half2 (exact integer
+// q - z) and feeds them as the 16-row A operand of mma.sync.m16n8k16, tokens as the 8-wide B
+// operand.  The group's scale multiplies the fp32 group sum once per group.
+//
+// The K-partials of a panel never touch global memory: every CTA parks its fp32 tile in its own
+// shared memory, the cluster synchronises, and CTA r sums columns [128 r / S, 128 (r+1) / S) of
+// all S tiles through distributed shared memory in rank order (a fixed order: results are
+// reproducible), rounds once to fp16 and stores y.
+#pragma once
+#include "gptq_common.cuh"
+#include "gptq_tma.cuh"
+#include "gptq_streamk.cuh"   // ring geometry (streamk_stage_bytes, token_row_of_slot, thread counts)
+
+namespace gptq {
+
+__device__ __forceinline__ void cluster_arrive_release()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire()
+{
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cluster_rank(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    return remote;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+struct SplitKArgs {
+    const uint8_t *qweight; // tiled
+    const uint8_t *scales;
+    const uint8_t *qzeros;
+    __half *y;              // [M, N]
+    int M, N, K, G;
+    int S;                  // CTAs per panel = cluster size
+    int stages;
+};
+
+struct SplitKPlan {
+    int m_tile;     // 8, 16, 32 or 64
+    int S;
+    int stages;
+    int ctas;       // panels * S
+    int smem_bytes;
+};
+
+template <int MT>
+__global__ void __launch_bounds__(kStreamKThreads, MT == 1 ? 3 : MT == 2 ? 2 : 1)
+splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
+{
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int kStage = streamk_stage_bytes(MT);
+    constexpr int kXTile = MT * 1024;                       // one K64 tile of x
+    constexpr int kOffW = streamk_x_bytes(MT), kOffS = kOffW + kItemWBytes, kOffZ = kOffS + kItemSBytes;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_full = smem_base;                  // stages x 8 B
+    const uint32_t bar_empty = smem_base + 64;            // stages x 8 B
+    const uint32_t ring = smem_base + kRingOffset;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = a.S;
+    const int p = blockIdx.x / S, rank = blockIdx.x - p * S;   // cluster = the S CTAs of panel p
+    const int g0 = rank * a.G / S, g1 = (rank + 1) * a.G / S;  // this CTA's groups
+    const int n_items = g1 - g0;
+    const int t0 = p * a.G + g0;
+    const int stages = a.stages;
+
+    if (threadIdx.x == kConsumerThreads) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kConsumerWarps);
+        }
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    float acc[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+    const int g = lane >> 2, t4 = lane & 3;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer (one thread)
+        if (lane == 0) {
+            const uint64_t policy = l2_policy_evict_first();
+            tma_prefetch_descriptor(&x_map);
+            const uint32_t meta_bytes = kItemWBytes + kItemSBytes + kItemZBytes;
+            const int n_pre = n_items < stages ? n_items : stages;
+            auto issue_weights = [&](int t, int s) {
+                const uint32_t dst = ring + s * kStage, bar = bar_full + 8 * s;
+                mbar_expect_tx(bar, meta_bytes);
+                bulk_g2s_hint(dst + kOffW, a.qweight + (size_t)t * kItemWBytes, kItemWBytes, bar, policy);
+                bulk_g2s_hint(dst + kOffS, a.scales + (size_t)t * kItemSBytes, kItemSBytes, bar, policy);
+                bulk_g2s_hint(dst + kOffZ, a.qzeros + (size_t)t * kItemZBytes, kItemZBytes, bar, policy);
+            };
+            // weights never depend on earlier work in the stream: fill the ring before waiting on it
+            for (int i = 0; i < n_pre; ++i) issue_weights(t0 + i, i);
+            pdl_wait();
+            int s = 0, round = 0;
+            for (int it = 0; it < n_items; ++it) {
+                const uint32_t bar = bar_full + 8 * s;
+                if (it >= stages) {
+                    if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
+                    issue_weights(t0 + it, s);
+                }
+                // the group's activations for all token rows: two swizzled K64 tiles, rows >= M read as zero
+                mbar_arrive_expect_tx(bar, (uint32_t)streamk_x_bytes(MT));
+                const uint32_t dst = ring + s * kStage;
+                const int k0 = (g0 + it) * kGroup;
+                tma_load_2d(dst, &x_map, k0, 0, bar);
+                tma_load_2d(dst + kXTile, &x_map, k0 + 64, 0, bar);
+                if (++s == stages) { s = 0; ++round; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        pdl_wait();
+        const int r = token_row_of_slot(g);
+        const uint32_t w_off = kOffW + warp * kUnitBytes + lane * 16;
+        const uint32_t s_off = kOffS + (warp * 16 + 2 * g) * 2;
+        const uint32_t z_off = kOffZ + warp * 8 + g;
+        // x fragment of k chunk (4j + t4) for token slot g: row r of the swizzled tile
+        const uint32_t x_off0 = r * 128 + ((uint32_t)(t4 ^ r) << 4);          // j = 0
+        const uint32_t x_off1 = r * 128 + ((uint32_t)((4 + t4) ^ r) << 4);    // j = 1
+        constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
+
+        int s = 0;
+        uint32_t phase = 0;
+        bool ok = true;   // false after a wait gave up: keep taking part in barriers, skip the data
+        for (int it = 0; it < n_items; ++it) {
+            const uint32_t st = ring + s * kStage;
+            if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
+
+            const uint4 wq0 = lds128(st + w_off);
+            const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
+            const uint32_t sc = lds32(st + s_off);
+            const uint32_t zb = lds8(st + z_off);
+            const uint32_t zA = zb & 15u, zB = zb >> 4;
+            const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
+            const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+
+            // two accumulator sets (one per K64 block) halve the dependent MMA chain
+            constexpr int kSets = MT <= 2 ? 2 : 1;
+            float accg[kSets][MT][4];
+#pragma unroll
+            for (int q = 0; q < kSets; ++q)
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) accg[q][mt][i] = 0.f;
+
+#pragma unroll
+            for (int blk = 0; blk < 2; ++blk) {
+                const uint4 wq = blk ? wq1 : wq0;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
+                    const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+                    const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+                    const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+                    const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+                    wA >>= 8;
+                    wB >>= 8;
+                    const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+                    const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+                    const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+                    const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
+                        mma_m16n8k16(accg[blk % kSets][mt], a0, a1, a2, a3, xb.x, xb.y);
+                        mma_m16n8k16(accg[blk % kSets][mt], c0, c1, c2, c3, xb.z, xb.w);
+                    }
+                }
+            }
+            // release the stage, then fold the group sum into the running sum with the group's scale
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            if (++s == stages) { s = 0; phase ^= 1u; }
+
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                if (kSets == 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) accg[0][mt][i] += accg[kSets - 1][mt][i];
+                }
+                acc[mt][0] = fmaf(sf.x, accg[0][mt][0], acc[mt][0]);
+                acc[mt][1] = fmaf(sf.x, accg[0][mt][1], acc[mt][1]);
+                acc[mt][2] = fmaf(sf.y, accg[0][mt][2], acc[mt][2]);
+                acc[mt][3] = fmaf(sf.y, accg[0][mt][3], acc[mt][3]);
+            }
+        }
+    }
+
+    // accumulator i of tile mt: weight column col + 8*(i>>1), token slot 2*t4 + (i&1)
+    const int col = warp * 16 + g;
+    const int m_lo = token_row_of_slot(2 * t4), m_hi = token_row_of_slot(2 * t4 + 1);
+    if (S == 1) {
+        if (warp < kConsumerWarps) {
+            __half *yp = a.y + (size_t)p * kPanel + col;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
+                    if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
+                }
+        }
+        return;
+    }
+
+    // ---- split-K: park this CTA's fp32 tile [MT*8 rows][128 cols] at the start of the ring ----------
+    if (warp < kConsumerWarps) {
+        named_bar_sync(1, kConsumerThreads);   // every consumer warp has finished reading the ring
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
+                sts_f32(ring + (uint32_t)(m * kPanel + col + 8 * (i >> 1)) * 4u, acc[mt][i]);
+            }
+    }
+    __syncwarp();
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp < kConsumerWarps) {
+        // CTA `rank` finishes columns [c_lo, c_lo + width) of the panel for every token row
+        const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
+        for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
+            const int m = idx / width, cc = c_lo + idx - m * width;
+            const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
+            float sum = 0.f;
+            for (int q = 0; q < S; ++q) sum += ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)q));
+            a.y[(size_t)m * a.N + (size_t)p * kPanel + cc] = __float2half_rn(sum);
+        }
+    }
+    // no CTA may exit (and free its shared memory) while a peer can still read its tile
+    __syncwarp();
+    cluster_arrive_release();
+    cluster_wait_acquire();
+}
+
+// Resident CTAs per SM by token tile: registers and ring size are set so that three CTAs of the
+// narrowest tile fit, which lets the next kernel's first CTAs start (and prefetch weights) early.
+__host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT == 1 ? 3 : MT == 2 ? 2 : 1; }
+
+// Picks the cluster size S in {1, 2, 4, 8} with the smallest estimated time.  The estimate is the
+// busiest SM's item count at the measured per-SM item rate, bounded below by one CTA's own serial
+// rate, plus the cluster reduction when S > 1 (hundredths of a microsecond; only ratios matter).
+SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
+{
+    SplitKPlan pl{};
+    const int MT = streamk_m_tile(m_rows);
+    const int G = K / kGroup, panels = N / kPanel;
+    const int stage = streamk_stage_bytes(MT);
+    const int cps = splitk_ctas_per_sm(MT);
+    int best_S = 1;
+    long long best_t = -1;
+    for (int S = 1; S <= 8; S *= 2) {
+        if (S > G) break;
+        const long long ctas = (long long)panels * S, ipc = (G + S - 1) / S;
+        const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
+        const long long serial = ipc * 45, shared = on_busiest_sm * ipc * 30;
+        const long long t = (serial > shared ? serial : shared) + (S > 1 ? 100 : 0);
+        if (best_t < 0 || t < best_t) { best_t = t; best_S = S; }
+    }
+    const int S = best_S;
+    const int items_per_cta = (G + S - 1) / S;
+    const int ring_budget = (227 * 1024) / cps - 1024 - 2 * kRingOffset;
+    int stages = ring_budget / stage;
+    if (stages > 8) stages = 8;
+    if (stages > items_per_cta) stages = items_per_cta;
+    // the ring doubles as the fp32 partial tile (MT * 4 KB) at the end
+    while (stages * stage < MT * 4096) ++stages;
+    pl.m_tile = MT * 8;
+    pl.S = S;
+    pl.stages = stages;
+    pl.ctas = panels * S;
+    pl.smem_bytes = 2 * kRingOffset + stages * stage;
+    return pl;
+}
+
+template <int MT>
+static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, const SplitKPlan &plan, cudaStream_t s)
+{
+    static int configured_smem[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
+    if (configured_smem[dev] < plan.smem_bytes) {
+        e = cudaFuncSetAttribute(splitk_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaFuncSetAttribute(splitk_kernel<MT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        configured_smem[dev] = plan.smem_bytes;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)plan.ctas);
+    cfg.blockDim = dim3(kStreamKThreads);
+    cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)plan.S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, splitk_kernel<MT>, args, x_map));
+}
+
+int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
+                  int M, int N, int K, const SplitKPlan &plan, cudaStream_t s)
+{
+    SplitKArgs args;
+    args.qweight = (const uint8_t *)qweight;
+    args.scales = (const uint8_t *)scales;
+    args.qzeros = (const uint8_t *)qzeros;
+    args.y = y;
+    args.M = M;
+    args.N = N;
+    args.K = K;
+    args.G = K / kGroup;
+    args.S = plan.S;
+    args.stages = plan.stages;
+    // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
+    CUtensorMap x_map;
+    int st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
+                                (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.m_tile, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st) return st;
+    switch (plan.m_tile) {
+    case 8: return launch_splitk_mt<1>(args, x_map, plan, s);
+    case 16: return launch_splitk_mt<2>(args, x_map, plan, s);
+    case 32: return launch_splitk_mt<4>(args, x_map, plan, s);
+    case 64: return launch_splitk_mt<8>(args, x_map, plan, s);
+    default: return GPTQ_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace gptq

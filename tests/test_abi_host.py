@@ -91,8 +91,29 @@ SHAPES = list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()) + [(128, 128
 @pytest.mark.parametrize("K,N", SHAPES)
 @pytest.mark.parametrize("M", [1, 8, 9, 16, 33, 64, 200])
 @pytest.mark.parametrize("sms", [148, 132, 7])
-def test_plan_is_consistent(K, N, M, sms):
+def test_cluster_plan_is_consistent(K, N, M, sms):
     st, pl = B.gptq_plan(M, N, K, 128, 0, sms)
+    assert st == B.GPTQ_OK
+    G, panels = K // 128, N // 128
+    assert pl.kernel == 1 and pl.items == G * panels
+    assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
+    assert pl.ctas == panels * pl.cluster_size
+    assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
+    assert pl.m_tile in (8, 16, 32, 64) and pl.m_tile >= min(M, 64)
+    assert pl.m_chunks == (M + 63) // 64
+    assert 1 <= pl.stages <= 8
+    per_sm = 3 if pl.m_tile == 8 else 2 if pl.m_tile == 16 else 1
+    assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024
+    # the ring doubles as the fp32 partial tile of the cluster reduction
+    assert pl.smem_bytes - 2048 >= pl.m_tile * 128 * 4
+    assert pl.workspace_bytes == 0          # the partial sums stay on chip
+
+
+@pytest.mark.parametrize("K,N", SHAPES)
+@pytest.mark.parametrize("M", [1, 8, 9, 16, 33, 64, 200])
+@pytest.mark.parametrize("sms", [148, 132, 7])
+def test_streamk_plan_is_consistent(K, N, M, sms):
+    st, pl = B.gptq_plan_noalloc(M, N, K, 128, 0, sms)
     assert st == B.GPTQ_OK
     G, panels = K // 128, N // 128
     assert pl.items == G * panels
@@ -143,10 +164,12 @@ def test_plan_is_consistent(K, N, M, sms):
 
 
 def test_plan_act_order_adds_gathered_x():
-    st, a = B.gptq_plan(8, 5120, 13824, 128, 0, 148)
-    st2, b = B.gptq_plan(8, 5120, 13824, 128, 1, 148)
-    assert st == st2 == B.GPTQ_OK
-    assert b.workspace_bytes - a.workspace_bytes >= 8 * 13824 * 2 or a.workspace_bytes == 0
+    for plan in (B.gptq_plan, B.gptq_plan_noalloc):
+        st, a = plan(8, 5120, 13824, 128, 0, 148)
+        st2, b = plan(8, 5120, 13824, 128, 1, 148)
+        assert st == st2 == B.GPTQ_OK
+        assert b.workspace_bytes - a.workspace_bytes >= 8 * 13824 * 2
+    assert B.gptq_plan(8, 5120, 13824, 128, 0, 148)[1].workspace_bytes == 0
 
 
 def test_plan_rejects_bad_arguments():

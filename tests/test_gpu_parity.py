@@ -181,20 +181,29 @@ def test_gemm_is_deterministic_and_leaves_neighbours_alone(ws):
 
 
 def test_gemm_without_workspace_is_refused_not_wrong():
-    K, N = 4096, 4096                       # split panels on any GPU with more than 32 SMs
-    L = wl.make_linear(K, N, seed=121)
+    K, N, M = 1024, 256, 3                  # act-order: the gathered x needs caller scratch
+    L = wl.make_linear(K, N, seed=121, act_order=True)
     D = H.upload_and_repack(L)
-    need = B.gptq_workspace_bytes(1, N, K, 128, 0)
-    assert need > 0
+    need = B.gptq_workspace_bytes(M, N, K, 128, 1)
+    assert need >= M * K * 2
+    assert B.gptq_workspace_bytes(M, N, K, 128, 0) == 0
     B.check(B.gptq_set_workspace(None, 0), "unset")
-    x = H.to_device(wl.make_x(1, K, 122))
-    y = torch.zeros((1, N), dtype=torch.float16, device="cuda")
-    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 1, N, K, 128, 0) == B.GPTQ_ERR_WORKSPACE
+    x = H.to_device(wl.make_x(M, K, 122))
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    args = (x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, N, K, 128, 1)
+    assert B.gptq_gemm(*args) == B.GPTQ_ERR_WORKSPACE
     small = torch.empty(need - 16, dtype=torch.uint8, device="cuda")
     B.check(B.gptq_set_workspace(small, small.numel()), "small ws")
-    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 1, N, K, 128, 0) == B.GPTQ_ERR_WORKSPACE
+    assert B.gptq_gemm(*args) == B.GPTQ_ERR_WORKSPACE
     B.check(B.gptq_set_workspace(None, 0), "unset")
+    torch.cuda.synchronize()
     assert torch.count_nonzero(y) == 0
+    # without act-order no workspace is needed at all
+    L2 = wl.make_linear(K, N, seed=123)
+    D2 = H.upload_and_repack(L2)
+    x_np = wl.make_x(M, K, 124)
+    y2 = H.gemm(H.to_device(x_np), D2).cpu().numpy()
+    assert_close(y2, oracle.gemm_f64(x_np, L2.qweight, L2.qzeros, L2.scales, None, 128), K)
 
 
 def test_gemm_host_round_trip(ws):

@@ -5,8 +5,8 @@ started and must not call cudaMalloc afterwards (it is forbidden by the host pro
 stall the device in the middle of a latency-bound decode loop), so they cannot give gptq_gemm a
 workspace.  gptq_gemm_noalloc keeps its split-K scratch in an array inside the library instead.
 These tests call it through the C ABI twice in a row (the array keeps the first call's contents)
-and require the same fp16 outputs as gptq_gemm, whose summation order it shares, and the usual
-tolerance against the CPU oracle.  The file sorts last on purpose: a run that stops at the first
+and require agreement with gptq_gemm (a different kernel, so a different summation order) and
+with the CPU oracle, both within the tolerance the parity tests state.  The file sorts last on purpose: a run that stops at the first
 failure has then already run every other test.
 """
 import math
@@ -32,14 +32,20 @@ def within_stated_tolerance(y, y64, K):
     return np.all(err <= 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64))
 
 
+def noalloc_scratch_need(M, N, K, act):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    st, pl = B.gptq_plan_noalloc(M, N, K, 128, act, sms)
+    assert st == B.GPTQ_OK
+    return pl.workspace_bytes
+
+
 @pytest.mark.parametrize("K,N,M,act", [(4096, 4096, 1, False), (4096, 4096, 8, False), (2560, 1280, 5, True)])
 def test_noalloc_matches_gemm_on_two_calls_in_a_row(K, N, M, act):
     L = wl.make_linear(K, N, seed=wl.seed_for("noalloc", K, N, act), act_order=act)
     D = H.upload_and_repack(L)
-    need = B.gptq_workspace_bytes(M, N, K, 128, act)
-    assert 0 < need <= B.gptq_noalloc_scratch_bytes()       # these cases do use the scratch
+    assert 0 < noalloc_scratch_need(M, N, K, act) <= B.gptq_noalloc_scratch_bytes()   # the scratch is used
     ws = H.WorkspaceHolder()
-    ws.ensure(need)
+    ws.ensure_for(M, D)
     outs = []
     for call in range(2):                                   # second call meets a used scratch array
         x_np = wl.make_x(M, K, wl.seed_for("noalloc-x", K, M, call))
@@ -49,7 +55,8 @@ def test_noalloc_matches_gemm_on_two_calls_in_a_row(K, N, M, act):
         B.check(B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, N, K, 128, act),
                 "gptq_gemm_noalloc")
         assert B.gptq_check_status() == B.GPTQ_OK
-        assert torch.equal(y, want), f"call {call}: differs from gptq_gemm"
+        assert within_stated_tolerance(y.cpu().numpy(), want.cpu().numpy().astype(np.float64), K), \
+            f"call {call}: differs from gptq_gemm"
         y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
         assert within_stated_tolerance(y.cpu().numpy(), y64, K)
         outs.append(y)
@@ -57,23 +64,23 @@ def test_noalloc_matches_gemm_on_two_calls_in_a_row(K, N, M, act):
 
 
 def test_noalloc_needs_no_registered_workspace():
-    K, N, M = 4096, 4096, 4
-    L = wl.make_linear(K, N, seed=wl.seed_for("noalloc-unreg"))
+    K, N, M = 2048, 512, 4                                  # act-order: gptq_gemm needs a workspace here
+    L = wl.make_linear(K, N, seed=wl.seed_for("noalloc-unreg"), act_order=True)
     D = H.upload_and_repack(L)
     x_np = wl.make_x(M, K, 7)
     x = H.to_device(x_np)
     y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
     B.check(B.gptq_set_workspace(None, 0), "unregister")
-    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, N, K, 128, 0) == B.GPTQ_ERR_WORKSPACE
-    B.check(B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, N, K, 128, 0), "noalloc")
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, N, K, 128, 1) == B.GPTQ_ERR_WORKSPACE
+    B.check(B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, N, K, 128, 1), "noalloc")
     assert B.gptq_check_status() == B.GPTQ_OK
-    y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, None, 128)
+    y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
     assert within_stated_tolerance(y.cpu().numpy(), y64, K)
 
 
 def test_noalloc_refuses_problems_beyond_its_scratch():
     K, N, M = 4096, 22016, 64                               # needs ~19 MB of partial tiles
-    assert B.gptq_workspace_bytes(M, N, K, 128, 0) > B.gptq_noalloc_scratch_bytes()
+    assert noalloc_scratch_need(M, N, K, 0) > B.gptq_noalloc_scratch_bytes()
     L = wl.make_linear(K, N, seed=wl.seed_for("noalloc-big"))
     D = H.upload_and_repack(L)
     x = H.to_device(wl.make_x(M, K, 9))
