@@ -161,60 +161,52 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
             const uint32_t sc = lds32(st + s_off);
             const uint32_t zb = lds8(st + z_off);
-            const uint32_t zA = zb & 15u, zB = zb >> 4;
-            const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
-            const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+            const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
 
-            // two accumulator sets (one per K64 block) halve the dependent MMA chain
-            constexpr int kSets = MT <= 2 ? 2 : 1;
-            float accg[kSets][MT][4];
-#pragma unroll
-            for (int q = 0; q < kSets; ++q)
+            {
+                const uint32_t zA = zb & 15u, zB = zb >> 4;
+                const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
+                const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+                float accg[MT][4];
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) accg[q][mt][i] = 0.f;
-
+                    for (int i = 0; i < 4; ++i) accg[mt][i] = 0.f;
 #pragma unroll
-            for (int blk = 0; blk < 2; ++blk) {
-                const uint4 wq = blk ? wq1 : wq0;
+                for (int blk = 0; blk < 2; ++blk) {
+                    const uint4 wq = blk ? wq1 : wq0;
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
-                    const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                    const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                    const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                    const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
-                    wA >>= 8;
-                    wB >>= 8;
-                    const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                    const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                    const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                    const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+                    for (int j = 0; j < 2; ++j) {
+                        uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
+                        const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+                        const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+                        const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+                        const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+                        wA >>= 8;
+                        wB >>= 8;
+                        const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+                        const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+                        const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+                        const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
-                        mma_m16n8k16(accg[blk % kSets][mt], a0, a1, a2, a3, xb.x, xb.y);
-                        mma_m16n8k16(accg[blk % kSets][mt], c0, c1, c2, c3, xb.z, xb.w);
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
+                            mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
+                            mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
+                        }
                     }
                 }
-            }
-            // release the stage, then fold the group sum into the running sum with the group's scale
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-            if (++s == stages) { s = 0; phase ^= 1u; }
-
-            const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
+                // release the stage, then fold the group sum into the running sum with the group's scale
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+                if (++s == stages) { s = 0; phase ^= 1u; }
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                if (kSets == 2) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) accg[0][mt][i] += accg[kSets - 1][mt][i];
+                for (int mt = 0; mt < MT; ++mt) {
+                    acc[mt][0] = fmaf(sf.x, accg[mt][0], acc[mt][0]);
+                    acc[mt][1] = fmaf(sf.x, accg[mt][1], acc[mt][1]);
+                    acc[mt][2] = fmaf(sf.y, accg[mt][2], acc[mt][2]);
+                    acc[mt][3] = fmaf(sf.y, accg[mt][3], acc[mt][3]);
                 }
-                acc[mt][0] = fmaf(sf.x, accg[0][mt][0], acc[mt][0]);
-                acc[mt][1] = fmaf(sf.x, accg[0][mt][1], acc[mt][1]);
-                acc[mt][2] = fmaf(sf.y, accg[0][mt][2], acc[mt][2]);
-                acc[mt][3] = fmaf(sf.y, accg[0][mt][3], acc[mt][3]);
             }
         }
     }
@@ -256,8 +248,12 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
             const int m = idx / width, cc = c_lo + idx - m * width;
             const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = q < S ? ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)q)) : 0.f;
             float sum = 0.f;
-            for (int q = 0; q < S; ++q) sum += ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)q));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) sum += v[q];   // rank order
             a.y[(size_t)m * a.N + (size_t)p * kPanel + cc] = __float2half_rn(sum);
         }
     }
@@ -271,30 +267,39 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 // narrowest tile fit, which lets the next kernel's first CTAs start (and prefetch weights) early.
 __host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT == 1 ? 3 : MT == 2 ? 2 : 1; }
 
-// Picks the cluster size S in {1, 2, 4, 8} with the smallest estimated time.  The estimate is the
-// busiest SM's item count at the measured per-SM item rate, bounded below by one CTA's own serial
-// rate, plus the cluster reduction when S > 1 (hundredths of a microsecond; only ratios matter).
+// Picks the cluster size S in {1, 2, 4, 8} with the smallest estimated time among those whose
+// panels * S CTAs are all resident at once (falling back to all S if none is).  The estimate is
+// the busiest SM's item count at the measured per-SM item rate, bounded below by one CTA's own
+// serial rate, plus the cluster reduction when S > 1 (hundredths of a microsecond; only ratios
+// matter).  Shared memory is then padded so that exactly ceil(CTAs / SMs) CTAs fit on an SM: the
+// cluster scheduler otherwise packs three CTAs onto some SMs and leaves others empty.
 SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
 {
     SplitKPlan pl{};
     const int MT = streamk_m_tile(m_rows);
     const int G = K / kGroup, panels = N / kPanel;
     const int stage = streamk_stage_bytes(MT);
-    const int cps = splitk_ctas_per_sm(MT);
+    const int cps_max = splitk_ctas_per_sm(MT);
     int best_S = 1;
     long long best_t = -1;
-    for (int S = 1; S <= 8; S *= 2) {
-        if (S > G) break;
-        const long long ctas = (long long)panels * S, ipc = (G + S - 1) / S;
-        const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
-        const long long serial = ipc * 45, shared = on_busiest_sm * ipc * 30;
-        const long long t = (serial > shared ? serial : shared) + (S > 1 ? 100 : 0);
-        if (best_t < 0 || t < best_t) { best_t = t; best_S = S; }
+    for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
+        for (int S = 1; S <= 8; S *= 2) {
+            if (S > G) break;
+            const long long ctas = (long long)panels * S, ipc = (G + S - 1) / S;
+            const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
+            if (pass == 0 && on_busiest_sm > cps_max) continue;
+            const long long serial = ipc * 45, shared = on_busiest_sm * ipc * 30;
+            const long long t = (serial > shared ? serial : shared) + (S > 1 ? 100 : 0);
+            if (best_t < 0 || t < best_t) { best_t = t; best_S = S; }
+        }
     }
     const int S = best_S;
     const int items_per_cta = (G + S - 1) / S;
-    const int ring_budget = (227 * 1024) / cps - 1024 - 2 * kRingOffset;
-    int stages = ring_budget / stage;
+    int per_sm = (panels * S + sm_count - 1) / sm_count;
+    if (per_sm > cps_max) per_sm = cps_max;
+    const int smem_cap = (227 * 1024) / per_sm - 1024;                 // per_sm CTAs fit ...
+    const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;          // ... per_sm + 1 do not
+    int stages = (smem_cap - 2 * kRingOffset) / stage;
     if (stages > 8) stages = 8;
     if (stages > items_per_cta) stages = items_per_cta;
     // the ring doubles as the fp32 partial tile (MT * 4 KB) at the end
@@ -304,6 +309,7 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
     pl.stages = stages;
     pl.ctas = panels * S;
     pl.smem_bytes = 2 * kRingOffset + stages * stage;
+    if (pl.smem_bytes < smem_floor) pl.smem_bytes = smem_floor;
     return pl;
 }
 
