@@ -4,6 +4,7 @@
 #include "gptq_layout.cuh"
 #include "gptq_streamk.cuh"
 #include "gptq_splitk.cuh"
+#include "gptq_umma.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -173,6 +174,20 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     st = check_fast_path(N, K, group_size);
     if (st) return st;
     if (sm_count < 1) return GPTQ_ERR_SHAPE;
+    if (M > kStreamKMaxRows) {
+        const UmmaPlan up = plan_umma(M, N);
+        out->kernel = 2;
+        out->m_tile = up.tok;
+        out->m_chunks = 1;
+        out->stages = up.stages;
+        out->ctas = up.ctas;
+        out->items = (N / kPanel) * (K / kGroup);
+        out->split_panels = 0;
+        out->smem_bytes = up.smem_bytes;
+        out->workspace_bytes = gemm_workspace_need(M, K, act_order);
+        out->cluster_size = 1;
+        return GPTQ_OK;
+    }
     const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
     const SplitKPlan pl = plan_splitk(rows, N, K, sm_count);
     out->kernel = 1;
@@ -277,6 +292,11 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
         st = launch_gather_x((const __half *)x, g_idx, x_perm, M, K, s);
         if (st) return st;
         xin = x_perm;
+    }
+    if (M > kStreamKMaxRows) {
+        // many tokens: tcgen05 kernel, 128-token tiles
+        const UmmaPlan pl = plan_umma(M, N);
+        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, pl, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;

@@ -1,0 +1,398 @@
+// Prefill GPTQ matmul (many tokens): tcgen05 tensor cores with the dequantisation fused in front
+// of the MMA.
+//
+// Swap-AB: a CTA computes D[n, m] = sum_k W^T[n, k] x^T[k, m] for one 128-column panel (the MMA's
+// M = 128 rows, one TMEM lane per weight column) and a tile of TOK tokens (the MMA's N).  x[M, K]
+// row-major is already the K-major B operand, so it goes from global memory to swizzled shared
+// memory by TMA and is read by the tensor core through a shared-memory descriptor.  The weights
+// need arithmetic, so they take another road: TMA brings the packed K64 block of the panel (4 KB,
+// 64-byte swizzle) to shared memory, four dequant warps (one per 32 TMEM lanes) read the eight
+// words of "their" column, turn nibbles into fp16 with lop3 (1024+q / 64+q), subtract the zero
+// (exact integer) and multiply by the group scale as packed half2, and write the 64 fp16 values
+// with tcgen05.st into a ring of A-operand stages in tensor memory.  One thread issues
+// tcgen05.mma (kind::f16, A from TMEM, B from shared memory, fp32 accumulator in TMEM) and
+// tcgen05.commit hands ring slots back through mbarriers.  At the end of the K loop the dequant
+// warps read the accumulator with tcgen05.ld, round once to fp16 and store y.
+//
+// Two CTAs fit on an SM (256 TMEM columns and <= 110 KB of shared memory each), so one CTA's
+// epilogue overlaps the other's main loop.  Every wait is bounded.
+#pragma once
+#include "gptq_common.cuh"
+#include "gptq_tma.cuh"
+
+namespace gptq {
+
+constexpr int kUmmaThreads = 192;        // warp 0: TMA producer, warp 1: MMA issue + TMEM, warps 2..5: dequant/epilogue
+constexpr int kUmmaDequantWarps = 4;
+constexpr int kUmmaAStages = 4;          // A-operand ring in TMEM, 32 columns (one K64 block) per stage
+constexpr int kUmmaBlockK = 64;
+constexpr int kUmmaWBlockBytes = 4096;   // packed weights of one K64 block of a panel
+
+// ---- tcgen05 wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync()
+{
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after_sync()
+{
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// arrives on the mbarrier once every tcgen05 operation issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]; M, N and the operand types come from idesc
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 columns of 32 bits: thread t of the warp writes / reads lane (base + t), register i <-> column i
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,"
+        "%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what a tensor-map load with SWIZZLE_128B writes): groups of 8 rows are 1024
+// bytes apart (stride byte offset), the leading byte offset is unused for swizzled K-major tiles.
+__device__ __forceinline__ uint64_t umma_desc_k_major_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address, bits 0..13
+    d |= (uint64_t)1 << 16;                                // leading byte offset (ignored), bits 16..29
+    d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset, bits 32..45
+    d |= (uint64_t)1 << 46;                                // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                                // layout type: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: fp16 A and B, both K-major, fp32 accumulator, MMA shape M x N (K = 16).
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N)
+{
+    return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct UmmaArgs {
+    const uint8_t *scales;  // tiled
+    const uint8_t *qzeros;  // tiled
+    __half *y;              // [M, N]
+    int M, N, K, G;
+    int stages;             // shared-memory ring depth
+};
+
+__host__ __device__ constexpr int umma_stage_bytes(int TOK)
+{
+    return (TOK * 128 + kUmmaWBlockBytes + kItemSBytes + kItemZBytes + 1023) & ~1023;
+}
+__host__ __device__ constexpr int umma_tmem_cols(int TOK)
+{
+    // accumulator (TOK columns) + A ring, rounded up to a power of two >= 32
+    int need = TOK + kUmmaAStages * 32, c = 32;
+    while (c < need) c <<= 1;
+    return c;
+}
+
+template <int TOK>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
+{
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int kStage = umma_stage_bytes(TOK);
+    constexpr int kOffW = TOK * 128, kOffS = kOffW + kUmmaWBlockBytes, kOffZ = kOffS + kItemSBytes;
+    constexpr uint32_t kCols = umma_tmem_cols(TOK);
+    constexpr uint32_t kAcol = TOK;                        // first column of the A ring
+    constexpr int NA = kUmmaAStages;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 160;
+    const uint32_t bar_dfull = base + 192, tmem_slot = base + 200;
+    const uint32_t ring = base + 1024;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NS = a.stages;
+    const int panels = a.N / kPanel;
+    const int mt = blockIdx.x / panels, p = blockIdx.x - mt * panels;   // neighbours share the x tile
+    const int m0 = mt * TOK;
+    const int NB = a.K / kUmmaBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kUmmaDequantWarps + 1);   // dequant warps read W, the MMA reads x
+        }
+        for (int s = 0; s < NA; ++s) {
+            mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
+            mbar_init(bar_aempty + 8 * s, 1);
+        }
+        mbar_init(bar_dfull, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = lds32(tmem_slot);
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer (one thread)
+        if (lane == 0) {
+            tma_prefetch_descriptor(&w_map);
+            tma_prefetch_descriptor(&x_map);
+            auto issue_w = [&](int b, int s) {
+                const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
+                const bool first_of_group = (b & 1) == 0;
+                mbar_expect_tx(bar, kUmmaWBlockBytes + (first_of_group ? kItemSBytes + kItemZBytes : 0));
+                // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
+                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b) * 64, bar);
+                if (first_of_group) {
+                    const size_t t = (size_t)p * a.G + (b >> 1);
+                    bulk_g2s(st + kOffS, a.scales + t * kItemSBytes, kItemSBytes, bar);
+                    bulk_g2s(st + kOffZ, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
+                }
+            };
+            const int n_pre = NB < NS ? NB : NS;
+            for (int b = 0; b < n_pre; ++b) issue_w(b, b);   // weights do not depend on earlier kernels
+            pdl_wait();
+            int s = 0, round = 0;
+            for (int b = 0; b < NB; ++b) {
+                const uint32_t bar = bar_full + 8 * s;
+                if (b >= NS) {
+                    if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
+                    issue_w(b, s);
+                }
+                mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
+                tma_load_2d(ring + s * kStage, &x_map, b * kUmmaBlockK, m0, bar);
+                if (++s == NS) { s = 0; ++round; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issue (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_f16(128, TOK);
+            int s = 0, sa = 0;
+            uint32_t ph = 0, pha = 0;
+            bool ok = true;
+            for (int b = 0; b < NB && ok; ++b) {
+                ok = mbar_wait(bar_full + 8 * s, ph) && mbar_wait(bar_afull + 8 * sa, pha);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
+                    umma_f16_ts(tmem_base, tmem_base + kAcol + sa * 32 + kk * 8, bdesc + (uint64_t)(kk * 2), idesc,
+                                (uint32_t)((b | kk) != 0));
+                umma_commit(bar_empty + 8 * s);      // x tile of this stage may be overwritten
+                umma_commit(bar_aempty + 8 * sa);    // and so may this A stage
+                if (++s == NS) { s = 0; ph ^= 1u; }
+                if (++sa == NA) { sa = 0; pha ^= 1u; }
+            }
+            umma_commit(bar_dfull);
+        }
+    } else {
+        // ---------------------------------------------------------------- dequant warps, then epilogue
+        const int q = warp & 3;                 // the 32 TMEM lanes this warp may touch
+        const int n = 32 * q + lane;            // weight column inside the panel = TMEM lane
+        const int u = n >> 4, g = n & 7, h = (n >> 3) & 1;
+        // the column's 8 bytes (two words: rows +0..7 and +32..39) in each of the four 16-byte chunks
+        uint32_t w_rd[4];
+#pragma unroll
+        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
+        const uint32_t s_rd = kOffS + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + 8 * u + g;
+        constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
+        uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
+        int s = 0, sa = 0;
+        uint32_t ph = 0, pha = 0;
+        bool ok = true;
+        for (int b = 0; b < NB && ok; ++b) {
+            const uint32_t st = ring + s * kStage;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
+            if (!ok) break;
+            if ((b & 1) == 0) {
+                uint32_t sh;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
+                s2 = sh * 0x00010001u;
+                const uint32_t zb = lds8(st + z_rd);
+                const uint32_t z = h ? (zb >> 4) : (zb & 15u);
+                zlo = (z * 0x00010001u) | MAGIC_LO;
+                zhi = (z * 0x00100010u) | MAGIC_HI;
+            }
+            uint2 wv[4];
+#pragma unroll
+            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
+            uint32_t r[32];
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int t4 = 0; t4 < 4; ++t4) {
+                    uint32_t w = j ? wv[t4].y : wv[t4].x;        // rows 32 j + 8 t4 + (0..7), TMEM columns 16 j + 4 t4 + (0..3)
+                    uint32_t *o = r + 16 * j + 4 * t4;
+                    o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
+                    o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                    w >>= 8;
+                    o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
+                    o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                }
+            if (b >= NA) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1u));
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+            tmem_st_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + kAcol + sa * 32, r);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar_afull + 8 * sa);
+                mbar_arrive(bar_empty + 8 * s);
+            }
+            if (++s == NS) { s = 0; ph ^= 1u; }
+            if (++sa == NA) { sa = 0; pha ^= 1u; }
+        }
+        // ---- epilogue: lane n of the accumulator holds y[m0 .. m0+TOK, 128 p + n]
+        pdl_wait();
+        ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
+        if (ok) {
+            tc_fence_after_sync();
+            __half *yp = a.y + (size_t)p * kPanel + n;
+#pragma unroll 1
+            for (int c0 = 0; c0 < TOK; c0 += 32) {
+                if (m0 + c0 >= a.M) break;
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int m = m0 + c0 + i;
+                    if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kCols);
+    }
+}
+
+struct UmmaPlan {
+    int tok;        // tokens per CTA tile
+    int stages;
+    int ctas;       // panels * token tiles
+    int smem_bytes;
+};
+
+inline UmmaPlan plan_umma(int M, int N)
+{
+    UmmaPlan pl{};
+    pl.tok = 128;
+    pl.stages = 4;
+    pl.ctas = (N / kPanel) * ((M + pl.tok - 1) / pl.tok);
+    pl.smem_bytes = 2048 + pl.stages * umma_stage_bytes(pl.tok);
+    return pl;
+}
+
+template <int TOK>
+static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
+                           const UmmaPlan &plan, cudaStream_t s)
+{
+    static int configured_smem[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
+    if (configured_smem[dev] < plan.smem_bytes) {
+        e = cudaFuncSetAttribute(umma_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaFuncSetAttribute(umma_kernel<TOK>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        configured_smem[dev] = plan.smem_bytes;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)plan.ctas);
+    cfg.blockDim = dim3(kUmmaThreads);
+    cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, umma_kernel<TOK>, args, w_map, x_map));
+}
+
+int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
+                int K, const UmmaPlan &plan, cudaStream_t s)
+{
+    UmmaArgs args;
+    args.scales = (const uint8_t *)scales;
+    args.qzeros = (const uint8_t *)qzeros;
+    args.y = y;
+    args.M = M;
+    args.N = N;
+    args.K = K;
+    args.G = K / kGroup;
+    args.stages = plan.stages;
+    // packed weights as rows of 64 bytes (16 words); a box is one K64 block of a panel (64 rows)
+    CUtensorMap w_map, x_map;
+    const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
+    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 64,
+                                CU_TENSOR_MAP_SWIZZLE_64B);
+    if (st) return st;
+    // x as [M rows, K halves]; a box is 64 k of one token tile
+    st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
+                            (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.tok, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st) return st;
+    switch (plan.tok) {
+    case 128: return launch_umma_tok<128>(args, w_map, x_map, plan, s);
+    default: return GPTQ_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace gptq

@@ -95,7 +95,13 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     st, pl = B.gptq_plan(M, N, K, 128, 0, sms)
     assert st == B.GPTQ_OK
     G, panels = K // 128, N // 128
-    assert pl.kernel == 1 and pl.items == G * panels
+    assert pl.items == G * panels and pl.workspace_bytes == 0
+    if M > 64:                                # tcgen05 kernel: one launch, 128-token tiles, two CTAs per SM
+        assert pl.kernel == 2 and pl.m_tile == 128 and pl.m_chunks == 1 and pl.cluster_size == 1
+        assert pl.ctas == panels * -(-M // 128) and pl.split_panels == 0
+        assert 2 * (pl.smem_bytes + 1024) <= 227 * 1024 and pl.stages >= 2
+        return
+    assert pl.kernel == 1
     assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
     assert pl.ctas == panels * pl.cluster_size
     assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)

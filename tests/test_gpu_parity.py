@@ -28,14 +28,19 @@ def ws():
     return H.WorkspaceHolder()
 
 
-def assert_close(y_gpu: np.ndarray, y64: np.ndarray, K: int):
+def assert_close(y_gpu: np.ndarray, y64: np.ndarray, K: int, M: int | None = None):
+    """Stated tolerance always.  Up to 64 token rows the kernel multiplies exact integers q - z and applies the
+    scale in fp32, so it also meets the tighter derived bound; above that the tcgen05 kernel rounds each scaled
+    weight to fp16 once (relative 2^-11, about 1.4e-3 * sqrt(K/4096) rms on y for these inputs), which the stated
+    tolerance is there to cover."""
     y = y_gpu.astype(np.float64)
     err = np.abs(y - y64)
     loose = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64)
-    tight = 1e-4 * math.sqrt(K / 4096) + 2.0 ** -11 * np.abs(y64)
     assert np.all(np.isfinite(y))
     assert np.all(err <= loose), f"stated tolerance: {int((err > loose).sum())} violations, max err {err.max():.3e}"
-    assert np.all(err <= tight), f"implementation bound: {int((err > tight).sum())} violations, max err {err.max():.3e}"
+    if (y_gpu.shape[0] if M is None else M) <= 64:
+        tight = 1e-4 * math.sqrt(K / 4096) + 2.0 ** -11 * np.abs(y64)
+        assert np.all(err <= tight), f"implementation bound: {int((err > tight).sum())} violations, max err {err.max():.3e}"
 
 
 def run_gemm(L, x_np, ws):
@@ -233,7 +238,7 @@ def sampled_check(L, x, y, n_samples, seed):
     rows[:4] = [0, 0, M - 1, M - 1]
     cols[:4] = [0, L.N - 1, 0, L.N - 1]
     want = oracle.gemm_f64_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128, rows, cols)
-    assert_close(y[rows, cols], want, L.K)
+    assert_close(y[rows, cols], want, L.K, M)
 
 
 def test_config1_full_compare(ws):
