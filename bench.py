@@ -186,8 +186,21 @@ def step_bytes_flops(spec, layers):
 
 
 def launches_per_gemm(spec, M):
-    """Kernels one gptq_gemm call launches: one per 64-token chunk, plus the x gather with act-order."""
-    return (M + 63) // 64 + (1 if spec["act_order"] else 0)
+    """Kernels one gptq_gemm call launches: the matmul, plus the x gather with act-order."""
+    return 1 + (1 if spec["act_order"] else 0)
+
+
+def kernel_of(M):
+    """The kernel gptq_gemm dispatches to for M token rows (mirrors gptq_plan)."""
+    if M <= 8:
+        return "splitk_kernel<1>"
+    if M <= 16:
+        return "splitk_kernel<2>"
+    if M <= 32:
+        return "umma_kernel<32,2>"
+    if M <= 64:
+        return "umma_kernel<64,2>"
+    return "umma_kernel<128,4>"
 
 
 # ------------------------------------------------------------------------------------ reference arm
@@ -287,9 +300,12 @@ def main():
     ap.add_argument("--workload", default="decode7b", choices=list(WORKLOADS))
     ap.add_argument("--layers", type=int, default=0, help="distinct weight copies per shape (0 = workload default)")
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
+    ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    spec = WORKLOADS[args.workload]
+    spec = dict(WORKLOADS[args.workload])
+    if args.ms:
+        spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
     layers = args.layers or spec["layers"]
     if args.impl == "reference":
         run_reference(args, spec)
@@ -443,20 +459,14 @@ def main():
                 "TFLOP/s": round(flops_m[M] * args.steps / s / 1e12, 2),
                 "us_per_matmul": round(1e6 * s / args.steps / len(per_m[M]), 3),
             }
-        # dominant kernel: the streaming kernel instantiation that took most of the timed region
-        if spec["kind"] == "prefill":
-            dom_Ms = Ms
-            kname = "streamk_kernel<8>"
-        else:
-            groups = {}
-            for M in Ms:
-                tile = 8 if M <= 8 else 16 if M <= 16 else 32 if M <= 32 else 64
-                groups.setdefault(tile, []).append(M)
-            tile = max(groups, key=lambda t: sum(seg_ms[M] for M in groups[t]))
-            dom_Ms = groups[tile]
-            kname = f"streamk_kernel<{tile // 8}>"
+        # dominant kernel: the kernel instantiation that took most of the timed region
+        groups = {}
+        for M in Ms:
+            groups.setdefault(kernel_of(M), []).append(M)
+        kname = max(groups, key=lambda k: sum(seg_ms[M] for M in groups[k]))
+        dom_Ms = groups[kname]
         dom_s = sum(seg_ms[M] for M in dom_Ms) / 1e3
-        dom_launches = sum(((M + 63) // 64) * len(per_m[M]) for M in dom_Ms) * args.steps
+        dom_launches = sum(len(per_m[M]) for M in dom_Ms) * args.steps
         if spec["kind"] == "prefill":
             achieved = sum(flops_m[M] for M in dom_Ms) * args.steps / dom_s / 1e12
             peak, bound, runit = peaks["tflops_sustained"], "tensor", "TFLOP/s"

@@ -147,8 +147,8 @@ int gptq_check_status(void *stream);
 /* ---- host-only: how a problem would be launched (no CUDA call; usable without a GPU) -- */
 
 typedef struct {
-    int kernel;       /* 1 = cluster split-K mma.sync kernel (gptq_gemm, M <= 64),
-                         2 = tcgen05 kernel (gptq_gemm, M > 64),
+    int kernel;       /* 1 = cluster split-K mma.sync kernel (gptq_gemm, M <= 16),
+                         2 = tcgen05 kernel (gptq_gemm, M >= 17),
                          3 = stream-K mma.sync kernel (gptq_gemm_noalloc) */
     int m_tile;       /* tokens per CTA tile */
     int m_chunks;     /* launches along M */

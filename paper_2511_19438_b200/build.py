@@ -36,7 +36,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+    extra = os.environ.get("GPTQ_NVCC_EXTRA", "").split()      # e.g. -DGPTQ_UMMA_MIN_TOKENS=17
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

@@ -22,7 +22,11 @@ int record_cuda_error(cudaError_t e)
 
 constexpr int kMaxDevices = 64;
 constexpr size_t kTicketAreaBytes = 16384;   // 4096 panels
-constexpr int kStreamKMaxRows = 64;          // tokens per stream-K launch
+constexpr int kStreamKMaxRows = 64;          // tokens per mma.sync launch
+#ifndef GPTQ_UMMA_MIN_TOKENS
+#define GPTQ_UMMA_MIN_TOKENS 17
+#endif
+constexpr int kUmmaMinTokens = GPTQ_UMMA_MIN_TOKENS;   // from this many tokens on, gptq_gemm uses the tcgen05 kernel
 
 static Workspace g_workspace[kMaxDevices];
 static int g_sm_count[kMaxDevices];
@@ -174,8 +178,8 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     st = check_fast_path(N, K, group_size);
     if (st) return st;
     if (sm_count < 1) return GPTQ_ERR_SHAPE;
-    if (M > kStreamKMaxRows) {
-        const UmmaPlan up = plan_umma(M, N);
+    if (M >= kUmmaMinTokens) {
+        const UmmaPlan up = plan_umma(M, N, K, sm_count);
         out->kernel = 2;
         out->m_tile = up.tok;
         out->m_chunks = 1;
@@ -185,7 +189,8 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
         out->split_panels = 0;
         out->smem_bytes = up.smem_bytes;
         out->workspace_bytes = gemm_workspace_need(M, K, act_order);
-        out->cluster_size = 1;
+        out->cluster_size = up.S;
+        out->split_panels = up.S > 1 ? N / kPanel : 0;
         return GPTQ_OK;
     }
     const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
@@ -293,9 +298,9 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
         if (st) return st;
         xin = x_perm;
     }
-    if (M > kStreamKMaxRows) {
-        // many tokens: tcgen05 kernel, 128-token tiles
-        const UmmaPlan pl = plan_umma(M, N);
+    if (M >= kUmmaMinTokens) {
+        // tcgen05 kernel: 16- to 128-token tiles
+        const UmmaPlan pl = plan_umma(M, N, K, sms);
         return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, pl, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {

@@ -19,12 +19,12 @@
 #pragma once
 #include "gptq_common.cuh"
 #include "gptq_tma.cuh"
+#include "gptq_splitk.cuh"   // cluster barrier and distributed-shared-memory helpers
 
 namespace gptq {
 
 constexpr int kUmmaThreads = 192;        // warp 0: TMA producer, warp 1: MMA issue + TMEM, warps 2..5: dequant/epilogue
 constexpr int kUmmaDequantWarps = 4;
-constexpr int kUmmaAStages = 4;          // A-operand ring in TMEM, 32 columns (one K64 block) per stage
 constexpr int kUmmaBlockK = 64;
 constexpr int kUmmaWBlockBytes = 4096;   // packed weights of one K64 block of a panel
 
@@ -117,6 +117,7 @@ struct UmmaArgs {
     const uint8_t *qzeros;  // tiled
     __half *y;              // [M, N]
     int M, N, K, G;
+    int S;                  // CTAs that share one output tile along K (cluster size)
     int stages;             // shared-memory ring depth
 };
 
@@ -124,24 +125,23 @@ __host__ __device__ constexpr int umma_stage_bytes(int TOK)
 {
     return (TOK * 128 + kUmmaWBlockBytes + kItemSBytes + kItemZBytes + 1023) & ~1023;
 }
-__host__ __device__ constexpr int umma_tmem_cols(int TOK)
+__host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA)
 {
-    // accumulator (TOK columns) + A ring, rounded up to a power of two >= 32
-    int need = TOK + kUmmaAStages * 32, c = 32;
+    // accumulator (TOK columns) + A ring (32 columns = one K64 block per stage), a power of two >= 32
+    int need = TOK + NA * 32, c = 32;
     while (c < need) c <<= 1;
     return c;
 }
 
-template <int TOK>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+template <int TOK, int NA>
+__global__ void __launch_bounds__(kUmmaThreads, TOK <= 32 ? 3 : 2)
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
     constexpr int kStage = umma_stage_bytes(TOK);
     constexpr int kOffW = TOK * 128, kOffS = kOffW + kUmmaWBlockBytes, kOffZ = kOffS + kItemSBytes;
-    constexpr uint32_t kCols = umma_tmem_cols(TOK);
+    constexpr uint32_t kCols = umma_tmem_cols(TOK, NA);
     constexpr uint32_t kAcol = TOK;                        // first column of the A ring
-    constexpr int NA = kUmmaAStages;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 160;
@@ -150,9 +150,12 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NS = a.stages;
     const int panels = a.N / kPanel;
-    const int mt = blockIdx.x / panels, p = blockIdx.x - mt * panels;   // neighbours share the x tile
+    const int S = a.S;
+    const int tile = blockIdx.x / S, rank = blockIdx.x - tile * S;      // cluster = the S CTAs of one tile
+    const int mt = tile / panels, p = tile - mt * panels;               // neighbours share the x tile
     const int m0 = mt * TOK;
-    const int NB = a.K / kUmmaBlockK;
+    const int g0 = rank * a.G / S, g1 = (rank + 1) * a.G / S;           // this CTA's K groups
+    const int NB = 2 * (g1 - g0), b_first = 2 * g0;                     // its K64 blocks
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
@@ -187,9 +190,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 const bool first_of_group = (b & 1) == 0;
                 mbar_expect_tx(bar, kUmmaWBlockBytes + (first_of_group ? kItemSBytes + kItemZBytes : 0));
                 // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
-                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b) * 64, bar);
+                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
                 if (first_of_group) {
-                    const size_t t = (size_t)p * a.G + (b >> 1);
+                    const size_t t = (size_t)p * a.G + g0 + (b >> 1);
                     bulk_g2s(st + kOffS, a.scales + t * kItemSBytes, kItemSBytes, bar);
                     bulk_g2s(st + kOffZ, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
                 }
@@ -205,7 +208,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     issue_w(b, s);
                 }
                 mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
-                tma_load_2d(ring + s * kStage, &x_map, b * kUmmaBlockK, m0, bar);
+                tma_load_2d(ring + s * kStage, &x_map, (b_first + b) * kUmmaBlockK, m0, bar);
                 if (++s == NS) { s = 0; ++round; }
             }
         }
@@ -304,13 +307,46 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
                 tmem_wait_ld();
+                if (S == 1) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int m = m0 + c0 + i;
-                    if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i) {
+                        const int m = m0 + c0 + i;
+                        if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
+                    }
+                } else {
+                    // split-K: park the fp32 partial tile [token][column] at the start of the (idle) ring
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c0 + i < TOK) sts_f32(ring + (uint32_t)((c0 + i) * kPanel + n) * 4u, __uint_as_float(r[i]));
                 }
             }
         }
+    }
+    if (S > 1) {
+        // every CTA of the cluster has parked its tile; CTA `rank` finishes columns [c_lo, c_lo + width)
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (warp >= 2) {
+            const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
+            const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
+            for (int idx = threadIdx.x - 64; idx < rows * width; idx += kUmmaDequantWarps * 32) {
+                const int m = idx / width, cc = c_lo + idx - m * width;
+                const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
+                float v[8];
+#pragma unroll
+                for (int qq = 0; qq < 8; ++qq)
+                    v[qq] = qq < S ? ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)qq)) : 0.f;
+                float sum = 0.f;
+#pragma unroll
+                for (int qq = 0; qq < 8; ++qq) sum += v[qq];   // rank order
+                a.y[(size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc] = __float2half_rn(sum);
+            }
+        }
+        // no CTA may exit (and free its shared memory) while a peer can still read its tile
+        __syncwarp();
+        cluster_arrive_release();
+        cluster_wait_acquire();
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -321,19 +357,57 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
 }
 
 struct UmmaPlan {
-    int tok;        // tokens per CTA tile
+    int tok;        // tokens per CTA tile: 16, 32, 64 or 128
+    int S;          // CTAs per output tile along K (cluster size)
     int stages;
-    int ctas;       // panels * token tiles
+    int ctas;       // panels * token tiles * S
     int smem_bytes;
 };
 
-inline UmmaPlan plan_umma(int M, int N)
+__host__ __device__ constexpr int umma_a_stages(int tok) { return tok >= 128 ? 4 : 2; }
+// resident CTAs per SM: tensor memory (512 columns) and shared memory allow this many
+__host__ __device__ constexpr int umma_ctas_per_sm(int tok) { return tok <= 32 ? 3 : 2; }
+
+// Token tile by M; cluster size and shared-memory padding by the same rules as the mma.sync kernel:
+// the smallest estimated time among the S whose whole grid is resident at once, then padding so the
+// CTAs spread evenly over the SMs.
+inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
 {
     UmmaPlan pl{};
-    pl.tok = 128;
-    pl.stages = 4;
-    pl.ctas = (N / kPanel) * ((M + pl.tok - 1) / pl.tok);
-    pl.smem_bytes = 2048 + pl.stages * umma_stage_bytes(pl.tok);
+    const int tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
+    const int G = K / kGroup, tiles = (N / kPanel) * ((M + tok - 1) / tok);
+    const int stage = umma_stage_bytes(tok);
+    const int cps_max = umma_ctas_per_sm(tok);
+    int best_S = 1;
+    long long best_t = -1;
+    for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
+        for (int S = 1; S <= 8; S *= 2) {
+            if (S > G) break;
+            if (S > 1 && tok > 64) break;                      // the split-K epilogue handles tiles up to 64 tokens
+            const long long ctas = (long long)tiles * S, ipc = (G + S - 1) / S;
+            const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
+            if (pass == 0 && on_busiest_sm > cps_max) continue;
+            const long long serial = ipc * 45, shared = on_busiest_sm * ipc * 30;
+            const long long t = (serial > shared ? serial : shared) + (S > 1 ? 100 : 0);
+            if (best_t < 0 || t < best_t) { best_t = t; best_S = S; }
+        }
+    }
+    const int S = best_S;
+    const int blocks_per_cta = 2 * ((G + S - 1) / S);
+    int per_sm = (tiles * S + sm_count - 1) / sm_count;
+    if (per_sm > cps_max) per_sm = cps_max;
+    const int smem_cap = (227 * 1024) / per_sm - 1024;
+    const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;
+    int stages = (smem_cap - 2048) / stage;
+    if (stages > 8) stages = 8;
+    if (stages > blocks_per_cta) stages = blocks_per_cta;
+    while (S > 1 && stages * stage < tok * kPanel * 4) ++stages;   // the ring doubles as the fp32 partial tile
+    pl.tok = tok;
+    pl.S = S;
+    pl.stages = stages;
+    pl.ctas = tiles * S;
+    pl.smem_bytes = 2048 + stages * stage;
+    if (pl.smem_bytes < smem_floor) pl.smem_bytes = smem_floor;
     return pl;
 }
 
@@ -341,16 +415,16 @@ template <int TOK>
 static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
                            const UmmaPlan &plan, cudaStream_t s)
 {
+    auto kernel = umma_kernel<TOK, umma_a_stages(TOK)>;
     static int configured_smem[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
     if (configured_smem[dev] < plan.smem_bytes) {
-        e = cudaFuncSetAttribute(umma_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(umma_kernel<TOK>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return record_cuda_error(e);
         configured_smem[dev] = plan.smem_bytes;
     }
@@ -359,12 +433,16 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
     cfg.blockDim = dim3(kUmmaThreads);
     cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)plan.S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return record_cuda_error(cudaLaunchKernelEx(&cfg, umma_kernel<TOK>, args, w_map, x_map));
+    cfg.numAttrs = 2;
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, kernel, args, w_map, x_map));
 }
 
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
@@ -378,6 +456,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.N = N;
     args.K = K;
     args.G = K / kGroup;
+    args.S = plan.S;
     args.stages = plan.stages;
     // packed weights as rows of 64 bytes (16 words); a box is one K64 block of a panel (64 rows)
     CUtensorMap w_map, x_map;
@@ -390,6 +469,9 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
                             (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.tok, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st) return st;
     switch (plan.tok) {
+    case 16: return launch_umma_tok<16>(args, w_map, x_map, plan, s);
+    case 32: return launch_umma_tok<32>(args, w_map, x_map, plan, s);
+    case 64: return launch_umma_tok<64>(args, w_map, x_map, plan, s);
     case 128: return launch_umma_tok<128>(args, w_map, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }

@@ -96,11 +96,19 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     assert st == B.GPTQ_OK
     G, panels = K // 128, N // 128
     assert pl.items == G * panels and pl.workspace_bytes == 0
-    if M > 64:                                # tcgen05 kernel: one launch, 128-token tiles, two CTAs per SM
-        assert pl.kernel == 2 and pl.m_tile == 128 and pl.m_chunks == 1 and pl.cluster_size == 1
-        assert pl.ctas == panels * -(-M // 128) and pl.split_panels == 0
-        assert 2 * (pl.smem_bytes + 1024) <= 227 * 1024 and pl.stages >= 2
+    if pl.kernel == 2:                        # tcgen05 kernel: one launch, 16- to 128-token tiles
+        tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128
+        assert pl.m_tile == tok and pl.m_chunks == 1
+        assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G and (tok <= 64 or pl.cluster_size == 1)
+        assert pl.ctas == panels * -(-M // tok) * pl.cluster_size
+        assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
+        per_sm = min(-(-pl.ctas // sms), 3 if tok <= 32 else 2)
+        assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024 and pl.stages >= 2
+        assert (per_sm + 1) * (pl.smem_bytes + 1024) > 227 * 1024
+        if pl.cluster_size > 1:               # the ring doubles as the fp32 partial tile
+            assert pl.smem_bytes - 2048 >= tok * 128 * 4
         return
+    assert M <= 16
     assert pl.kernel == 1
     assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
     assert pl.ctas == panels * pl.cluster_size
