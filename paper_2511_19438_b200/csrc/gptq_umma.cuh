@@ -23,8 +23,10 @@
 
 namespace gptq {
 
-constexpr int kUmmaThreads = 192;        // warp 0: TMA producer, warp 1: MMA issue + TMEM, warps 2..5: dequant/epilogue
-constexpr int kUmmaDequantWarps = 4;
+// warp 0: TMA producer, warp 1: MMA issue + TMEM, then four dequant/epilogue warps per panel of the CTA
+// (two sets of them, taking alternate K64 blocks, when one warp per scheduler cannot keep up with the MMA)
+__host__ __device__ constexpr int umma_threads(int NP, int SETS) { return 64 + 128 * NP * SETS; }
+constexpr int kUmmaDequantWarps = 4;     // per panel: one warp per 32 TMEM lanes
 constexpr int kUmmaBlockK = 64;
 constexpr int kUmmaWBlockBytes = 4096;   // packed weights of one K64 block of a panel
 
@@ -121,38 +123,40 @@ struct UmmaArgs {
     int stages;             // shared-memory ring depth
 };
 
-__host__ __device__ constexpr int umma_stage_bytes(int TOK)
+__host__ __device__ constexpr int umma_stage_bytes(int TOK, int NP)
 {
-    return (TOK * 128 + kUmmaWBlockBytes + kItemSBytes + kItemZBytes + 1023) & ~1023;
+    return (TOK * 128 + NP * (kUmmaWBlockBytes + kItemSBytes + kItemZBytes) + 1023) & ~1023;
 }
-__host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA)
+__host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP)
 {
-    // accumulator (TOK columns) + A ring (32 columns = one K64 block per stage), a power of two >= 32
-    int need = TOK + NA * 32, c = 32;
+    // per panel: accumulator (TOK columns) + A ring (32 columns = one K64 block per stage); a power of two >= 32
+    int need = NP * (TOK + NA * 32), c = 32;
     while (c < need) c <<= 1;
     return c;
 }
 
-template <int TOK, int NA>
-__global__ void __launch_bounds__(kUmmaThreads, TOK <= 32 ? 3 : 2)
+template <int TOK, int NA, int NP, int SETS>
+__global__ void __launch_bounds__(umma_threads(NP, SETS), (NP > 1 || TOK > 128) ? 1 : TOK <= 32 ? 3 : 2)
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
-    constexpr int kStage = umma_stage_bytes(TOK);
-    constexpr int kOffW = TOK * 128, kOffS = kOffW + kUmmaWBlockBytes, kOffZ = kOffS + kItemSBytes;
-    constexpr uint32_t kCols = umma_tmem_cols(TOK, NA);
-    constexpr uint32_t kAcol = TOK;                        // first column of the A ring
+    constexpr int kStage = umma_stage_bytes(TOK, NP);
+    // stage: [x tile][W block of each panel][scales of each panel][zeros of each panel]
+    constexpr int kOffW = TOK * 128, kOffS = kOffW + NP * kUmmaWBlockBytes, kOffZ = kOffS + NP * kItemSBytes;
+    constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP);
+    constexpr uint32_t kAcol = NP * TOK;                   // accumulators first, then the A rings (panel-major)
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 160;
-    const uint32_t bar_dfull = base + 192, tmem_slot = base + 200;
+    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 192;
+    const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
     const uint32_t ring = base + 1024;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NS = a.stages;
     const int panels = a.N / kPanel;
     const int S = a.S;
     const int tile = blockIdx.x / S, rank = blockIdx.x - tile * S;      // cluster = the S CTAs of one tile
-    const int mt = tile / panels, p = tile - mt * panels;               // neighbours share the x tile
+    const int ptiles = panels / NP;
+    const int mt = tile / ptiles, p0 = (tile - mt * ptiles) * NP;       // first panel; neighbours share the x tile
     const int m0 = mt * TOK;
     const int g0 = rank * a.G / S, g1 = (rank + 1) * a.G / S;           // this CTA's K groups
     const int NB = 2 * (g1 - g0), b_first = 2 * g0;                     // its K64 blocks
@@ -160,9 +164,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, kUmmaDequantWarps + 1);   // dequant warps read W, the MMA reads x
+            mbar_init(bar_empty + 8 * s, NP * kUmmaDequantWarps + 1);   // dequant warps read W, the MMA reads x
         }
-        for (int s = 0; s < NA; ++s) {
+        for (int s = 0; s < NP * NA; ++s) {
             mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
             mbar_init(bar_aempty + 8 * s, 1);
         }
@@ -187,14 +191,16 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             tma_prefetch_descriptor(&x_map);
             auto issue_w = [&](int b, int s) {
                 const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
-                const bool first_of_group = (b & 1) == 0;
-                mbar_expect_tx(bar, kUmmaWBlockBytes + (first_of_group ? kItemSBytes + kItemZBytes : 0));
-                // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
-                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
-                if (first_of_group) {
+                mbar_expect_tx(bar, NP * (kUmmaWBlockBytes + kItemSBytes + kItemZBytes));
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    const int p = p0 + j;
+                    // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
+                    tma_load_2d(st + kOffW + j * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
+                    // the group's scales and zeros travel with both of its blocks (320 bytes)
                     const size_t t = (size_t)p * a.G + g0 + (b >> 1);
-                    bulk_g2s(st + kOffS, a.scales + t * kItemSBytes, kItemSBytes, bar);
-                    bulk_g2s(st + kOffZ, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
+                    bulk_g2s(st + kOffS + j * kItemSBytes, a.scales + t * kItemSBytes, kItemSBytes, bar);
+                    bulk_g2s(st + kOffZ + j * kItemZBytes, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
                 }
             };
             const int n_pre = NB < NS ? NB : NS;
@@ -220,16 +226,22 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             uint32_t ph = 0, pha = 0;
             bool ok = true;
             for (int b = 0; b < NB && ok; ++b) {
-                ok = mbar_wait(bar_full + 8 * s, ph) && mbar_wait(bar_afull + 8 * sa, pha);
+                ok = mbar_wait(bar_full + 8 * s, ph);
                 if (!ok) break;
-                tc_fence_after_sync();
                 const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
-                    umma_f16_ts(tmem_base, tmem_base + kAcol + sa * 32 + kk * 8, bdesc + (uint64_t)(kk * 2), idesc,
-                                (uint32_t)((b | kk) != 0));
-                umma_commit(bar_empty + 8 * s);      // x tile of this stage may be overwritten
-                umma_commit(bar_aempty + 8 * sa);    // and so may this A stage
+                for (int j = 0; j < NP; ++j) {
+                    ok = mbar_wait(bar_afull + 8 * (j * NA + sa), pha);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
+                        umma_f16_ts(tmem_base + j * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
+                                    bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)((b | kk) != 0));
+                    umma_commit(bar_aempty + 8 * (j * NA + sa));   // this A stage may be overwritten
+                }
+                if (!ok) break;
+                umma_commit(bar_empty + 8 * s);      // and so may the x tile of this stage
                 if (++s == NS) { s = 0; ph ^= 1u; }
                 if (++sa == NA) { sa = 0; pha ^= 1u; }
             }
@@ -238,41 +250,40 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     } else {
         // ---------------------------------------------------------------- dequant warps, then epilogue
         const int q = warp & 3;                 // the 32 TMEM lanes this warp may touch
+        const int j = ((warp - 2) >> 2) % NP;   // which of the CTA's panels this warp dequantises
+        const int set = ((warp - 2) >> 2) / NP; // and which K64 blocks: set, set + SETS, ...
+        const int p = p0 + j;
         const int n = 32 * q + lane;            // weight column inside the panel = TMEM lane
         const int u = n >> 4, g = n & 7, h = (n >> 3) & 1;
         // the column's 8 bytes (two words: rows +0..7 and +32..39) in each of the four 16-byte chunks
         uint32_t w_rd[4];
 #pragma unroll
-        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
-        const uint32_t s_rd = kOffS + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + 8 * u + g;
+        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + j * kUmmaWBlockBytes + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
+        const uint32_t s_rd = kOffS + j * kItemSBytes + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + j * kItemZBytes + 8 * u + g;
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-        uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
-        int s = 0, sa = 0;
-        uint32_t ph = 0, pha = 0;
+        int s = set % NS, sa = set % NA;
+        uint32_t ph = (uint32_t)(set / NS) & 1u, pha = (uint32_t)(set / NA) & 1u;
         bool ok = true;
-        for (int b = 0; b < NB && ok; ++b) {
+        for (int b = set; b < NB && ok; b += SETS) {
             const uint32_t st = ring + s * kStage;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
             if (!ok) break;
-            if ((b & 1) == 0) {
-                uint32_t sh;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
-                s2 = sh * 0x00010001u;
-                const uint32_t zb = lds8(st + z_rd);
-                const uint32_t z = h ? (zb >> 4) : (zb & 15u);
-                zlo = (z * 0x00010001u) | MAGIC_LO;
-                zhi = (z * 0x00100010u) | MAGIC_HI;
-            }
+            uint32_t sh;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
+            const uint32_t s2 = sh * 0x00010001u;
+            const uint32_t zb = lds8(st + z_rd);
+            const uint32_t z = h ? (zb >> 4) : (zb & 15u);
+            const uint32_t zlo = (z * 0x00010001u) | MAGIC_LO, zhi = (z * 0x00100010u) | MAGIC_HI;
             uint2 wv[4];
 #pragma unroll
             for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
             uint32_t r[32];
 #pragma unroll
-            for (int j = 0; j < 2; ++j)
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int t4 = 0; t4 < 4; ++t4) {
-                    uint32_t w = j ? wv[t4].y : wv[t4].x;        // rows 32 j + 8 t4 + (0..7), TMEM columns 16 j + 4 t4 + (0..3)
-                    uint32_t *o = r + 16 * j + 4 * t4;
+                    uint32_t w = jj ? wv[t4].y : wv[t4].x;       // rows 32 jj + 8 t4 + (0..7), TMEM columns 16 jj + 4 t4 + (0..3)
+                    uint32_t *o = r + 16 * jj + 4 * t4;
                     o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
                     o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
                     w >>= 8;
@@ -280,20 +291,22 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
                 }
             if (b >= NA) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1u));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * (j * NA + sa), pha ^ 1u));
                 if (!ok) break;
                 tc_fence_after_sync();
             }
-            tmem_st_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + kAcol + sa * 32, r);
+            tmem_st_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + kAcol + (j * NA + sa) * 32, r);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(bar_afull + 8 * sa);
+                mbar_arrive(bar_afull + 8 * (j * NA + sa));
                 mbar_arrive(bar_empty + 8 * s);
             }
-            if (++s == NS) { s = 0; ph ^= 1u; }
-            if (++sa == NA) { sa = 0; pha ^= 1u; }
+            s += SETS;
+            if (s >= NS) { s -= NS; ph ^= 1u; }
+            sa += SETS;
+            if (sa >= NA) { sa -= NA; pha ^= 1u; }
         }
         // ---- epilogue: lane n of the accumulator holds y[m0 .. m0+TOK, 128 p + n]
         pdl_wait();
@@ -304,8 +317,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
 #pragma unroll 1
             for (int c0 = 0; c0 < TOK; c0 += 32) {
                 if (m0 + c0 >= a.M) break;
+                if (SETS > 1 && ((c0 >> 5) % SETS) != set) continue;   // the warp sets share the token chunks
                 uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
+                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + j * TOK + c0, r);
                 tmem_wait_ld();
                 if (S == 1) {
 #pragma unroll
@@ -328,9 +342,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         cluster_arrive_release();
         cluster_wait_acquire();
         if (warp >= 2) {
+            const int p = p0;   // split-K runs with one panel per CTA
             const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
             const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
-            for (int idx = threadIdx.x - 64; idx < rows * width; idx += kUmmaDequantWarps * 32) {
+            for (int idx = threadIdx.x - 64; idx < rows * width; idx += 128) {
                 const int m = idx / width, cc = c_lo + idx - m * width;
                 const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
                 float v[8];
@@ -357,27 +372,33 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
 }
 
 struct UmmaPlan {
-    int tok;        // tokens per CTA tile: 16, 32, 64 or 128
+    int tok;        // tokens per CTA tile: 16, 32, 64, 128 or 256
+    int np;         // 128-column panels per CTA
+    int sets;       // dequant warp sets per panel
     int S;          // CTAs per output tile along K (cluster size)
     int stages;
-    int ctas;       // panels * token tiles * S
+    int ctas;       // panel tiles * token tiles * S
     int smem_bytes;
 };
 
-__host__ __device__ constexpr int umma_a_stages(int tok) { return tok >= 128 ? 4 : 2; }
+// A-ring depth per panel: with two panels the 512 tensor-memory columns hold exactly 2 x (128 + 4 x 32)
+__host__ __device__ constexpr int umma_a_stages(int tok, int np) { return tok >= 128 ? 4 : 2; }
 // resident CTAs per SM: tensor memory (512 columns) and shared memory allow this many
-__host__ __device__ constexpr int umma_ctas_per_sm(int tok) { return tok <= 32 ? 3 : 2; }
+__host__ __device__ constexpr int umma_ctas_per_sm(int tok, int np) { return (np > 1 || tok > 128) ? 1 : tok <= 32 ? 3 : 2; }
 
-// Token tile by M; cluster size and shared-memory padding by the same rules as the mma.sync kernel:
-// the smallest estimated time among the S whose whole grid is resident at once, then padding so the
-// CTAs spread evenly over the SMs.
+// Token tile by M (256 tokens from M = 256 up: one dequantised block then feeds twice the MMA work);
+// cluster size and shared-memory padding by the same rules as the mma.sync kernel.  Two panels per CTA
+// (np = 2) halve the x traffic per flop but allow only one CTA per SM and measured slower, so np = 1.
 inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
 {
     UmmaPlan pl{};
-    const int tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
-    const int G = K / kGroup, tiles = (N / kPanel) * ((M + tok - 1) / tok);
-    const int stage = umma_stage_bytes(tok);
-    const int cps_max = umma_ctas_per_sm(tok);
+    const int tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M < 256 ? 128 : 256;
+    const int panels = N / kPanel;
+    const int np = 1;
+    const int sets = tok >= 128 ? 2 : 1;
+    const int G = K / kGroup, tiles = (panels / np) * ((M + tok - 1) / tok);
+    const int stage = umma_stage_bytes(tok, np);
+    const int cps_max = umma_ctas_per_sm(tok, np);
     int best_S = 1;
     long long best_t = -1;
     for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
@@ -403,6 +424,8 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     if (stages > blocks_per_cta) stages = blocks_per_cta;
     while (S > 1 && stages * stage < tok * kPanel * 4) ++stages;   // the ring doubles as the fp32 partial tile
     pl.tok = tok;
+    pl.np = np;
+    pl.sets = sets;
     pl.S = S;
     pl.stages = stages;
     pl.ctas = tiles * S;
@@ -411,11 +434,11 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     return pl;
 }
 
-template <int TOK>
+template <int TOK, int NP, int SETS>
 static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
                            const UmmaPlan &plan, cudaStream_t s)
 {
-    auto kernel = umma_kernel<TOK, umma_a_stages(TOK)>;
+    auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS>;
     static int configured_smem[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -430,7 +453,7 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
-    cfg.blockDim = dim3(kUmmaThreads);
+    cfg.blockDim = dim3(umma_threads(NP, SETS));
     cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
@@ -469,10 +492,11 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
                             (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.tok, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st) return st;
     switch (plan.tok) {
-    case 16: return launch_umma_tok<16>(args, w_map, x_map, plan, s);
-    case 32: return launch_umma_tok<32>(args, w_map, x_map, plan, s);
-    case 64: return launch_umma_tok<64>(args, w_map, x_map, plan, s);
-    case 128: return launch_umma_tok<128>(args, w_map, x_map, plan, s);
+    case 16: return launch_umma_tok<16, 1, 1>(args, w_map, x_map, plan, s);
+    case 32: return launch_umma_tok<32, 1, 1>(args, w_map, x_map, plan, s);
+    case 64: return launch_umma_tok<64, 1, 1>(args, w_map, x_map, plan, s);
+    case 128: return launch_umma_tok<128, 1, 2>(args, w_map, x_map, plan, s);
+    case 256: return launch_umma_tok<256, 1, 2>(args, w_map, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }

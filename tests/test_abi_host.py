@@ -89,7 +89,7 @@ SHAPES = list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()) + [(128, 128
 
 
 @pytest.mark.parametrize("K,N", SHAPES)
-@pytest.mark.parametrize("M", [1, 8, 9, 16, 33, 64, 200])
+@pytest.mark.parametrize("M", [1, 8, 9, 16, 33, 64, 200, 1000])
 @pytest.mark.parametrize("sms", [148, 132, 7])
 def test_cluster_plan_is_consistent(K, N, M, sms):
     st, pl = B.gptq_plan(M, N, K, 128, 0, sms)
@@ -97,12 +97,12 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     G, panels = K // 128, N // 128
     assert pl.items == G * panels and pl.workspace_bytes == 0
     if pl.kernel == 2:                        # tcgen05 kernel: one launch, 16- to 128-token tiles
-        tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128
+        tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M < 256 else 256
         assert pl.m_tile == tok and pl.m_chunks == 1
         assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G and (tok <= 64 or pl.cluster_size == 1)
         assert pl.ctas == panels * -(-M // tok) * pl.cluster_size
         assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
-        per_sm = min(-(-pl.ctas // sms), 3 if tok <= 32 else 2)
+        per_sm = min(-(-pl.ctas // sms), 1 if tok > 128 else 3 if tok <= 32 else 2)
         assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024 and pl.stages >= 2
         assert (per_sm + 1) * (pl.smem_bytes + 1024) > 227 * 1024
         if pl.cluster_size > 1:               # the ring doubles as the fp32 partial tile
