@@ -40,9 +40,14 @@ NOMINAL_FP16_TFLOPS = 2250.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_TFLOPS = 1590.0
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture, keyed by kernel name, with
-# the digest of the kernel sources they were taken on; reported as null once the sources change.
-NCU_TRAFFIC = {}
+# DRAM traffic of the dominant kernels from ncu captures (profiles/), as measured bytes over
+# algorithmic bytes of the captured launches, with the digest of the kernel sources they were taken
+# on (`--print-digest`); `traffic` is that ratio times the timed launches' algorithmic bytes, and
+# null once the sources have changed since the capture.
+NCU_TRAFFIC = {
+    "splitk_kernel<1>": {"digest": "PENDING", "ratio": 1.0004},      # M = 1, the four 7B shapes
+    "umma_kernel<256,4,1,2>": {"digest": "PENDING", "ratio": 0.678},  # qkv, M = 2048 (y still in L2 at kernel end)
+}
 
 WORKLOADS = {
     "decode7b": dict(shapes=wl.SHAPES_7B, Ms=wl.DECODE_M, act_order=False, layers=8, kind="decode",
@@ -197,10 +202,12 @@ def kernel_of(M):
     if M <= 16:
         return "splitk_kernel<2>"
     if M <= 32:
-        return "umma_kernel<32,2>"
+        return "umma_kernel<32,2,1,1>"
     if M <= 64:
-        return "umma_kernel<64,2>"
-    return "umma_kernel<128,4>"
+        return "umma_kernel<64,2,1,1>"
+    if M < 256:
+        return "umma_kernel<128,4,1,2>"
+    return "umma_kernel<256,4,1,2>"
 
 
 # ------------------------------------------------------------------------------------ reference arm
@@ -302,7 +309,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
     ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--print-digest", action="store_true", help="print the kernel-source digest and exit")
     args = ap.parse_args()
+    if args.print_digest:
+        print(kernel_source_digest())
+        return
     spec = dict(WORKLOADS[args.workload])
     if args.ms:
         spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
@@ -477,7 +488,7 @@ def main():
         traffic = None
         t = NCU_TRAFFIC.get(kname)
         if t and t.get("digest") == digest:
-            traffic = t["bytes_per_launch"]
+            traffic = round(t["ratio"] * sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_launches)
         roofline = {
             "bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": runit,
             "frac": round(achieved / peak, 4), "traffic": traffic, "kernel": kname, "peak_source": peaks["source"],

@@ -7,11 +7,13 @@
  * 4-bit GPTQ weights inside every linear layer of the served model; Section 4.2: fp16
  * activations and fp16 weights after dequantisation).  The paper's three kernel-level
  * ideas map onto this library as follows: vectorised loads (Section 3.2, Algorithm 2)
- * become 16-byte-granular bulk copies of re-tiled weights; native packed-half arithmetic
- * (Section 3.3, Algorithm 3) becomes lop3/sub.f16x2 dequantisation feeding tensor-core
- * MMAs; block-level pre-reduction with one committing thread (Section 3.1, Algorithm 1)
- * becomes an fp32 partial-tile workspace reduced in a fixed order by the last-arriving
- * block, with one plain fp16 store and no global atomics on the output.
+ * become 16-byte-granular bulk and tensor-map (TMA) copies of re-tiled weights and of the
+ * activation tiles; native packed-half arithmetic (Section 3.3, Algorithm 3) becomes
+ * lop3 / sub.f16x2 / mul.f16x2 dequantisation feeding tensor-core MMAs (mma.sync for up to 16
+ * token rows, tcgen05 with the dequantised operand in tensor memory above that); block-level
+ * pre-reduction with one committing thread (Section 3.1, Algorithm 1) becomes split-K inside a
+ * thread-block cluster, reduced through distributed shared memory in a fixed order, with one
+ * plain fp16 store and no atomics on the output.
  *
  * Storage format ("canonical", what checkpoints hold):
  *   qweight int32[K/8, N]  nibble i (bits 4i..4i+3, word read as unsigned) of word (r,n)
@@ -100,7 +102,9 @@ int gptq_set_workspace(void *ptr, size_t bytes, void *stream);
 
 /* y fp16[M,N] = x fp16[M,K] . dequant(W).  qweight/qzeros/scales are the REPACKED buffers from
  * gptq_repack; with act_order != 0, g_idx is gptq_repack's perm_out (else it may be NULL).
- * fp32 accumulation, one round-to-nearest-even conversion to fp16.  Any M >= 1.
+ * fp32 accumulation, one round-to-nearest-even conversion to fp16.  Any M >= 1.  Up to 16 rows the
+ * weights enter the MMA as exact integers q - z and the scale multiplies fp32 group sums; above
+ * that each scaled weight is rounded to fp16 once before the MMA.
  * The kernels begin fetching weights before earlier work on the stream has finished
  * (programmatic dependent launch); x, y and the workspace are only touched afterwards.  The
  * weight buffers must therefore not be written by a kernel launched immediately before this
