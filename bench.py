@@ -275,7 +275,7 @@ def run_reference(args, spec):
         return
     import oracle
     oracle.build()
-    items, text = oracle_sample(spec, budget_s=min(12.0, 150.0 / max(args.steps + min(args.warmup, 1), 1)))
+    items, text = oracle_sample(spec, budget_s=min(12.0, args.ref_budget / max(args.steps + min(args.warmup, 1), 1)))
     for _ in range(min(args.warmup, 1)):
         run_oracle_once(items, spec)
     total = 0.0
@@ -297,6 +297,23 @@ def run_reference(args, spec):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------ replicas
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise maximum over all ranks of a list of per-rank times (a collective when world > 1)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(spec, world, step_bytes, step_flops, steps, slowest_ms):
+    """Replicas only: every rank runs the same workload on its own GPU, so the job processed
+    world x the units of one rank in the time of the slowest rank."""
+    return world * to_metric(spec, step_bytes * steps, step_flops * steps, slowest_ms / 1e3)
+
+
 # ------------------------------------------------------------------------------------ product arm
 def main():
     ap = argparse.ArgumentParser()
@@ -309,6 +326,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
     ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-budget", type=float, default=150.0,
+                    help="--impl reference: seconds of CPU time the whole run should take (sizes the per-step sample)")
     ap.add_argument("--print-digest", action="store_true", help="print the kernel-source digest and exit")
     args = ap.parse_args()
     if args.print_digest:
@@ -447,10 +466,7 @@ def main():
     sampler.stop()
 
     # ---- reduce over ranks (max time), aggregate over replicas
-    times = torch.tensor([total_ms, e2e_ms] + [seg_ms[M] for M in Ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    times = times.tolist()
+    times = max_over_ranks([total_ms, e2e_ms] + [seg_ms[M] for M in Ms], world, device)
     total_ms, e2e_ms = times[0], times[1]
     seg_ms = {M: times[2 + i] for i, M in enumerate(Ms)}
 
@@ -458,9 +474,8 @@ def main():
         peaks = measured_peaks()
         metric, unit = metric_of(spec)
         step_bytes, step_flops = sum(bytes_m.values()), sum(flops_m.values())
-        sec = total_ms / 1e3
-        value = world * to_metric(spec, step_bytes * args.steps, step_flops * args.steps, sec)
-        e2e_value = world * to_metric(spec, step_bytes * e2e_steps, step_flops * e2e_steps, e2e_ms / 1e3)
+        value = whole_job_value(spec, world, step_bytes, step_flops, args.steps, total_ms)
+        e2e_value = whole_job_value(spec, world, step_bytes, step_flops, e2e_steps, e2e_ms)
         launches_step = sum(launches_per_gemm(spec, M) * len(per_m[M]) for M in Ms)
         per_m_report = {}
         for M in Ms:

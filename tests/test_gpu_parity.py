@@ -126,7 +126,34 @@ def test_gemm_small_full_compare(K, N, M, act, ws):
     assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
 
 
-@pytest.mark.parametrize("M", [1, 7, 16, 24, 64])
+@pytest.mark.parametrize("M", [15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 300, 513])
+@pytest.mark.parametrize("act", [False, True])
+def test_gemm_token_count_boundaries(M, act, ws):
+    """Every switch of kernel, token tile and cluster size along M, with a ragged last tile."""
+    K, N = (1024, 384) if not act else (640, 256)
+    L = wl.make_linear(K, N, seed=wl.seed_for("edge", K, N, act), act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("edge-x", K, M))
+    y, _ = run_gemm(L, x, ws)
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+
+
+def test_gemm_leaves_rows_beyond_m_alone(ws):
+    """The last token tile is ragged: rows past M of the output buffer must not be written."""
+    K, N = 512, 256
+    L = wl.make_linear(K, N, seed=wl.seed_for("guard", K, N))
+    D = H.upload_and_repack(L)
+    for M in (20, 70, 130, 260):
+        guard = torch.full((M + 3, N), 7.0, dtype=torch.float16, device="cuda")
+        x = H.to_device(wl.make_x(M, K, wl.seed_for("guard-x", M)))
+        ws.ensure_for(M, D)
+        H.gemm(x, D, guard[1:M + 1])
+        torch.cuda.synchronize()
+        assert torch.all(guard[0] == 7.0) and torch.all(guard[M + 1:] == 7.0)
+        assert not torch.any(guard[1:M + 1] == 7.0)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+@pytest.mark.parametrize("M", [1, 7, 16, 24, 64, 200])
 def test_gemm_integer_case_is_exact(M, ws):
     """z = 8, s = 1, small-integer x: every product and partial sum is an integer below 2^24, so
     any summation order gives the exact result, and it is exact in fp16 wherever |y| <= 2048."""
