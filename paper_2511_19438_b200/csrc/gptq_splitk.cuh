@@ -284,7 +284,7 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
     long long best_t = -1;
     for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
         for (int S = 1; S <= 8; S *= 2) {
-            if (S > G) break;
+            if (S > G || (pass == 1 && S > 1)) break;          // nothing fits at once: several waves, no split
             const long long ctas = (long long)panels * S, ipc = (G + S - 1) / S;
             const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
             if (pass == 0 && on_busiest_sm > cps_max) continue;

@@ -342,10 +342,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         cluster_arrive_release();
         cluster_wait_acquire();
         if (warp >= 2) {
-            const int p = p0;   // split-K runs with one panel per CTA
+            const int p = p0;   // split-K runs with one panel per CTA (NP == 1)
             const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
             const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
-            for (int idx = threadIdx.x - 64; idx < rows * width; idx += 128) {
+            for (int idx = threadIdx.x - 64; idx < rows * width; idx += 128 * NP * SETS) {
                 const int m = idx / width, cc = c_lo + idx - m * width;
                 const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
                 float v[8];
@@ -403,8 +403,7 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     long long best_t = -1;
     for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
         for (int S = 1; S <= 8; S *= 2) {
-            if (S > G) break;
-            if (S > 1 && tok > 64) break;                      // the split-K epilogue handles tiles up to 64 tokens
+            if (S > G || (pass == 1 && S > 1)) break;          // nothing fits at once: several waves, no split
             const long long ctas = (long long)tiles * S, ipc = (G + S - 1) / S;
             const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
             if (pass == 0 && on_busiest_sm > cps_max) continue;

@@ -99,7 +99,7 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     if pl.kernel == 2:                        # tcgen05 kernel: one launch, 16- to 128-token tiles
         tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M < 256 else 256
         assert pl.m_tile == tok and pl.m_chunks == 1
-        assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G and (tok <= 64 or pl.cluster_size == 1)
+        assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
         assert pl.ctas == panels * -(-M // tok) * pl.cluster_size
         assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
         per_sm = min(-(-pl.ctas // sms), 1 if tok > 128 else 3 if tok <= 32 else 2)
