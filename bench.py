@@ -325,6 +325,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="distinct weight copies per shape (0 = workload default)")
     ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
     ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
+    ap.add_argument("--cta-pairs", action="store_true", help="prefill on CTA pairs (tcgen05 cta_group::2), off by default")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-budget", type=float, default=150.0,
                     help="--impl reference: seconds of CPU time the whole run should take (sizes the per-step sample)")
@@ -364,6 +365,8 @@ def main():
     from paper_2511_19438_b200 import binding as B
     from paper_2511_19438_b200 import harness as H
 
+    if args.cta_pairs:
+        B.check(B.gptq_set_cta_pairs(1), "gptq_set_cta_pairs")
     per_m, _host = build_problems(spec, layers, H, torch, device)
     ws = H.WorkspaceHolder(device)
     need = 0

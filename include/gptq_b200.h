@@ -113,6 +113,12 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
 
+/* Process-wide switch: with enable != 0, gptq_gemm runs problems with M >= 256 and an even number
+ * of 128-column panels on CTA pairs (tcgen05.mma.cta_group::2: two SMs share one 256 x 256 x 16 MMA and
+ * each loads half of the x tile).  Same arithmetic and tolerance as the default kernel; it halves the
+ * L2 traffic per flop but measured slower on the Llama shapes, so it is off by default. */
+int gptq_set_cta_pairs(int enable);
+
 /* The same product for callers whose activations live in host memory: copies x_host (pinned
  * for true asynchrony) to x_stage, runs gptq_gemm, copies y_stage to y_host, all on `stream`.
  * x_stage (M*K fp16) and y_stage (M*N fp16) are caller-owned device buffers. */

@@ -53,6 +53,7 @@ _SIGNATURES = {
     "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "gptq_set_workspace": (_i, [_vp, _sz, _vp]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_set_cta_pairs": (_i, [_i]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_noalloc_scratch_bytes": (_sz, []),
@@ -142,6 +143,10 @@ def gptq_set_workspace(ptr, nbytes, stream=None) -> int:
 def gptq_gemm(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
     return _lib.gptq_gemm(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N, K,
                           group_size, int(act_order), _stream(stream))
+
+
+def gptq_set_cta_pairs(enable) -> int:
+    return _lib.gptq_set_cta_pairs(int(bool(enable)))
 
 
 def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_stage, M, N, K, group_size,

@@ -5,6 +5,7 @@
 #include "gptq_streamk.cuh"
 #include "gptq_splitk.cuh"
 #include "gptq_umma.cuh"
+#include "gptq_umma2.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -12,6 +13,7 @@
 namespace gptq {
 
 static std::atomic<int> g_last_cuda_error{0};
+static std::atomic<int> g_use_cta_pairs{0};
 
 int record_cuda_error(cudaError_t e)
 {
@@ -115,6 +117,12 @@ const char *gptq_status_string(int status)
 }
 
 int gptq_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+int gptq_set_cta_pairs(int enable)
+{
+    g_use_cta_pairs.store(enable ? 1 : 0);
+    return GPTQ_OK;
+}
 
 int gptq_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out, int N, int K,
                    int group_size, void *stream)
@@ -299,7 +307,11 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
         xin = x_perm;
     }
     if (M >= kUmmaMinTokens) {
-        // tcgen05 kernel: 16- to 128-token tiles
+        if (g_use_cta_pairs.load() && umma2_applicable(M, N)) {
+            const Umma2Plan p2 = plan_umma2(M, N, K);
+            return launch_umma2(xin, qweight, qzeros, scales, (__half *)y, M, N, K, p2, s);
+        }
+        // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
         return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, pl, s);
     }

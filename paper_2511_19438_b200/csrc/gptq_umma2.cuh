@@ -1,0 +1,354 @@
+// Prefill GPTQ matmul on CTA pairs: the tcgen05 kernel of gptq_umma.cuh with cta_group::2.
+//
+// Two CTAs of a cluster (two SMs) share one MMA of shape 256 x 256 x 16: CTA r owns weight panel
+// 2 t + r (its 128 rows of the A operand, dequantised into its own tensor memory, and its 128 lanes
+// of the accumulator) and loads only tokens [128 r, 128 r + 128) of the 256-token x tile; the
+// tensor cores of the pair read both halves of the B operand from the two shared memories.  Per
+// flop this halves the x traffic from L2 to shared memory, which is what bounds the single-CTA
+// kernel, and halves the dequantisation work per MMA cycle.
+//
+// Synchronisation across the pair uses no multicast load: every CTA's TMA completes on its own
+// mbarriers; the dequant warps of both CTAs arrive (cluster scope) on the LEADER's a_full barrier
+// after they have waited for their own stage - so an arrival says "my A stage is in tensor memory
+// and my half of the x tile has landed"; the leader's MMA thread issues tcgen05.mma.cta_group::2
+// and hands slots back to both CTAs with tcgen05.commit ... multicast::cluster.
+#pragma once
+#include "gptq_umma.cuh"
+
+namespace gptq {
+
+constexpr int kUmma2Threads = 320;     // TMA warp, MMA/TMEM warp, two sets of four dequant warps
+constexpr int kUmma2Tok = 256;         // tokens per pair tile (128 loaded by each CTA)
+constexpr int kUmma2AStages = 8;
+constexpr uint32_t kUmma2Cols = 512;   // accumulator 256 + A ring 8 x 32
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in every CTA of `cta_mask` once all tcgen05
+// operations issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(cta_mask)
+        : "memory");
+}
+__device__ __forceinline__ void umma_f16_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive (release, cluster scope) on a barrier of another CTA of the cluster, given its cluster-window address
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded like mbar_wait, but observing arrivals from the peer CTA
+__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    const uint64_t start = global_timer_ns();
+    for (;;) {
+        for (int it = 0; it < 256; ++it)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (global_timer_ns() - start > kWaitLimitNs) break;
+    }
+    atomicMax(&g_device_status, (int)kStatusWaitTimeout);
+    return false;
+}
+
+__global__ void __launch_bounds__(kUmma2Threads, 1)
+umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
+{
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int kHalfTok = kUmma2Tok / 2;                 // tokens whose x rows this CTA loads
+    constexpr int kStage = umma_stage_bytes(kHalfTok, 1);
+    constexpr int kOffW = kHalfTok * 128, kOffS = kOffW + kUmmaWBlockBytes, kOffZ = kOffS + kItemSBytes;
+    constexpr uint32_t kAcol = kUmma2Tok;                  // accumulator first, then the A ring
+    constexpr int NA = kUmma2AStages, SETS = 2;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 192;
+    const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
+    const uint32_t ring = base + 1024;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NS = a.stages;
+    const int ptiles = a.N / kPanel / 2;
+    const int pair = blockIdx.x >> 1, rank = blockIdx.x & 1;             // cluster = CTAs 2 pair, 2 pair + 1
+    const int mt = pair / ptiles, p = (pair - mt * ptiles) * 2 + rank;   // this CTA's weight panel
+    const int m0 = mt * kUmma2Tok;
+    const int NB = a.K / kUmmaBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kUmmaDequantWarps + 1);       // this CTA's dequant warps + the pair's MMA
+        }
+        for (int s = 0; s < NA; ++s) {
+            mbar_init(bar_afull + 8 * s, 2 * kUmmaDequantWarps);       // dequant warps of BOTH CTAs (leader's copy is used)
+            mbar_init(bar_aempty + 8 * s, 1);
+        }
+        mbar_init(bar_dfull, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, kUmma2Cols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    // both CTAs' barriers exist before anything arrives on them from the other CTA
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = lds32(tmem_slot);
+    pdl_launch_dependents();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer (one thread per CTA)
+        if (lane == 0) {
+            tma_prefetch_descriptor(&w_map);
+            tma_prefetch_descriptor(&x_map);
+            auto issue_w = [&](int b, int s) {
+                const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
+                mbar_expect_tx(bar, kUmmaWBlockBytes + kItemSBytes + kItemZBytes);
+                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b) * 64, bar);
+                const size_t t = (size_t)p * a.G + (b >> 1);
+                bulk_g2s(st + kOffS, a.scales + t * kItemSBytes, kItemSBytes, bar);
+                bulk_g2s(st + kOffZ, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
+            };
+            const int n_pre = NB < NS ? NB : NS;
+            for (int b = 0; b < n_pre; ++b) issue_w(b, b);   // weights do not depend on earlier kernels
+            pdl_wait();
+            int s = 0, round = 0;
+            for (int b = 0; b < NB; ++b) {
+                const uint32_t bar = bar_full + 8 * s;
+                if (b >= NS) {
+                    if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
+                    issue_w(b, s);
+                }
+                // this CTA's half of the token tile: rows m0 + 128 rank .. + 127 (rows >= M read as zero)
+                mbar_arrive_expect_tx(bar, (uint32_t)(kHalfTok * 128));
+                tma_load_2d(ring + s * kStage, &x_map, b * kUmmaBlockK, m0 + rank * kHalfTok, bar);
+                if (++s == NS) { s = 0; ++round; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issue (one thread of the leader CTA)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = umma_idesc_f16(256, kUmma2Tok);
+            int s = 0, sa = 0;
+            uint32_t ph = 0, pha = 0;
+            bool ok = true;
+            for (int b = 0; b < NB && ok; ++b) {
+                // own x half landed; both CTAs' A stages written (which implies the peer's x half landed too)
+                ok = mbar_wait(bar_full + 8 * s, ph) && mbar_wait_cluster(bar_afull + 8 * sa, pha);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    umma_f16_ts_pair(tmem_base, tmem_base + kAcol + sa * 32 + kk * 8, bdesc + (uint64_t)(kk * 2), idesc,
+                                     (uint32_t)((b | kk) != 0));
+                umma_commit_pair(bar_aempty + 8 * sa, 3);   // both CTAs: this A stage may be overwritten
+                umma_commit_pair(bar_empty + 8 * s, 3);     // both CTAs: and so may the x tile of this stage
+                if (++s == NS) { s = 0; ph ^= 1u; }
+                if (++sa == NA) { sa = 0; pha ^= 1u; }
+            }
+            umma_commit_pair(bar_dfull, 3);
+        }
+    } else {
+        // ---------------------------------------------------------------- dequant warps, then epilogue
+        const int q = warp & 3;                 // the 32 TMEM lanes this warp may touch
+        const int set = (warp - 2) >> 2;        // which K64 blocks: set, set + 2, ...
+        const int n = 32 * q + lane;            // weight column inside the panel = TMEM lane
+        const int u = n >> 4, g = n & 7, h = (n >> 3) & 1;
+        uint32_t w_rd[4];
+#pragma unroll
+        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
+        const uint32_t s_rd = kOffS + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + 8 * u + g;
+        constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
+        const uint32_t leader_afull = map_to_cluster_rank(bar_afull, 0);   // the leader's a_full barriers
+        int s = set % NS, sa = set % NA;
+        uint32_t ph = (uint32_t)(set / NS) & 1u, pha = (uint32_t)(set / NA) & 1u;
+        bool ok = true;
+        for (int b = set; b < NB && ok; b += SETS) {
+            const uint32_t st = ring + s * kStage;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
+            if (!ok) break;
+            uint32_t sh;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
+            const uint32_t s2 = sh * 0x00010001u;
+            const uint32_t zb = lds8(st + z_rd);
+            const uint32_t z = h ? (zb >> 4) : (zb & 15u);
+            const uint32_t zlo = (z * 0x00010001u) | MAGIC_LO, zhi = (z * 0x00100010u) | MAGIC_HI;
+            uint2 wv[4];
+#pragma unroll
+            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
+            uint32_t r[32];
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+                for (int t4 = 0; t4 < 4; ++t4) {
+                    uint32_t w = jj ? wv[t4].y : wv[t4].x;       // rows 32 jj + 8 t4 + (0..7), TMEM columns 16 jj + 4 t4 + (0..3)
+                    uint32_t *o = r + 16 * jj + 4 * t4;
+                    o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
+                    o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                    w >>= 8;
+                    o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
+                    o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                }
+            if (b >= NA) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1u));
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+            tmem_st_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + kAcol + sa * 32, r);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster(leader_afull + 8 * sa);   // "my A stage and my x half are ready" to the leader
+                mbar_arrive(bar_empty + 8 * s);               // the packed weights of this stage have been read
+            }
+            s += SETS;
+            if (s >= NS) { s -= NS; ph ^= 1u; }
+            sa += SETS;
+            if (sa >= NA) { sa -= NA; pha ^= 1u; }
+        }
+        // ---- epilogue: lane n of this CTA's accumulator holds y[m0 .. m0+256, 128 p + n]
+        pdl_wait();
+        ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
+        if (ok) {
+            tc_fence_after_sync();
+            __half *yp = a.y + (size_t)p * kPanel + n;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kUmma2Tok; c0 += 32) {
+                if (m0 + c0 >= a.M) break;
+                if (((c0 >> 5) & 1) != set) continue;       // the two warp sets share the token chunks
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int m = m0 + c0 + i;
+                    if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
+                }
+            }
+        }
+    }
+    // neither CTA may free tensor memory or exit while the pair's MMAs or the peer's arrivals can still touch it
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, kUmma2Cols);
+    }
+}
+
+struct Umma2Plan {
+    int stages;
+    int ctas;        // 2 * (panel pairs) * (256-token tiles)
+    int smem_bytes;
+};
+
+inline bool umma2_applicable(int M, int N) { return M >= 256 && (N / kPanel) % 2 == 0; }
+
+inline Umma2Plan plan_umma2(int M, int N, int K)
+{
+    Umma2Plan pl{};
+    const int stage = umma_stage_bytes(kUmma2Tok / 2, 1);
+    int stages = (227 * 1024 - 1024 - 2048) / stage;
+    if (stages > 8) stages = 8;
+    if (stages > K / kUmmaBlockK) stages = K / kUmmaBlockK;
+    pl.stages = stages;
+    pl.ctas = (N / kPanel) * ((M + kUmma2Tok - 1) / kUmma2Tok);
+    pl.smem_bytes = 2048 + stages * stage;
+    const int floor_one_per_sm = (227 * 1024) / 2 + 512;     // one CTA per SM: the pair owns all tensor memory
+    if (pl.smem_bytes < floor_one_per_sm) pl.smem_bytes = floor_one_per_sm;
+    return pl;
+}
+
+int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
+                 int K, const Umma2Plan &plan, cudaStream_t s)
+{
+    UmmaArgs args;
+    args.scales = (const uint8_t *)scales;
+    args.qzeros = (const uint8_t *)qzeros;
+    args.y = y;
+    args.M = M;
+    args.N = N;
+    args.K = K;
+    args.G = K / kGroup;
+    args.S = 1;
+    args.stages = plan.stages;
+    CUtensorMap w_map, x_map;
+    const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
+    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 64,
+                                CU_TENSOR_MAP_SWIZZLE_64B);
+    if (st) return st;
+    // x as [M rows, K halves]; a box is 64 k of one CTA's half (128 rows) of the token tile
+    st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
+                            (uint64_t)K * sizeof(__half), 64, kUmma2Tok / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (st) return st;
+    static int configured_smem[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
+    if (configured_smem[dev] < plan.smem_bytes) {
+        e = cudaFuncSetAttribute(umma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaFuncSetAttribute(umma2_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        configured_smem[dev] = plan.smem_bytes;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)plan.ctas);
+    cfg.blockDim = dim3(kUmma2Threads);
+    cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, umma2_kernel, args, w_map, x_map));
+}
+
+}  // namespace gptq

@@ -137,6 +137,23 @@ def test_gemm_token_count_boundaries(M, act, ws):
     assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
 
 
+@pytest.mark.parametrize("K,N,M,act", [(512, 256, 256, False), (1024, 512, 300, False), (640, 256, 513, True),
+                                        (4096, 4096, 1024, False)])
+def test_gemm_on_cta_pairs(K, N, M, act, ws):
+    """The optional cta_group::2 variant of the tcgen05 kernel: same result within the same tolerance."""
+    L = wl.make_linear(K, N, seed=wl.seed_for("pairs", K, N, act), act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("pairs-x", K, M))
+    B.check(B.gptq_set_cta_pairs(1), "pairs on")
+    try:
+        y, _ = run_gemm(L, x, ws)
+    finally:
+        B.check(B.gptq_set_cta_pairs(0), "pairs off")
+    if K * N * M <= 1 << 28:
+        assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+    else:
+        sampled_check(L, x, y, 4000, seed=M)
+
+
 def test_gemm_leaves_rows_beyond_m_alone(ws):
     """The last token tile is ragged: rows past M of the output buffer must not be written."""
     K, N = 512, 256
