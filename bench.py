@@ -45,8 +45,8 @@ FALLBACK_TFLOPS = 1590.0
 # on (`--print-digest`); `traffic` is that ratio times the timed launches' algorithmic bytes, and
 # null once the sources have changed since the capture.
 NCU_TRAFFIC = {
-    "splitk_kernel<1>": {"digest": "PENDING", "ratio": 1.0004},      # M = 1, the four 7B shapes
-    "umma_kernel<256,4,1,2>": {"digest": "PENDING", "ratio": 0.678},  # qkv, M = 2048 (y still in L2 at kernel end)
+    "splitk_kernel<1>": {"digest": "f249be066873b78a", "ratio": 1.0004},      # M = 1, the four 7B shapes
+    "umma_kernel<256,4,1,2>": {"digest": "f249be066873b78a", "ratio": 0.685},  # qkv, M = 2048 (y still in L2 at kernel end)
 }
 
 WORKLOADS = {
