@@ -150,6 +150,29 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
 /* Size in bytes of the built-in scratch array (host-only, no CUDA call). */
 size_t gptq_noalloc_scratch_bytes(void);
 
+/* One matmul of a step for gptq_gemm_host_batch: the arguments of gptq_gemm_host. */
+typedef struct {
+    const void *x_host;      /* fp16 [M, K], host (pinned for true asynchrony) */
+    const void *qweight;     /* device, repacked */
+    const void *qzeros;      /* device, repacked */
+    const void *scales;      /* device, repacked */
+    const int32_t *g_idx;    /* device perm_out, or NULL */
+    void *y_host;            /* fp16 [M, N], host */
+    void *x_stage;           /* device, M*K fp16 */
+    void *y_stage;           /* device, M*N fp16 */
+    int M, N, K, group_size, act_order;
+} gptq_host_problem_t;
+
+/* A step of matmuls whose activations live in host memory (the linears of a decode step, configs of
+ * Section 4's serving setting): for each problem in order, on `stream`: copy x to the device, gptq_gemm,
+ * copy y back - the same results as `count` gptq_gemm_host calls, but pipelined: the copies run on two
+ * internal streams (created on first use), so x of problem i+1 goes up and y of problem i-1 comes down
+ * while matmul i runs; the matmuls themselves stay in order on `stream`, and `stream` completes after
+ * the last copy.  Staging buffers may be shared between problems (reuse waits for the earlier user).
+ * All problems are validated before anything is enqueued; on an invalid problem *bad_index (if not
+ * NULL) receives its index and nothing runs. */
+int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
+
 /* Synchronises `stream` and returns GPTQ_ERR_TIMEOUT if any kernel's bounded wait gave up
  * since the last check (the flag is then cleared), GPTQ_ERR_CUDA on a runtime error, else OK. */
 int gptq_check_status(void *stream);

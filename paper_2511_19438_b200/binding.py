@@ -42,6 +42,16 @@ class gptq_plan_t(ctypes.Structure):
     ]
 
 
+class gptq_host_problem_t(ctypes.Structure):
+    _fields_ = [
+        ("x_host", ctypes.c_void_p), ("qweight", ctypes.c_void_p), ("qzeros", ctypes.c_void_p),
+        ("scales", ctypes.c_void_p), ("g_idx", ctypes.c_void_p), ("y_host", ctypes.c_void_p),
+        ("x_stage", ctypes.c_void_p), ("y_stage", ctypes.c_void_p),
+        ("M", ctypes.c_int), ("N", ctypes.c_int), ("K", ctypes.c_int), ("group_size", ctypes.c_int),
+        ("act_order", ctypes.c_int),
+    ]
+
+
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
 _SIGNATURES = {
     "gptq_status_string": (ctypes.c_char_p, [_i]),
@@ -57,6 +67,7 @@ _SIGNATURES = {
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_noalloc_scratch_bytes": (_sz, []),
+    "gptq_gemm_host_batch": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_check_status": (_i, [_vp]),
     "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_noalloc": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
@@ -163,6 +174,23 @@ def gptq_gemm_noalloc(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size,
 
 def gptq_noalloc_scratch_bytes() -> int:
     return _lib.gptq_noalloc_scratch_bytes()
+
+
+def make_host_problems(items):
+    """Marshals a list of (x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_stage, M, N, K, group_size,
+    act_order) tuples into a C array for gptq_gemm_host_batch (build once, reuse every step)."""
+    arr = (gptq_host_problem_t * len(items))()
+    for i, it in enumerate(items):
+        ptrs = [_ptr(v) for v in it[:8]]
+        arr[i] = gptq_host_problem_t(*ptrs, int(it[8]), int(it[9]), int(it[10]), int(it[11]), int(bool(it[12])))
+    return arr
+
+
+def gptq_gemm_host_batch(problems, stream=None):
+    """Returns (status, bad_index); `problems` comes from make_host_problems."""
+    bad = ctypes.c_int(-1)
+    st = _lib.gptq_gemm_host_batch(problems, len(problems), _stream(stream), ctypes.byref(bad))
+    return st, bad.value
 
 
 def gptq_check_status(stream=None) -> int:

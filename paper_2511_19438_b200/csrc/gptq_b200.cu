@@ -9,6 +9,7 @@
 
 #include <atomic>
 #include <mutex>
+#include <vector>
 
 namespace gptq {
 
@@ -91,6 +92,31 @@ static StreamKGemmPlan make_streamk_plan(int M, int N, int K, int act_order, int
 static size_t gemm_workspace_need(int M, int K, int act_order)
 {
     return act_order ? (((size_t)M * K * sizeof(__half) + 255) & ~(size_t)255) : 0;
+}
+
+// Copy streams and events of gptq_gemm_host_batch (per device, created on first use; no device memory).
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    std::vector<cudaEvent_t> events;
+};
+static HostPipe g_host_pipe[kMaxDevices];
+
+static int ensure_host_pipe(int dev, size_t n_events, HostPipe **out)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    HostPipe &p = g_host_pipe[dev];
+    cudaError_t e;
+    if (p.in == nullptr && (e = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking)) != cudaSuccess)
+        return record_cuda_error(e);
+    if (p.out == nullptr && (e = cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking)) != cudaSuccess)
+        return record_cuda_error(e);
+    while (p.events.size() < n_events) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return record_cuda_error(e);
+        p.events.push_back(ev);
+    }
+    *out = &p;
+    return GPTQ_OK;
 }
 
 }  // namespace gptq
@@ -409,6 +435,79 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
         if (st) return st;
     }
     return GPTQ_OK;
+}
+
+int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
+{
+    if (!problems || count < 0) return GPTQ_ERR_NULL;
+    for (int i = 0; i < count; ++i) {
+        const gptq_host_problem_t &q = problems[i];
+        int st = GPTQ_OK;
+        if (!q.x_host || !q.y_host || !q.x_stage || !q.y_stage || !q.qweight || !q.qzeros || !q.scales ||
+            (q.act_order && !q.g_idx))
+            st = GPTQ_ERR_NULL;
+        if (!st) st = check_shape(q.M, q.N, q.K, q.group_size);
+        if (!st && (!aligned16(q.x_stage) || !aligned16(q.y_stage) || !aligned16(q.qweight) || !aligned16(q.qzeros) ||
+                    !aligned16(q.scales)))
+            st = GPTQ_ERR_ALIGN;
+        if (!st) st = check_fast_path(q.N, q.K, q.group_size);
+        if (st) {
+            if (bad_index) *bad_index = i;
+            return st;
+        }
+    }
+    if (count == 0) return GPTQ_OK;
+    // Three-stage pipeline over two internal copy streams: x_i goes up while matmul i-1 runs and y_i-1 comes down.
+    int dev, sms;
+    int st = current_device_sms(&dev, &sms);
+    if (st) return st;
+    HostPipe *pipe = nullptr;
+    st = ensure_host_pipe(dev, 3 * (size_t)count + 1, &pipe);
+    if (st) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaEvent_t *ev_x = pipe->events.data(), *ev_g = ev_x + count, *ev_y = ev_g + count, ev_start = ev_y[count];
+    auto check = [&](cudaError_t e) { return record_cuda_error(e); };
+    // copies must not start before earlier work on `stream` (which may still use the staging buffers)
+    if ((st = check(cudaEventRecord(ev_start, s)))) return st;
+    if ((st = check(cudaStreamWaitEvent(pipe->in, ev_start, 0)))) return st;
+    if ((st = check(cudaStreamWaitEvent(pipe->out, ev_start, 0)))) return st;
+    for (int i = 0; i < count; ++i) {
+        const gptq_host_problem_t &q = problems[i];
+        // a staging buffer shared with an earlier problem is reused only after that problem is done with it
+        for (int j = i - 1; j >= 0; --j)
+            if (problems[j].x_stage == q.x_stage) {
+                if ((st = check(cudaStreamWaitEvent(pipe->in, ev_g[j], 0)))) return st;
+                break;
+            }
+        if ((st = check(cudaMemcpyAsync(q.x_stage, q.x_host, (size_t)q.M * q.K * sizeof(__half), cudaMemcpyHostToDevice,
+                                        pipe->in))))
+            return st;
+        if ((st = check(cudaEventRecord(ev_x[i], pipe->in)))) return st;
+        if ((st = check(cudaStreamWaitEvent(s, ev_x[i], 0)))) return st;
+        for (int j = i - 1; j >= 0; --j)
+            if (problems[j].y_stage == q.y_stage) {
+                if ((st = check(cudaStreamWaitEvent(s, ev_y[j], 0)))) return st;
+                break;
+            }
+        st = gptq_gemm(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
+                       q.act_order, stream);
+        if (st) {
+            if (bad_index) *bad_index = i;
+            break;   // still join the copy streams below
+        }
+        if ((st = check(cudaEventRecord(ev_g[i], s)))) return st;
+        if ((st = check(cudaStreamWaitEvent(pipe->out, ev_g[i], 0)))) return st;
+        if ((st = check(cudaMemcpyAsync(q.y_host, q.y_stage, (size_t)q.M * q.N * sizeof(__half), cudaMemcpyDeviceToHost,
+                                        pipe->out))))
+            return st;
+        if ((st = check(cudaEventRecord(ev_y[i], pipe->out)))) return st;
+    }
+    // `stream` finishes after the last copy of each direction
+    int st2 = check(cudaEventRecord(ev_start, pipe->in));
+    if (!st2) st2 = check(cudaStreamWaitEvent(s, ev_start, 0));
+    if (!st2) st2 = check(cudaEventRecord(ev_x[0], pipe->out));
+    if (!st2) st2 = check(cudaStreamWaitEvent(s, ev_x[0], 0));
+    return st ? st : st2;
 }
 
 int gptq_check_status(void *stream)

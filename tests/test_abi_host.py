@@ -73,6 +73,22 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_gemm_host(None, A16, A16, A16, None, A16, A16, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
 
 
+def test_host_batch_validates_every_problem_before_running():
+    good = (A16, A16, A16, A16, None, A16, A16, A16, 1, 128, 128, 128, 0)
+    bad_shape = good[:9] + (130,) + good[10:]
+    arr = B.make_host_problems([good, good, bad_shape])
+    st, bad = B._lib.gptq_gemm_host_batch(arr, 3, 0, None), None
+    assert st == B.GPTQ_ERR_SHAPE
+    import ctypes
+    idx = ctypes.c_int(-1)
+    assert B._lib.gptq_gemm_host_batch(arr, 3, 0, ctypes.byref(idx)) == B.GPTQ_ERR_SHAPE and idx.value == 2
+    missing = (None,) + good[1:]
+    arr = B.make_host_problems([missing])
+    assert B._lib.gptq_gemm_host_batch(arr, 1, 0, ctypes.byref(idx)) == B.GPTQ_ERR_NULL and idx.value == 0
+    assert B._lib.gptq_gemm_host_batch(None, 1, 0, None) == B.GPTQ_ERR_NULL
+    assert B._lib.gptq_gemm_host_batch(arr, 0, 0, None) == B.GPTQ_OK      # an empty step is fine
+
+
 def test_repack_bytes_equal_canonical_sizes():
     for (K, N) in list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()):
         G = K // 128

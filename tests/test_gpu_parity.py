@@ -272,6 +272,31 @@ def test_gemm_host_round_trip(ws):
     assert_close(y_host.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, None, 128), K)
 
 
+def test_gemm_host_batch_step(ws):
+    """A small step of three matmuls (one act-order, one on the tcgen05 kernel) through the native batch entry."""
+    specs = [(1024, 256, 2, False), (640, 256, 5, True), (512, 384, 40, False)]
+    items, keep = [], []
+    for (K, N, M, act) in specs:
+        L = wl.make_linear(K, N, seed=wl.seed_for("batch", K, N, act), act_order=act)
+        D = H.upload_and_repack(L)
+        ws.ensure_for(M, D)
+        x_np = wl.make_x(M, K, wl.seed_for("batch-x", K, M))
+        xh = torch.from_numpy(x_np).pin_memory()
+        yh = torch.zeros((M, N), dtype=torch.float16).pin_memory()
+        xs = torch.empty((M, K), dtype=torch.float16, device="cuda")
+        ys = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        items.append((xh, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, yh, xs, ys, M, N, K, 128, act))
+        keep.append((L, x_np, yh, D))
+    # the workspace must cover the largest act-order problem of the step
+    ws.ensure(max(B.gptq_workspace_bytes(M, N, K, 128, act) for (K, N, M, act) in specs))
+    st, bad = B.gptq_gemm_host_batch(B.make_host_problems(items))
+    assert (st, bad) == (B.GPTQ_OK, -1)
+    torch.cuda.synchronize()
+    assert B.gptq_check_status() == B.GPTQ_OK
+    for (L, x_np, yh, _D), (K, N, M, act) in zip(keep, specs):
+        assert_close(yh.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+
+
 # ------------------------------------------------------------------------------- matmul, full size
 def sampled_check(L, x, y, n_samples, seed):
     r = np.random.default_rng(seed)
