@@ -24,7 +24,7 @@
 namespace gptq {
 
 // warp 0: TMA producer, warp 1: MMA issue + TMEM, then four dequant/epilogue warps per panel of the CTA
-// (two sets of them, taking alternate K64 blocks, when one warp per scheduler cannot keep up with the MMA)
+// (two sets of them, taking alternate K groups, when one warp per scheduler cannot keep up with the MMA)
 __host__ __device__ constexpr int umma_threads(int NP, int SETS) { return 64 + 128 * NP * SETS; }
 constexpr int kUmmaDequantWarps = 4;     // per panel: one warp per 32 TMEM lanes
 constexpr int kUmmaBlockK = 64;
@@ -191,16 +191,20 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             tma_prefetch_descriptor(&x_map);
             auto issue_w = [&](int b, int s) {
                 const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
-                mbar_expect_tx(bar, NP * (kUmmaWBlockBytes + kItemSBytes + kItemZBytes));
+                const bool first_of_group = (b & 1) == 0;
+                mbar_expect_tx(bar, NP * (kUmmaWBlockBytes + (first_of_group ? kItemSBytes + kItemZBytes : 0)));
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     const int p = p0 + j;
                     // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
                     tma_load_2d(st + kOffW + j * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
-                    // the group's scales and zeros travel with both of its blocks (320 bytes)
-                    const size_t t = (size_t)p * a.G + g0 + (b >> 1);
-                    bulk_g2s(st + kOffS + j * kItemSBytes, a.scales + t * kItemSBytes, kItemSBytes, bar);
-                    bulk_g2s(st + kOffZ + j * kItemZBytes, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
+                    // scales and zeros travel with the group's first block; the dequant warps keep them in
+                    // registers for the second (every TMA operation costs the producer thread issue time)
+                    if (first_of_group) {
+                        const size_t t = (size_t)p * a.G + g0 + (b >> 1);
+                        bulk_g2s(st + kOffS + j * kItemSBytes, a.scales + t * kItemSBytes, kItemSBytes, bar);
+                        bulk_g2s(st + kOffZ + j * kItemZBytes, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
+                    }
                 }
             };
             const int n_pre = NB < NS ? NB : NS;
@@ -261,19 +265,25 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + j * kUmmaWBlockBytes + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
         const uint32_t s_rd = kOffS + j * kItemSBytes + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + j * kItemZBytes + 8 * u + g;
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-        int s = set % NS, sa = set % NA;
-        uint32_t ph = (uint32_t)(set / NS) & 1u, pha = (uint32_t)(set / NA) & 1u;
+        // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1
+        int b = 2 * set;
+        int s = b % NS, sa = b % NA;
+        uint32_t ph = (uint32_t)(b / NS) & 1u, pha = (uint32_t)(b / NA) & 1u;
+        uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
         bool ok = true;
-        for (int b = set; b < NB && ok; b += SETS) {
+        for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
             if (!ok) break;
-            uint32_t sh;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
-            const uint32_t s2 = sh * 0x00010001u;
-            const uint32_t zb = lds8(st + z_rd);
-            const uint32_t z = h ? (zb >> 4) : (zb & 15u);
-            const uint32_t zlo = (z * 0x00010001u) | MAGIC_LO, zhi = (z * 0x00100010u) | MAGIC_HI;
+            if ((b & 1) == 0) {
+                uint32_t sh;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
+                s2 = sh * 0x00010001u;
+                const uint32_t zb = lds8(st + z_rd);
+                const uint32_t z = h ? (zb >> 4) : (zb & 15u);
+                zlo = (z * 0x00010001u) | MAGIC_LO;
+                zhi = (z * 0x00100010u) | MAGIC_HI;
+            }
             uint2 wv[4];
 #pragma unroll
             for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
@@ -303,10 +313,11 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 mbar_arrive(bar_afull + 8 * (j * NA + sa));
                 mbar_arrive(bar_empty + 8 * s);
             }
-            s += SETS;
-            if (s >= NS) { s -= NS; ph ^= 1u; }
-            sa += SETS;
-            if (sa >= NA) { sa -= NA; pha ^= 1u; }
+            const int step = (b & 1) ? 2 * SETS - 1 : 1;   // to this set's next block
+            s += step;
+            while (s >= NS) { s -= NS; ph ^= 1u; }
+            sa += step;
+            while (sa >= NA) { sa -= NA; pha ^= 1u; }
         }
         // ---- epilogue: lane n of the accumulator holds y[m0 .. m0+TOK, 128 p + n]
         pdl_wait();
