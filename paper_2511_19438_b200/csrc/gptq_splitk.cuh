@@ -11,10 +11,12 @@
 // q - z) and feeds them as the 16-row A operand of mma.sync.m16n8k16, tokens as the 8-wide B
 // operand.  The group's scale multiplies the fp32 group sum once per group.
 //
-// The K-partials of a panel never touch global memory: every CTA parks its fp32 tile in its own
-// shared memory, the cluster synchronises, and CTA r sums columns [128 r / S, 128 (r+1) / S) of
-// all S tiles through distributed shared memory in rank order (a fixed order: results are
-// reproducible), rounds once to fp16 and stores y.
+// The K-partials of a panel never touch global memory: CTA r owns columns [128 r / S, 128 (r+1) / S);
+// every CTA sends each owner its slice of its fp32 tile with st.async into the owner's shared
+// memory (counted in bytes on the owner's mbarrier), and each owner, once all S slices have landed,
+// sums them in rank order (a fixed order: results are reproducible), rounds once to fp16 and
+// stores y.  The only cluster-wide barrier is split around the main loop (arrive after the
+// barriers are armed, wait before the first send), so no CTA waits for a slower neighbour.
 #pragma once
 #include "gptq_common.cuh"
 #include "gptq_tma.cuh"
@@ -43,6 +45,44 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr)
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
     return v;
 }
+// fire-and-forget 4-byte store into another CTA's shared memory; the 4 bytes are counted on that CTA's mbarrier
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar)
+                 : "memory");
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded like mbar_wait, but observing arrivals and stores from other CTAs of the cluster
+__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    const uint64_t start = global_timer_ns();
+    for (;;) {
+        for (int it = 0; it < 256; ++it)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (global_timer_ns() - start > kWaitLimitNs) break;
+    }
+    atomicMax(&g_device_status, (int)kStatusWaitTimeout);
+    return false;
+}
+
 __device__ __forceinline__ void sts_f32(uint32_t addr, float v)
 {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
@@ -78,6 +118,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_base;                  // stages x 8 B
     const uint32_t bar_empty = smem_base + 64;            // stages x 8 B
+    const uint32_t bar_recv = smem_base + 128;
     const uint32_t ring = smem_base + kRingOffset;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int S = a.S;
@@ -92,10 +133,14 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kConsumerWarps);
         }
+        mbar_init(bar_recv, 1);
         fence_barrier_init();
         fence_proxy_async();
+        // split-K: S slices of a.M x (128 / S) floats will arrive in this CTA's receive buffer
+        if (S > 1) mbar_arrive_expect_tx(bar_recv, (uint32_t)(a.M * kPanel * 4));
     }
     __syncthreads();
+    if (S > 1) cluster_arrive_release();   // "my receive barrier is armed"; waited for before the first send
     pdl_launch_dependents();
 
     float acc[MT][4];
@@ -228,39 +273,39 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         return;
     }
 
-    // ---- split-K: park this CTA's fp32 tile [MT*8 rows][128 cols] at the start of the ring ----------
+    // ---- split-K: send each owner its column slice, then finish the own slice ------------------------
+    __syncwarp();
+    cluster_wait_acquire();                 // every CTA of the cluster has armed its receive barrier
     if (warp < kConsumerWarps) {
-        named_bar_sync(1, kConsumerThreads);   // every consumer warp has finished reading the ring
+        const int width = kPanel / S;       // S is 2, 4 or 8
+        const uint32_t recv = ring + (uint32_t)a.stages * kStage;   // [sender rank][token row][width] floats
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
-                sts_f32(ring + (uint32_t)(m * kPanel + col + 8 * (i >> 1)) * 4u, acc[mt][i]);
+                if (m < a.M) {
+                    const int c = col + 8 * (i >> 1), q = c / width;
+                    const uint32_t off = (uint32_t)((rank * a.M + m) * width + (c - q * width)) * 4u;
+                    st_async_f32(map_to_cluster_rank(recv + off, (uint32_t)q), acc[mt][i],
+                                 map_to_cluster_rank(bar_recv, (uint32_t)q));
+                }
             }
-    }
-    __syncwarp();
-    cluster_arrive_release();
-    cluster_wait_acquire();
-    if (warp < kConsumerWarps) {
-        // CTA `rank` finishes columns [c_lo, c_lo + width) of the panel for every token row
-        const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
-        for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
-            const int m = idx / width, cc = c_lo + idx - m * width;
-            const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
-            float v[8];
+        if (mbar_wait_cluster(bar_recv, 0)) {
+            const int c_lo = rank * width;
+            for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
+                const int m = idx / width, cc = idx - m * width;
+                float v[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = q < S ? ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)q)) : 0.f;
-            float sum = 0.f;
+                for (int q = 0; q < 8; ++q)
+                    v[q] = q < S ? lds_f32(recv + (uint32_t)((q * a.M + m) * width + cc) * 4u) : 0.f;
+                float sum = 0.f;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) sum += v[q];   // rank order
-            a.y[(size_t)m * a.N + (size_t)p * kPanel + cc] = __float2half_rn(sum);
+                for (int q = 0; q < 8; ++q) sum += v[q];   // rank order
+                a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(sum);
+            }
         }
     }
-    // no CTA may exit (and free its shared memory) while a peer can still read its tile
-    __syncwarp();
-    cluster_arrive_release();
-    cluster_wait_acquire();
 }
 
 // Resident CTAs per SM by token tile: registers and ring size are set so that three CTAs of the
@@ -299,16 +344,15 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
     if (per_sm > cps_max) per_sm = cps_max;
     const int smem_cap = (227 * 1024) / per_sm - 1024;                 // per_sm CTAs fit ...
     const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;          // ... per_sm + 1 do not
-    int stages = (smem_cap - 2 * kRingOffset) / stage;
+    const int recv_bytes = MT * 4096;   // receive buffer of the split-K exchange, after the ring
+    int stages = (smem_cap - 2 * kRingOffset - recv_bytes) / stage;
     if (stages > 8) stages = 8;
     if (stages > items_per_cta) stages = items_per_cta;
-    // the ring doubles as the fp32 partial tile (MT * 4 KB) at the end
-    while (stages * stage < MT * 4096) ++stages;
     pl.m_tile = MT * 8;
     pl.S = S;
     pl.stages = stages;
     pl.ctas = panels * S;
-    pl.smem_bytes = 2 * kRingOffset + stages * stage;
+    pl.smem_bytes = 2 * kRingOffset + stages * stage + recv_bytes;
     if (pl.smem_bytes < smem_floor) pl.smem_bytes = smem_floor;
     return pl;
 }

@@ -62,31 +62,6 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded like mbar_wait, but observing arrivals from the peer CTA
-__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    const uint64_t start = global_timer_ns();
-    for (;;) {
-        for (int it = 0; it < 256; ++it)
-            if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (global_timer_ns() - start > kWaitLimitNs) break;
-    }
-    atomicMax(&g_device_status, (int)kStatusWaitTimeout);
-    return false;
-}
-
 __global__ void __launch_bounds__(kUmma2Threads, 1)
 umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
