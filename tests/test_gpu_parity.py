@@ -363,6 +363,39 @@ def test_config4_prefill_sampled(name, M, act, ws):
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
+def test_graph_replayed_step_matches_oracle(ws):
+    """The launch configuration bench.py times: gptq_gemm calls captured in a CUDA graph (programmatic dependent
+    launches inside a graph, back-to-back kernels that prefetch weights early), replayed, then sampled."""
+    shapes = [("qkv", 1), ("o", 8), ("gate_up", 16), ("down", 4), ("o", 64), ("qkv", 300)]
+    layers = []
+    for name, M in shapes:
+        K, N = wl.SHAPES_7B[name]
+        L = wl.make_linear(K, N, seed=wl.seed_for("graph", name, M))
+        D = H.upload_and_repack(L)
+        x_np = wl.make_x(M, K, wl.seed_for("graph-x", name, M))
+        x = H.to_device(x_np)
+        y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+        ws.ensure_for(M, D)
+        layers.append((L, D, x_np, x, y))
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for (_L, D, _x_np, x, y) in layers:        # eager pass configures the kernels
+            H.gemm(x, D, y)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for (_L, D, _x_np, x, y) in layers:
+                H.gemm(x, D, y)
+        for (_L, _D, _x_np, _x, y) in layers:
+            y.zero_()
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+    assert B.gptq_check_status() == B.GPTQ_OK
+    for (L, _D, x_np, _x, y) in layers:
+        sampled_check(L, x_np, y.cpu().numpy(), 2000, seed=x_np.shape[0])
+
+
 @pytest.mark.parametrize("M", wl.STEP_M)
 def test_config5_decode_step_layers(M, ws):
     """Layers 0 and 31 of the 32-layer step (distinct seeded weights per layer)."""
