@@ -107,7 +107,7 @@ struct SplitKPlan {
 };
 
 template <int MT>
-__global__ void __launch_bounds__(kStreamKThreads, MT == 1 ? 3 : MT == 2 ? 2 : 1)
+__global__ void __launch_bounds__(kStreamKThreads, MT <= 2 ? 3 : 1)
 splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -310,7 +310,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 
 // Resident CTAs per SM by token tile: registers and ring size are set so that three CTAs of the
 // narrowest tile fit, which lets the next kernel's first CTAs start (and prefetch weights) early.
-__host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT == 1 ? 3 : MT == 2 ? 2 : 1; }
+__host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT <= 2 ? 3 : 1; }
 
 // Picks the cluster size S in {1, 2, 4, 8} with the smallest estimated time among those whose
 // panels * S CTAs are all resident at once (falling back to all S if none is).  The estimate is

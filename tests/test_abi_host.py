@@ -132,7 +132,7 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     assert pl.m_tile in (8, 16, 32, 64) and pl.m_tile >= min(M, 64)
     assert pl.m_chunks == (M + 63) // 64
     assert 1 <= pl.stages <= 8
-    per_sm = min(-(-pl.ctas // sms), 3 if pl.m_tile == 8 else 2 if pl.m_tile == 16 else 1)
+    per_sm = min(-(-pl.ctas // sms), 3 if pl.m_tile <= 16 else 1)
     assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024          # that many CTAs fit on an SM ...
     assert (per_sm + 1) * (pl.smem_bytes + 1024) > 227 * 1024     # ... and no more (even spreading)
     # the ring doubles as the fp32 partial tile of the cluster reduction
