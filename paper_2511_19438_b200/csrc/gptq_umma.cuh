@@ -114,6 +114,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N)
     return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+__device__ __forceinline__ void sts_f16(uint32_t addr, __half v)
+{
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(v)) : "memory");
+}
+
 struct UmmaArgs {
     const uint8_t *scales;  // tiled
     const uint8_t *qzeros;  // tiled
@@ -322,28 +327,54 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // ---- epilogue: lane n of the accumulator holds y[m0 .. m0+TOK, 128 p + n]
         pdl_wait();
         ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
-        if (ok) {
-            tc_fence_after_sync();
-            __half *yp = a.y + (size_t)p * kPanel + n;
+        if (ok) tc_fence_after_sync();
+        if (S == 1) {
+            // The accumulator holds a column of y per TMEM lane, so a thread's 32 values of a chunk belong to 32
+            // different rows of y.  The four warps of a set turn their 32-token x 128-column chunk around through
+            // the (now idle) ring: fp16 rows of 256 bytes in shared memory, then 16 bytes per thread to y - whole
+            // 128-byte lines instead of 2-byte stores.  Every warp takes part in the named barriers, also
+            // after a wait that gave up (it then moves no data; the status word tells the host).
+            const uint32_t stg = ring + (uint32_t)((j * SETS + set) * (32 * kPanel * 2));
+            const int bar_id = 1 + j * SETS + set;
+            const int tq = 32 * q + lane;           // thread within the set
 #pragma unroll 1
             for (int c0 = 0; c0 < TOK; c0 += 32) {
                 if (m0 + c0 >= a.M) break;
                 if (SETS > 1 && ((c0 >> 5) % SETS) != set) continue;   // the warp sets share the token chunks
+                if (ok) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + j * TOK + c0, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
+                }
+                named_bar_sync(bar_id, 128);
+                if (ok) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int piece = tq + 128 * t, row = piece >> 4, c16 = piece & 15;   // 16 pieces per row
+                        const int m = m0 + c0 + row;
+                        if (m < a.M && c0 + row < TOK) {
+                            const uint4 v = lds128(stg + (uint32_t)piece * 16u);
+                            *reinterpret_cast<uint4 *>(a.y + (size_t)m * a.N + (size_t)p * kPanel + c16 * 8) = v;
+                        }
+                    }
+                }
+                named_bar_sync(bar_id, 128);   // the next chunk overwrites the staging rows
+            }
+        } else if (ok) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < TOK; c0 += 32) {
+                if (m0 + c0 >= a.M) break;
+                if (SETS > 1 && ((c0 >> 5) % SETS) != set) continue;
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + j * TOK + c0, r);
                 tmem_wait_ld();
-                if (S == 1) {
+                // split-K: park the fp32 partial tile [token][column] at the start of the (idle) ring
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int m = m0 + c0 + i;
-                        if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
-                    }
-                } else {
-                    // split-K: park the fp32 partial tile [token][column] at the start of the (idle) ring
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c0 + i < TOK) sts_f32(ring + (uint32_t)((c0 + i) * kPanel + n) * 4u, __uint_as_float(r[i]));
-                }
+                for (int i = 0; i < 32; ++i)
+                    if (c0 + i < TOK) sts_f32(ring + (uint32_t)((c0 + i) * kPanel + n) * 4u, __uint_as_float(r[i]));
             }
         }
     }
