@@ -90,7 +90,8 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
             mbar_init(bar_empty + 8 * s, kUmmaDequantWarps + 1);       // this CTA's dequant warps + the pair's MMA
         }
         for (int s = 0; s < NA; ++s) {
-            mbar_init(bar_afull + 8 * s, 2 * kUmmaDequantWarps);       // dequant warps of BOTH CTAs (leader's copy is used)
+            mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);           // leader's copy is used: its four warps arrive, the
+                                                                       // peer's four send 4 bytes each (transaction count)
             mbar_init(bar_aempty + 8 * s, 1);
         }
         mbar_init(bar_dfull, 1);
@@ -174,7 +175,11 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
         const uint32_t s_rd = kOffS + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + 8 * u + g;
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-        const uint32_t leader_afull = map_to_cluster_rank(bar_afull, 0);   // the leader's a_full barriers
+        // The peer's warps signal the leader's a_full barrier with a fire-and-forget 4-byte st.async that is counted
+        // on the barrier's transaction count (a remote mbarrier.arrive holds the issuing thread up for hundreds of
+        // cycles); the leader's warp 0 of the set arms those 16 bytes with its own arrival.
+        const uint32_t leader_afull = map_to_cluster_rank(bar_afull, 0);
+        const uint32_t leader_slot = map_to_cluster_rank(base + 512 + 4 * warp, 0);
         int s = set % NS, sa = set % NA;
         uint32_t ph = (uint32_t)(set / NS) & 1u, pha = (uint32_t)(set / NA) & 1u;
         bool ok = true;
@@ -214,7 +219,13 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_cluster(leader_afull + 8 * sa);   // "my A stage and my x half are ready" to the leader
+                // "my A stage and my x half are ready" to the leader
+                if (rank == 0) {
+                    if (q == 0) mbar_arrive_expect_tx(bar_afull + 8 * sa, 4 * kUmmaDequantWarps);
+                    else mbar_arrive(bar_afull + 8 * sa);
+                } else {
+                    st_async_f32(leader_slot, 0.f, leader_afull + 8 * sa);
+                }
                 mbar_arrive(bar_empty + 8 * s);               // the packed weights of this stage have been read
             }
             s += SETS;
@@ -225,21 +236,38 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         // ---- epilogue: lane n of this CTA's accumulator holds y[m0 .. m0+256, 128 p + n]
         pdl_wait();
         ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
-        if (ok) {
-            tc_fence_after_sync();
-            __half *yp = a.y + (size_t)p * kPanel + n;
+        if (ok) tc_fence_after_sync();
+        {
+            // as in the single-CTA kernel: each set's four warps turn a 32-token chunk around through the idle ring
+            // and write whole 128-byte lines of y; every warp takes part in the named barriers
+            const uint32_t stg = ring + (uint32_t)(set * (32 * kPanel * 2));
+            const int bar_id = 1 + set;
+            const int tq = 32 * q + lane;
 #pragma unroll 1
             for (int c0 = 0; c0 < kUmma2Tok; c0 += 32) {
                 if (m0 + c0 >= a.M) break;
                 if (((c0 >> 5) & 1) != set) continue;       // the two warp sets share the token chunks
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
-                tmem_wait_ld();
+                if (ok) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + c0, r);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int m = m0 + c0 + i;
-                    if (m < a.M) yp[(size_t)m * a.N] = __float2half_rn(__uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i)
+                        sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
                 }
+                named_bar_sync(bar_id, 128);
+                if (ok) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int piece = tq + 128 * t, row = piece >> 4, c16 = piece & 15;
+                        const int m = m0 + c0 + row;
+                        if (m < a.M) {
+                            const uint4 v = lds128(stg + (uint32_t)piece * 16u);
+                            *reinterpret_cast<uint4 *>(a.y + (size_t)m * a.N + (size_t)p * kPanel + c16 * 8) = v;
+                        }
+                    }
+                }
+                named_bar_sync(bar_id, 128);
             }
         }
     }
