@@ -151,8 +151,15 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP);
     constexpr uint32_t kAcol = NP * TOK;                   // accumulators first, then the A rings (panel-major)
 
+    // A warp set jumps 2 SETS - 1 blocks from one K group to its next.  Its parity wait on an A stage is only
+    // unambiguous if that jump is no longer than the A ring: then the wait it passed for the previous block implies
+    // that the stage's completion before the awaited one has already happened.
+    static_assert(SETS == 1 || NA >= 2 * SETS - 1, "A ring too short for this many dequant warp sets");
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_aempty = base + 192;
+    // full/empty: shared-memory ring slots (TMA landed / packed weights read by the dequant warps); a_full: A stage
+    // written; done[b & 7]: the MMAs of K64 block b have completed (one tcgen05.commit per block tells the producer
+    // that the slot's x tile and the dequant warps that the block's A stage may be overwritten)
+    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_done = base + 192;
     const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
     const uint32_t ring = base + 1024;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -169,12 +176,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, NP * kUmmaDequantWarps + 1);   // dequant warps read W, the MMA reads x
+            mbar_init(bar_empty + 8 * s, NP * kUmmaDequantWarps);       // the dequant warps that read the slot's W
         }
-        for (int s = 0; s < NP * NA; ++s) {
-            mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
-            mbar_init(bar_aempty + 8 * s, 1);
-        }
+        for (int s = 0; s < NP * NA; ++s) mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
+        for (int s = 0; s < 8; ++s) mbar_init(bar_done + 8 * s, 1);
         mbar_init(bar_dfull, 1);
         fence_barrier_init();
         fence_proxy_async();
@@ -219,7 +224,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             for (int b = 0; b < NB; ++b) {
                 const uint32_t bar = bar_full + 8 * s;
                 if (b >= NS) {
+                    // the slot's previous block b - NS: its weights have been read and its MMAs have completed
                     if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
+                    if (!mbar_wait(bar_done + 8 * ((b - NS) & 7), (uint32_t)(((b - NS) >> 3) & 1))) break;
                     issue_w(b, s);
                 }
                 mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
@@ -231,12 +238,14 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // ---------------------------------------------------------------- MMA issue (one thread)
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_f16(128, TOK);
+            // One thread, and every instruction it issues costs it 60-110 cycles (a tcgen05.mma about 60, a commit
+            // about 80, a barrier wait about 100 even when the barrier is ready), so the loop is kept to one wait
+            // per panel, the four MMAs and one commit per K64 block.  It does not wait for the slot's TMA data
+            // itself: the dequant warps did before they wrote the A stage, and their a_full arrival orders it.
             int s = 0, sa = 0;
-            uint32_t ph = 0, pha = 0;
+            uint32_t pha = 0;
             bool ok = true;
             for (int b = 0; b < NB && ok; ++b) {
-                ok = mbar_wait(bar_full + 8 * s, ph);
-                if (!ok) break;
                 const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
@@ -247,11 +256,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
                         umma_f16_ts(tmem_base + j * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
                                     bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)((b | kk) != 0));
-                    umma_commit(bar_aempty + 8 * (j * NA + sa));   // this A stage may be overwritten
                 }
                 if (!ok) break;
-                umma_commit(bar_empty + 8 * s);      // and so may the x tile of this stage
-                if (++s == NS) { s = 0; ph ^= 1u; }
+                umma_commit(bar_done + 8 * (b & 7));     // this block's A stage(s) and x tile may be overwritten
+                if (++s == NS) s = 0;
                 if (++sa == NA) { sa = 0; pha ^= 1u; }
             }
             umma_commit(bar_dfull);
@@ -273,7 +281,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1
         int b = 2 * set;
         int s = b % NS, sa = b % NA;
-        uint32_t ph = (uint32_t)(b / NS) & 1u, pha = (uint32_t)(b / NA) & 1u;
+        uint32_t ph = (uint32_t)(b / NS) & 1u;
         uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
@@ -305,8 +313,8 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
                     o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
                 }
-            if (b >= NA) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * (j * NA + sa), pha ^ 1u));
+            if (b >= NA) {     // the stage's previous block b - NA must have been multiplied
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((b - NA) & 7), (uint32_t)(((b - NA) >> 3) & 1)));
                 if (!ok) break;
                 tc_fence_after_sync();
             }
@@ -322,7 +330,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             s += step;
             while (s >= NS) { s -= NS; ph ^= 1u; }
             sa += step;
-            while (sa >= NA) { sa -= NA; pha ^= 1u; }
+            while (sa >= NA) sa -= NA;
         }
         // ---- epilogue: lane n of the accumulator holds y[m0 .. m0+TOK, 128 p + n]
         pdl_wait();
@@ -424,7 +432,7 @@ struct UmmaPlan {
 };
 
 // A-ring depth per panel: with two panels the 512 tensor-memory columns hold exactly 2 x (128 + 4 x 32)
-__host__ __device__ constexpr int umma_a_stages(int tok, int np) { return tok >= 128 ? 4 : 2; }
+__host__ __device__ constexpr int umma_a_stages(int tok, int np) { return tok >= 64 ? 4 : 3; }
 // resident CTAs per SM: tensor memory (512 columns) and shared memory allow this many
 __host__ __device__ constexpr int umma_ctas_per_sm(int tok, int np) { return (np > 1 || tok > 128) ? 1 : tok <= 32 ? 3 : 2; }
 
@@ -437,7 +445,7 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     const int tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M < 256 ? 128 : 256;
     const int panels = N / kPanel;
     const int np = 1;
-    const int sets = tok >= 128 ? 2 : 1;
+    const int sets = 2;
     const int G = K / kGroup, tiles = (panels / np) * ((M + tok - 1) / tok);
     const int stage = umma_stage_bytes(tok, np);
     const int cps_max = umma_ctas_per_sm(tok, np);
@@ -463,6 +471,8 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     int stages = (smem_cap - 2048) / stage;
     if (stages > 8) stages = 8;
     if (stages > blocks_per_cta) stages = blocks_per_cta;
+    // the same parity argument for the shared-memory ring: a warp set's jump of 2 sets - 1 blocks must fit in it
+    if (stages < 2 * sets - 1 && blocks_per_cta > 2) stages = 2 * sets - 1;
     while (S > 1 && stages * stage < tok * kPanel * 4) ++stages;   // the ring doubles as the fp32 partial tile
     pl.tok = tok;
     pl.np = np;
@@ -533,9 +543,9 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
                             (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.tok, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st) return st;
     switch (plan.tok) {
-    case 16: return launch_umma_tok<16, 1, 1>(args, w_map, x_map, plan, s);
-    case 32: return launch_umma_tok<32, 1, 1>(args, w_map, x_map, plan, s);
-    case 64: return launch_umma_tok<64, 1, 1>(args, w_map, x_map, plan, s);
+    case 16: return launch_umma_tok<16, 1, 2>(args, w_map, x_map, plan, s);
+    case 32: return launch_umma_tok<32, 1, 2>(args, w_map, x_map, plan, s);
+    case 64: return launch_umma_tok<64, 1, 2>(args, w_map, x_map, plan, s);
     case 128: return launch_umma_tok<128, 1, 2>(args, w_map, x_map, plan, s);
     case 256: return launch_umma_tok<256, 1, 2>(args, w_map, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
