@@ -156,10 +156,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     // that the stage's completion before the awaited one has already happened.
     static_assert(SETS == 1 || NA >= 2 * SETS - 1, "A ring too short for this many dequant warp sets");
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // full/empty: shared-memory ring slots (TMA landed / packed weights read by the dequant warps); a_full: A stage
-    // written; done[b & 7]: the MMAs of K64 block b have completed (one tcgen05.commit per block tells the producer
-    // that the slot's x tile and the dequant warps that the block's A stage may be overwritten)
-    const uint32_t bar_full = base, bar_empty = base + 64, bar_afull = base + 128, bar_done = base + 192;
+    // full[s]: the TMA data of ring slot s has landed; a_full: an A stage has been written; done[b & 7]: the MMAs of
+    // K64 block b have completed (one tcgen05.commit per block tells the producer that the block's ring slot and the
+    // dequant warps that its A stage may be overwritten)
+    const uint32_t bar_full = base, bar_afull = base + 128, bar_done = base + 192;
     const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
     const uint32_t ring = base + 1024;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -176,7 +176,6 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, NP * kUmmaDequantWarps);       // the dequant warps that read the slot's W
         }
         for (int s = 0; s < NP * NA; ++s) mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
         for (int s = 0; s < 8; ++s) mbar_init(bar_done + 8 * s, 1);
@@ -199,10 +198,13 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         if (lane == 0) {
             tma_prefetch_descriptor(&w_map);
             tma_prefetch_descriptor(&x_map);
+            // bytes of packed weights (+ the group's scales and zeros with its first block) that block b brings
+            auto w_bytes = [&](int b) {
+                return (uint32_t)(NP * (kUmmaWBlockBytes + ((b & 1) == 0 ? kItemSBytes + kItemZBytes : 0)));
+            };
             auto issue_w = [&](int b, int s) {
                 const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
                 const bool first_of_group = (b & 1) == 0;
-                mbar_expect_tx(bar, NP * (kUmmaWBlockBytes + (first_of_group ? kItemSBytes + kItemZBytes : 0)));
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     const int p = p0 + j;
@@ -218,20 +220,27 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 }
             };
             const int n_pre = NB < NS ? NB : NS;
-            for (int b = 0; b < n_pre; ++b) issue_w(b, b);   // weights do not depend on earlier kernels
+            for (int b = 0; b < n_pre; ++b) {                // weights do not depend on earlier kernels
+                mbar_expect_tx(bar_full + 8 * b, w_bytes(b));
+                issue_w(b, b);
+            }
             pdl_wait();
-            int s = 0, round = 0;
+            // Every instruction of this thread (a wait, an expect, a copy) costs it about 0.1 us, which bounds
+            // small token tiles, so a refill is one wait, one arrive-and-expect and the copies.  The slot is free
+            // once the MMAs of its previous block b - NS have completed: that also means that its packed weights
+            // were read (the A stage those MMAs used was written from them).
+            int s = 0;
             for (int b = 0; b < NB; ++b) {
                 const uint32_t bar = bar_full + 8 * s;
                 if (b >= NS) {
-                    // the slot's previous block b - NS: its weights have been read and its MMAs have completed
-                    if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
                     if (!mbar_wait(bar_done + 8 * ((b - NS) & 7), (uint32_t)(((b - NS) >> 3) & 1))) break;
+                    mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128) + w_bytes(b));
                     issue_w(b, s);
+                } else {
+                    mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
                 }
-                mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
                 tma_load_2d(ring + s * kStage, &x_map, (b_first + b) * kUmmaBlockK, m0, bar);
-                if (++s == NS) { s = 0; ++round; }
+                if (++s == NS) s = 0;
             }
         }
     } else if (warp == 1) {
@@ -322,10 +331,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar_afull + 8 * (j * NA + sa));
-                mbar_arrive(bar_empty + 8 * s);
-            }
+            if (lane == 0) mbar_arrive(bar_afull + 8 * (j * NA + sa));
             const int step = (b & 1) ? 2 * SETS - 1 : 1;   // to this set's next block
             s += step;
             while (s >= NS) { s -= NS; ph ^= 1u; }
