@@ -128,6 +128,16 @@ struct UmmaArgs {
     int stages;             // shared-memory ring depth
 };
 
+// K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
+// producer thread) except for 128-token tiles, where two CTAs share an SM and group-sized slots would leave each
+// a ring of only two
+__host__ __device__ constexpr int umma_blocks_per_slot(int TOK) { return TOK == 128 ? 1 : 2; }
+// one ring slot: x tile(s), packed weights of each panel, the group's scales and zeros
+__host__ __device__ constexpr int umma_slot_bytes(int TOK, int NP)
+{
+    return (umma_blocks_per_slot(TOK) * (TOK * 128 + NP * kUmmaWBlockBytes) + NP * (kItemSBytes + kItemZBytes) + 1023) & ~1023;
+}
+// one K64 block per slot (the CTA-pair kernel)
 __host__ __device__ constexpr int umma_stage_bytes(int TOK, int NP)
 {
     return (TOK * 128 + NP * (kUmmaWBlockBytes + kItemSBytes + kItemZBytes) + 1023) & ~1023;
@@ -145,9 +155,11 @@ __global__ void __launch_bounds__(umma_threads(NP, SETS), (NP > 1 || TOK > 128) 
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
-    constexpr int kStage = umma_stage_bytes(TOK, NP);
-    // stage: [x tile][W block of each panel][scales of each panel][zeros of each panel]
-    constexpr int kOffW = TOK * 128, kOffS = kOffW + NP * kUmmaWBlockBytes, kOffZ = kOffS + NP * kItemSBytes;
+    constexpr int kStage = umma_slot_bytes(TOK, NP);
+    // ring slot = BPS K64 blocks: [x tile of each block][W blocks of each panel][scales][zeros]
+    constexpr int BPS = umma_blocks_per_slot(TOK);
+    constexpr int kXTile = TOK * 128;
+    constexpr int kOffW = BPS * kXTile, kOffS = kOffW + NP * BPS * kUmmaWBlockBytes, kOffZ = kOffS + NP * kItemSBytes;
     constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP);
     constexpr uint32_t kAcol = NP * TOK;                   // accumulators first, then the A rings (panel-major)
 
@@ -198,48 +210,52 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         if (lane == 0) {
             tma_prefetch_descriptor(&w_map);
             tma_prefetch_descriptor(&x_map);
-            // bytes of packed weights (+ the group's scales and zeros with its first block) that block b brings
-            auto w_bytes = [&](int b) {
-                return (uint32_t)(NP * (kUmmaWBlockBytes + ((b & 1) == 0 ? kItemSBytes + kItemZBytes : 0)));
+            constexpr uint32_t kXBytes = BPS * kXTile;
+            const int NR = NB / BPS;                         // ring refills of this CTA
+            // bytes of packed weights (+ the group's scales and zeros with its first block) that refill i brings
+            auto w_bytes = [&](int i) {
+                return (uint32_t)(NP * (BPS * kUmmaWBlockBytes + ((i * BPS) % 2 == 0 ? kItemSBytes + kItemZBytes : 0)));
             };
-            auto issue_w = [&](int b, int s) {
+            auto issue_w = [&](int i, int s) {
                 const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
-                const bool first_of_group = (b & 1) == 0;
+                const int b = i * BPS;                       // first K64 block of the refill
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     const int p = p0 + j;
                     // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
-                    tma_load_2d(st + kOffW + j * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
-                    // scales and zeros travel with the group's first block; the dequant warps keep them in
-                    // registers for the second (every TMA operation costs the producer thread issue time)
-                    if (first_of_group) {
+                    tma_load_2d(st + kOffW + j * BPS * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
+                    if ((b & 1) == 0) {
                         const size_t t = (size_t)p * a.G + g0 + (b >> 1);
                         bulk_g2s(st + kOffS + j * kItemSBytes, a.scales + t * kItemSBytes, kItemSBytes, bar);
                         bulk_g2s(st + kOffZ + j * kItemZBytes, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
                     }
                 }
             };
-            const int n_pre = NB < NS ? NB : NS;
-            for (int b = 0; b < n_pre; ++b) {                // weights do not depend on earlier kernels
-                mbar_expect_tx(bar_full + 8 * b, w_bytes(b));
-                issue_w(b, b);
+            const int n_pre = NR < NS ? NR : NS;
+            for (int i = 0; i < n_pre; ++i) {                // weights do not depend on earlier kernels
+                mbar_expect_tx(bar_full + 8 * i, w_bytes(i));
+                issue_w(i, i);
             }
             pdl_wait();
             // Every instruction of this thread (a wait, an expect, a copy) costs it about 0.1 us, which bounds
-            // small token tiles, so a refill is one wait, one arrive-and-expect and the copies.  The slot is free
-            // once the MMAs of its previous block b - NS have completed: that also means that its packed weights
-            // were read (the A stage those MMAs used was written from them).
+            // the kernel when there are many of them per byte, so a ring slot holds a whole K group where shared
+            // memory allows and a refill is one wait, one arrive-and-expect and the copies.  The slot is free
+            // once the MMAs of its previous refill's last block have completed: that also means that its packed
+            // weights were read (the A stages those MMAs used were written from them).
             int s = 0;
-            for (int b = 0; b < NB; ++b) {
-                const uint32_t bar = bar_full + 8 * s;
-                if (b >= NS) {
-                    if (!mbar_wait(bar_done + 8 * ((b - NS) & 7), (uint32_t)(((b - NS) >> 3) & 1))) break;
-                    mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128) + w_bytes(b));
-                    issue_w(b, s);
+            for (int i = 0; i < NR; ++i) {
+                const uint32_t bar = bar_full + 8 * s, st = ring + s * kStage;
+                if (i >= NS) {
+                    const int c = (i - NS) * BPS + BPS - 1;
+                    if (!mbar_wait(bar_done + 8 * (c & 7), (uint32_t)((c >> 3) & 1))) break;
+                    mbar_arrive_expect_tx(bar, kXBytes + w_bytes(i));
+                    issue_w(i, s);
                 } else {
-                    mbar_arrive_expect_tx(bar, (uint32_t)(TOK * 128));
+                    mbar_arrive_expect_tx(bar, kXBytes);
                 }
-                tma_load_2d(ring + s * kStage, &x_map, (b_first + b) * kUmmaBlockK, m0, bar);
+#pragma unroll
+                for (int t = 0; t < BPS; ++t)
+                    tma_load_2d(st + t * kXTile, &x_map, (b_first + i * BPS + t) * kUmmaBlockK, m0, bar);
                 if (++s == NS) s = 0;
             }
         }
@@ -255,7 +271,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             uint32_t pha = 0;
             bool ok = true;
             for (int b = 0; b < NB && ok; ++b) {
-                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
+                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage + (b % BPS) * kXTile);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     ok = mbar_wait(bar_afull + 8 * (j * NA + sa), pha);
@@ -268,7 +284,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 }
                 if (!ok) break;
                 umma_commit(bar_done + 8 * (b & 7));     // this block's A stage(s) and x tile may be overwritten
-                if (++s == NS) s = 0;
+                if ((b % BPS) == BPS - 1 && ++s == NS) s = 0;
                 if (++sa == NA) { sa = 0; pha ^= 1u; }
             }
             umma_commit(bar_dfull);
@@ -284,19 +300,25 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // the column's 8 bytes (two words: rows +0..7 and +32..39) in each of the four 16-byte chunks
         uint32_t w_rd[4];
 #pragma unroll
-        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + j * kUmmaWBlockBytes + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
+        for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + j * BPS * kUmmaWBlockBytes + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
         const uint32_t s_rd = kOffS + j * kItemSBytes + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + j * kItemZBytes + 8 * u + g;
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-        // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1
+        // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1; block b lives in ring refill b / BPS
         int b = 2 * set;
-        int s = b % NS, sa = b % NA;
-        uint32_t ph = (uint32_t)(b / NS) & 1u;
+        int s = (b / BPS) % NS, sa = b % NA;
+        uint32_t ph = (uint32_t)((b / BPS) / NS) & 1u;
         uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
-            if (!ok) break;
+            if ((b % BPS) == 0) {
+                // A set skips the other sets' slots, so its parity wait on a slot is only unambiguous once the slot's
+                // previous refill is known to have landed: the MMAs of that refill's last block have completed.
+                const int c = (b / BPS - NS) * BPS + BPS - 1;
+                if (c > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * (c & 7), (uint32_t)((c >> 3) & 1)));
+                ok = ok && __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
+                if (!ok) break;
+            }
             if ((b & 1) == 0) {
                 uint32_t sh;
                 asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
@@ -306,9 +328,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 zlo = (z * 0x00010001u) | MAGIC_LO;
                 zhi = (z * 0x00100010u) | MAGIC_HI;
             }
+            const uint32_t wb = st + (b % BPS) * kUmmaWBlockBytes;
             uint2 wv[4];
 #pragma unroll
-            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
+            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(wb + w_rd[t4]);
             uint32_t r[32];
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -333,7 +356,8 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_afull + 8 * (j * NA + sa));
             const int step = (b & 1) ? 2 * SETS - 1 : 1;   // to this set's next block
-            s += step;
+            // and to that block's ring slot
+            s += (b + step) / BPS - b / BPS;
             while (s >= NS) { s -= NS; ph ^= 1u; }
             sa += step;
             while (sa >= NA) sa -= NA;
@@ -453,7 +477,7 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     const int np = 1;
     const int sets = 2;
     const int G = K / kGroup, tiles = (panels / np) * ((M + tok - 1) / tok);
-    const int stage = umma_stage_bytes(tok, np);
+    const int stage = umma_slot_bytes(tok, np);
     const int cps_max = umma_ctas_per_sm(tok, np);
     int best_S = 1;
     long long best_t = -1;
@@ -469,16 +493,15 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
         }
     }
     const int S = best_S;
-    const int blocks_per_cta = 2 * ((G + S - 1) / S);
+    const int groups_per_cta = (G + S - 1) / S;
     int per_sm = (tiles * S + sm_count - 1) / sm_count;
     if (per_sm > cps_max) per_sm = cps_max;
     const int smem_cap = (227 * 1024) / per_sm - 1024;
     const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;
     int stages = (smem_cap - 2048) / stage;
     if (stages > 8) stages = 8;
-    if (stages > blocks_per_cta) stages = blocks_per_cta;
-    // the same parity argument for the shared-memory ring: a warp set's jump of 2 sets - 1 blocks must fit in it
-    if (stages < 2 * sets - 1 && blocks_per_cta > 2) stages = 2 * sets - 1;
+    const int refills_per_cta = 2 * groups_per_cta / umma_blocks_per_slot(tok);
+    if (stages > refills_per_cta) stages = refills_per_cta;
     while (S > 1 && stages * stage < tok * kPanel * 4) ++stages;   // the ring doubles as the fp32 partial tile
     pl.tok = tok;
     pl.np = np;
@@ -538,10 +561,11 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
-    // packed weights as rows of 64 bytes (16 words); a box is one K64 block of a panel (64 rows)
+    // packed weights as rows of 64 bytes (16 words); a box is one ring slot's K64 blocks of a panel (64 rows each)
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
-    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 64,
+    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16,
+                                (uint32_t)(64 * umma_blocks_per_slot(plan.tok)),
                                 CU_TENSOR_MAP_SWIZZLE_64B);
     if (st) return st;
     // x as [M rows, K halves]; a box is 64 k of one token tile

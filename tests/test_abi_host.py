@@ -119,7 +119,12 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
         assert pl.ctas == panels * -(-M // tok) * pl.cluster_size
         assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
         per_sm = min(-(-pl.ctas // sms), 1 if tok > 128 else 3 if tok <= 32 else 2)
-        assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024 and pl.stages >= 2
+        assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024
+        # ring slots hold one K group (one K64 block for 128-token tiles): never more than the CTA has, unless the
+        # ring must also hold the fp32 partial tile of the split-K exchange
+        assert 1 <= pl.stages <= 8
+        if pl.cluster_size == 1:
+            assert pl.stages <= (2 * G if tok == 128 else G)
         assert (per_sm + 1) * (pl.smem_bytes + 1024) > 227 * 1024
         if pl.cluster_size > 1:               # the ring doubles as the fp32 partial tile
             assert pl.smem_bytes - 2048 >= tok * 128 * 4
