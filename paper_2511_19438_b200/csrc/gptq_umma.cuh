@@ -29,6 +29,7 @@ __host__ __device__ constexpr int umma_threads(int NP, int SETS) { return 64 + 1
 constexpr int kUmmaDequantWarps = 4;     // per panel: one warp per 32 TMEM lanes
 constexpr int kUmmaBlockK = 64;
 constexpr int kUmmaWBlockBytes = 4096;   // packed weights of one K64 block of a panel
+constexpr int kUmmaDoneRing = 16;        // "block multiplied" barriers, indexed by block number mod 16
 
 // ---- tcgen05 wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols)
@@ -132,10 +133,10 @@ struct UmmaArgs {
 // producer thread) except for 128-token tiles, where two CTAs share an SM and group-sized slots would leave each
 // a ring of only two
 __host__ __device__ constexpr int umma_blocks_per_slot(int TOK) { return TOK == 128 ? 1 : 2; }
-// one ring slot: x tile(s), packed weights of each panel, the group's scales and zeros
+// one ring slot: x tile(s) and packed weights of each panel (scales and zeros do not pass through shared memory)
 __host__ __device__ constexpr int umma_slot_bytes(int TOK, int NP)
 {
-    return (umma_blocks_per_slot(TOK) * (TOK * 128 + NP * kUmmaWBlockBytes) + NP * (kItemSBytes + kItemZBytes) + 1023) & ~1023;
+    return (umma_blocks_per_slot(TOK) * (TOK * 128 + NP * kUmmaWBlockBytes) + 1023) & ~1023;
 }
 // one K64 block per slot (the CTA-pair kernel)
 __host__ __device__ constexpr int umma_stage_bytes(int TOK, int NP)
@@ -156,10 +157,10 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
 {
     extern __shared__ uint8_t smem_raw[];
     constexpr int kStage = umma_slot_bytes(TOK, NP);
-    // ring slot = BPS K64 blocks: [x tile of each block][W blocks of each panel][scales][zeros]
+    // ring slot = BPS K64 blocks: [x tile of each block][W blocks of each panel]
     constexpr int BPS = umma_blocks_per_slot(TOK);
     constexpr int kXTile = TOK * 128;
-    constexpr int kOffW = BPS * kXTile, kOffS = kOffW + NP * BPS * kUmmaWBlockBytes, kOffZ = kOffS + NP * kItemSBytes;
+    constexpr int kOffW = BPS * kXTile;
     constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP);
     constexpr uint32_t kAcol = NP * TOK;                   // accumulators first, then the A rings (panel-major)
 
@@ -168,10 +169,11 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     // that the stage's completion before the awaited one has already happened.
     static_assert(SETS == 1 || NA >= 2 * SETS - 1, "A ring too short for this many dequant warp sets");
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // full[s]: the TMA data of ring slot s has landed; a_full: an A stage has been written; done[b & 7]: the MMAs of
-    // K64 block b have completed (one tcgen05.commit per block tells the producer that the block's ring slot and the
-    // dequant warps that its A stage may be overwritten)
-    const uint32_t bar_full = base, bar_afull = base + 128, bar_done = base + 192;
+    // full[s]: the TMA data of ring slot s has landed; a_full: an A stage has been written; done[b mod 16]: the MMAs
+    // of K64 block b have completed (one tcgen05.commit per block tells the producer that the block's ring slot and
+    // the dequant warps that its A stage may be overwritten).  A parity wait for block c must look at done[c mod 16]
+    // before block c + 16 completes, so fewer than 16 blocks may be in the ring at once (the planner sees to that).
+    const uint32_t bar_full = base, bar_afull = base + 128, bar_done = base + 320;
     const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
     const uint32_t ring = base + 1024;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -190,7 +192,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             mbar_init(bar_full + 8 * s, 1);
         }
         for (int s = 0; s < NP * NA; ++s) mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
-        for (int s = 0; s < 8; ++s) mbar_init(bar_done + 8 * s, 1);
+        for (int s = 0; s < kUmmaDoneRing; ++s) mbar_init(bar_done + 8 * s, 1);
         mbar_init(bar_dfull, 1);
         fence_barrier_init();
         fence_proxy_async();
@@ -212,28 +214,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             tma_prefetch_descriptor(&x_map);
             constexpr uint32_t kXBytes = BPS * kXTile;
             const int NR = NB / BPS;                         // ring refills of this CTA
-            // bytes of packed weights (+ the group's scales and zeros with its first block) that refill i brings
-            auto w_bytes = [&](int i) {
-                return (uint32_t)(NP * (BPS * kUmmaWBlockBytes + ((i * BPS) % 2 == 0 ? kItemSBytes + kItemZBytes : 0)));
-            };
+            constexpr uint32_t kWBytes = NP * BPS * kUmmaWBlockBytes;
+            // the packed weights of refill i (scales and zeros are read by the dequant warps themselves)
             auto issue_w = [&](int i, int s) {
                 const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
                 const int b = i * BPS;                       // first K64 block of the refill
 #pragma unroll
-                for (int j = 0; j < NP; ++j) {
-                    const int p = p0 + j;
+                for (int j = 0; j < NP; ++j)
                     // packed weights viewed as rows of 64 bytes; block b of panel p starts at row (2 G p + b) * 64
-                    tma_load_2d(st + kOffW + j * BPS * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * p + b_first + b) * 64, bar);
-                    if ((b & 1) == 0) {
-                        const size_t t = (size_t)p * a.G + g0 + (b >> 1);
-                        bulk_g2s(st + kOffS + j * kItemSBytes, a.scales + t * kItemSBytes, kItemSBytes, bar);
-                        bulk_g2s(st + kOffZ + j * kItemZBytes, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
-                    }
-                }
+                    tma_load_2d(st + kOffW + j * BPS * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * (p0 + j) + b_first + b) * 64, bar);
             };
             const int n_pre = NR < NS ? NR : NS;
             for (int i = 0; i < n_pre; ++i) {                // weights do not depend on earlier kernels
-                mbar_expect_tx(bar_full + 8 * i, w_bytes(i));
+                mbar_expect_tx(bar_full + 8 * i, kWBytes);
                 issue_w(i, i);
             }
             pdl_wait();
@@ -247,15 +240,13 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 const uint32_t bar = bar_full + 8 * s, st = ring + s * kStage;
                 if (i >= NS) {
                     const int c = (i - NS) * BPS + BPS - 1;
-                    if (!mbar_wait(bar_done + 8 * (c & 7), (uint32_t)((c >> 3) & 1))) break;
-                    mbar_arrive_expect_tx(bar, kXBytes + w_bytes(i));
+                    if (!mbar_wait(bar_done + 8 * (c & (kUmmaDoneRing - 1)), (uint32_t)((c / kUmmaDoneRing) & 1))) break;
+                    mbar_arrive_expect_tx(bar, kXBytes + kWBytes);
                     issue_w(i, s);
                 } else {
                     mbar_arrive_expect_tx(bar, kXBytes);
                 }
-#pragma unroll
-                for (int t = 0; t < BPS; ++t)
-                    tma_load_2d(st + t * kXTile, &x_map, (b_first + i * BPS + t) * kUmmaBlockK, m0, bar);
+                tma_load_3d(st, &x_map, 0, m0, b_first + i * BPS, bar);   // the refill's BPS x tiles in one copy
                 if (++s == NS) s = 0;
             }
         }
@@ -283,7 +274,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                                     bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)((b | kk) != 0));
                 }
                 if (!ok) break;
-                umma_commit(bar_done + 8 * (b & 7));     // this block's A stage(s) and x tile may be overwritten
+                umma_commit(bar_done + 8 * (b & (kUmmaDoneRing - 1)));     // this block's A stage(s) and x tile may be overwritten
                 if ((b % BPS) == BPS - 1 && ++s == NS) s = 0;
                 if (++sa == NA) { sa = 0; pha ^= 1u; }
             }
@@ -301,7 +292,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         uint32_t w_rd[4];
 #pragma unroll
         for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + j * BPS * kUmmaWBlockBytes + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
-        const uint32_t s_rd = kOffS + j * kItemSBytes + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + j * kItemZBytes + 8 * u + g;
+        // The column's scale and zero point of a group come straight from global memory (2 bytes and a nibble per
+        // lane: 64 + 16 bytes per warp), fetched one group ahead into registers, which spares the producer thread two
+        // copies per group.  In the tiled layout the pair (column, column + 8) is adjacent.
+        const uint8_t *s_gl = a.scales + ((size_t)p * a.G + g0) * kItemSBytes + (16 * u + 2 * g + h) * 2;
+        const uint8_t *z_gl = a.qzeros + ((size_t)p * a.G + g0) * kItemZBytes + 8 * u + g;
+        auto load_sz = [&](int gg, uint32_t &sc, uint32_t &zb) {
+            // through L2 only: this kernel may start while its predecessor still runs, and the buffers may have been
+            // rewritten since an earlier kernel left lines of them in this SM's L1
+            sc = __ldcg(reinterpret_cast<const unsigned short *>(s_gl + (size_t)gg * kItemSBytes));
+            zb = __ldcg(z_gl + (size_t)gg * kItemZBytes);
+        };
+        uint32_t sc_next = 0, zb_next = 0;
+        if (2 * set < NB) load_sz(set, sc_next, zb_next);
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
         // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1; block b lives in ring refill b / BPS
         int b = 2 * set;
@@ -315,18 +318,16 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 // A set skips the other sets' slots, so its parity wait on a slot is only unambiguous once the slot's
                 // previous refill is known to have landed: the MMAs of that refill's last block have completed.
                 const int c = (b / BPS - NS) * BPS + BPS - 1;
-                if (c > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * (c & 7), (uint32_t)((c >> 3) & 1)));
+                if (c > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * (c & (kUmmaDoneRing - 1)), (uint32_t)((c / kUmmaDoneRing) & 1)));
                 ok = ok && __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
                 if (!ok) break;
             }
             if ((b & 1) == 0) {
-                uint32_t sh;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
-                s2 = sh * 0x00010001u;
-                const uint32_t zb = lds8(st + z_rd);
-                const uint32_t z = h ? (zb >> 4) : (zb & 15u);
+                s2 = sc_next * 0x00010001u;
+                const uint32_t z = h ? (zb_next >> 4) : (zb_next & 15u);
                 zlo = (z * 0x00010001u) | MAGIC_LO;
                 zhi = (z * 0x00100010u) | MAGIC_HI;
+                if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next group
             }
             const uint32_t wb = st + (b % BPS) * kUmmaWBlockBytes;
             uint2 wv[4];
@@ -346,7 +347,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
                 }
             if (b >= NA) {     // the stage's previous block b - NA must have been multiplied
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((b - NA) & 7), (uint32_t)(((b - NA) >> 3) & 1)));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((b - NA) & (kUmmaDoneRing - 1)), (uint32_t)(((b - NA) / kUmmaDoneRing) & 1)));
                 if (!ok) break;
                 tc_fence_after_sync();
             }
@@ -500,6 +501,8 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;
     int stages = (smem_cap - 2048) / stage;
     if (stages > 8) stages = 8;
+    // fewer blocks in the ring than "block multiplied" barriers (see the kernel)
+    if (stages * umma_blocks_per_slot(tok) >= kUmmaDoneRing) stages = (kUmmaDoneRing - 1) / umma_blocks_per_slot(tok);
     const int refills_per_cta = 2 * groups_per_cta / umma_blocks_per_slot(tok);
     if (stages > refills_per_cta) stages = refills_per_cta;
     while (S > 1 && stages * stage < tok * kPanel * 4) ++stages;   // the ring doubles as the fp32 partial tile
@@ -561,6 +564,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
+    if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;
     // packed weights as rows of 64 bytes (16 words); a box is one ring slot's K64 blocks of a panel (64 rows each)
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
@@ -568,9 +572,9 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
                                 (uint32_t)(64 * umma_blocks_per_slot(plan.tok)),
                                 CU_TENSOR_MAP_SWIZZLE_64B);
     if (st) return st;
-    // x as [M rows, K halves]; a box is 64 k of one token tile
-    st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
-                            (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.tok, CU_TENSOR_MAP_SWIZZLE_128B);
+    // x as K / 64 tiles of [M rows, 64 k]; a box is one ring slot's tiles of one token tile
+    st = make_tensor_map_ktiles(&x_map, x, (uint64_t)K, (uint64_t)M, (uint32_t)plan.tok,
+                                (uint32_t)umma_blocks_per_slot(plan.tok));
     if (st) return st;
     switch (plan.tok) {
     case 16: return launch_umma_tok<16, 1, 2>(args, w_map, x_map, plan, s);
