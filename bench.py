@@ -190,9 +190,14 @@ def step_bytes_flops(spec, layers):
     return b, f
 
 
-def launches_per_gemm(spec, M):
-    """Kernels one gptq_gemm call launches: the matmul, plus the x gather with act-order."""
-    return 1 + (1 if spec["act_order"] else 0)
+def launches_per_gemm(spec, M, name, sm_count):
+    """Kernels one gptq_gemm call launches: the matmul (two launches when the tcgen05 kernel's last wave is split
+    along K), plus the x gather with act-order."""
+    from paper_2511_19438_b200 import binding as B
+    K, N = spec["shapes"][name]
+    st, pl = B.gptq_plan(M, N, K, wl.GROUP_SIZE, 1 if spec["act_order"] else 0, sm_count)
+    assert st == B.GPTQ_OK
+    return 1 + (1 if pl.tail_ctas > 0 else 0) + (1 if spec["act_order"] else 0)
 
 
 def kernel_of(M):
@@ -202,9 +207,9 @@ def kernel_of(M):
     if M <= 16:
         return "splitk_kernel<2>"
     if M <= 32:
-        return "umma_kernel<32,2,1,1>"
+        return "umma_kernel<32,3,1,2>"
     if M <= 64:
-        return "umma_kernel<64,2,1,1>"
+        return "umma_kernel<64,4,1,2>"
     if M < 256:
         return "umma_kernel<128,4,1,2>"
     return "umma_kernel<256,4,1,2>"
@@ -484,7 +489,8 @@ def main():
         step_bytes, step_flops = sum(bytes_m.values()), sum(flops_m.values())
         value = whole_job_value(spec, world, step_bytes, step_flops, args.steps, total_ms)
         e2e_value = whole_job_value(spec, world, step_bytes, step_flops, e2e_steps, e2e_ms)
-        launches_step = sum(launches_per_gemm(spec, M) * len(per_m[M]) for M in Ms)
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        launches_step = sum(launches_per_gemm(spec, M, name, sms) for M in Ms for (_D, _x, _y, name) in per_m[M])
         per_m_report = {}
         for M in Ms:
             s = seg_ms[M] / 1e3

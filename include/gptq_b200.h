@@ -191,7 +191,10 @@ typedef struct {
     int split_panels; /* panels whose K range is shared by several CTAs */
     int smem_bytes;   /* dynamic shared memory per CTA */
     size_t workspace_bytes;
-    int cluster_size; /* CTAs that share one panel (kernel 1); 1 for kernel 3 */
+    int cluster_size; /* CTAs that share one panel (kernel 1) or one output tile (kernel 2); 1 for kernel 3 */
+    int tail_ctas;    /* kernel 2 only: grid of a second launch that takes the tiles of a partly filled last
+                         wave and splits K over clusters (`ctas` is then the first launch alone); 0 = none */
+    int tail_cluster_size; /* cluster size of that second launch (1 when there is none) */
 } gptq_plan_t;
 
 /* How gptq_gemm would launch this problem on a GPU with sm_count SMs. */

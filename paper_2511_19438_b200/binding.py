@@ -39,6 +39,7 @@ class gptq_plan_t(ctypes.Structure):
         ("stages", ctypes.c_int), ("ctas", ctypes.c_int), ("items", ctypes.c_int),
         ("split_panels", ctypes.c_int), ("smem_bytes", ctypes.c_int),
         ("workspace_bytes", ctypes.c_size_t), ("cluster_size", ctypes.c_int),
+        ("tail_ctas", ctypes.c_int), ("tail_cluster_size", ctypes.c_int),
     ]
 
 

@@ -224,6 +224,8 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
         out->smem_bytes = up.smem_bytes;
         out->workspace_bytes = gemm_workspace_need(M, K, act_order);
         out->cluster_size = up.S;
+        out->tail_ctas = up.tail_tiles * up.tail_S;
+        out->tail_cluster_size = up.tail_S;
         out->split_panels = up.S > 1 ? N / kPanel : 0;
         return GPTQ_OK;
     }
@@ -239,6 +241,8 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     out->smem_bytes = pl.smem_bytes;
     out->workspace_bytes = gemm_workspace_need(M, K, act_order);
     out->cluster_size = pl.S;
+    out->tail_ctas = 0;
+    out->tail_cluster_size = 1;
     return GPTQ_OK;
 }
 
@@ -261,6 +265,8 @@ int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm
     out->smem_bytes = gp.sk.smem_bytes;
     out->workspace_bytes = gp.workspace_bytes;
     out->cluster_size = 1;
+    out->tail_ctas = 0;
+    out->tail_cluster_size = 1;
     return GPTQ_OK;
 }
 

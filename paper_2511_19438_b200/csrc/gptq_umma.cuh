@@ -120,12 +120,23 @@ __device__ __forceinline__ void sts_f16(uint32_t addr, __half v)
     asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(v)) : "memory");
 }
 
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(addr)
+                 : "memory");
+    return v;
+}
+
 struct UmmaArgs {
     const uint8_t *scales;  // tiled
     const uint8_t *qzeros;  // tiled
     __half *y;              // [M, N]
     int M, N, K, G;
     int S;                  // CTAs that share one output tile along K (cluster size)
+    int tile0;              // first output tile of this launch (a matmul may take a main and a tail launch)
     int stages;             // shared-memory ring depth
 };
 
@@ -180,7 +191,8 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     const int NS = a.stages;
     const int panels = a.N / kPanel;
     const int S = a.S;
-    const int tile = blockIdx.x / S, rank = blockIdx.x - tile * S;      // cluster = the S CTAs of one tile
+    const int cl = blockIdx.x / S, rank = blockIdx.x - cl * S;          // cluster = the S CTAs of one tile
+    const int tile = cl + a.tile0;
     const int ptiles = panels / NP;
     const int mt = tile / ptiles, p0 = (tile - mt * ptiles) * NP;       // first panel; neighbours share the x tile
     const int m0 = mt * TOK;
@@ -426,17 +438,27 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             const int p = p0;   // split-K runs with one panel per CTA (NP == 1)
             const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
             const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
-            for (int idx = threadIdx.x - 64; idx < rows * width; idx += 128 * NP * SETS) {
-                const int m = idx / width, cc = c_lo + idx - m * width;
+            const int w4 = width >> 2;      // width is 16, 32 or 64: four columns (16 bytes) per thread and step
+            for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
+                const int m = idx / w4, cc = c_lo + 4 * (idx - m * w4);
                 const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
-                float v[8];
+                float4 v[8];
 #pragma unroll
                 for (int qq = 0; qq < 8; ++qq)
-                    v[qq] = qq < S ? ld_cluster_f32(map_to_cluster_rank(local, (uint32_t)qq)) : 0.f;
-                float sum = 0.f;
+                    v[qq] = qq < S ? ld_cluster_f32x4(map_to_cluster_rank(local, (uint32_t)qq)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int qq = 0; qq < 8; ++qq) sum += v[qq];   // rank order
-                a.y[(size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc] = __float2half_rn(sum);
+                for (int qq = 0; qq < 8; ++qq) {   // rank order
+                    sum.x += v[qq].x;
+                    sum.y += v[qq].y;
+                    sum.z += v[qq].z;
+                    sum.w += v[qq].w;
+                }
+                const __half2 lo = __floats2half2_rn(sum.x, sum.y), hi = __floats2half2_rn(sum.z, sum.w);
+                uint2 out;
+                out.x = *reinterpret_cast<const uint32_t *>(&lo);
+                out.y = *reinterpret_cast<const uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>(a.y + (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc) = out;
             }
         }
         // no CTA may exit (and free its shared memory) while a peer can still read its tile
@@ -458,8 +480,11 @@ struct UmmaPlan {
     int sets;       // dequant warp sets per panel
     int S;          // CTAs per output tile along K (cluster size)
     int stages;
-    int ctas;       // panel tiles * token tiles * S
+    int ctas;       // grid of the main launch: (tiles - tail_tiles) * S
     int smem_bytes;
+    // When the tiles fill the SMs more than once and the last wave would leave most SMs idle, that wave's tiles
+    // go to a second launch that splits K over clusters of tail_S CTAs (0 tiles: no second launch).
+    int tail_tiles, tail_S, tail_stages;
 };
 
 // A-ring depth per panel: with two panels the 512 tensor-memory columns hold exactly 2 x (128 + 4 x 32)
@@ -511,15 +536,33 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     pl.sets = sets;
     pl.S = S;
     pl.stages = stages;
-    pl.ctas = tiles * S;
     pl.smem_bytes = 2048 + stages * stage;
     if (pl.smem_bytes < smem_floor) pl.smem_bytes = smem_floor;
+    pl.tail_tiles = 0;
+    pl.tail_S = 1;
+    pl.tail_stages = stages;
+    const int slots = sm_count * cps_max;              // CTAs resident at once
+    if (S == 1 && tiles > slots && tiles % slots != 0) {
+        const int r = tiles % slots;
+        int ts = 1;
+        while (ts * 2 <= 8 && ts * 2 <= G && r * ts * 2 <= slots) ts *= 2;
+        int tstages = stages;
+        const int trefills = 2 * ((G + ts - 1) / ts) / umma_blocks_per_slot(tok);
+        if (tstages > trefills) tstages = trefills;
+        while (tstages * stage < tok * kPanel * 4) ++tstages;      // the ring doubles as the fp32 partial tile
+        if (ts > 1 && 2048 + tstages * stage <= pl.smem_bytes && tstages * umma_blocks_per_slot(tok) < kUmmaDoneRing) {
+            pl.tail_tiles = r;
+            pl.tail_S = ts;
+            pl.tail_stages = tstages;
+        }
+    }
+    pl.ctas = (tiles - pl.tail_tiles) * S;
     return pl;
 }
 
 template <int TOK, int NP, int SETS>
 static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
-                           const UmmaPlan &plan, cudaStream_t s)
+                           const UmmaPlan &plan, int ctas, cudaStream_t s)
 {
     auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS>;
     static int configured_smem[64] = {};
@@ -535,7 +578,7 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
         configured_smem[dev] = plan.smem_bytes;
     }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)plan.ctas);
+    cfg.gridDim = dim3((unsigned)ctas);
     cfg.blockDim = dim3(umma_threads(NP, SETS));
     cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
     cfg.stream = s;
@@ -543,7 +586,7 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = (unsigned)plan.S;
+    attr[1].val.clusterDim.x = (unsigned)args.S;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
@@ -576,14 +619,31 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     st = make_tensor_map_ktiles(&x_map, x, (uint64_t)K, (uint64_t)M, (uint32_t)plan.tok,
                                 (uint32_t)umma_blocks_per_slot(plan.tok));
     if (st) return st;
-    switch (plan.tok) {
-    case 16: return launch_umma_tok<16, 1, 2>(args, w_map, x_map, plan, s);
-    case 32: return launch_umma_tok<32, 1, 2>(args, w_map, x_map, plan, s);
-    case 64: return launch_umma_tok<64, 1, 2>(args, w_map, x_map, plan, s);
-    case 128: return launch_umma_tok<128, 1, 2>(args, w_map, x_map, plan, s);
-    case 256: return launch_umma_tok<256, 1, 2>(args, w_map, x_map, plan, s);
-    default: return GPTQ_ERR_UNSUPPORTED;
+    auto launch = [&](const UmmaArgs &la, int ctas) {
+        switch (plan.tok) {
+        case 16: return launch_umma_tok<16, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        case 256: return launch_umma_tok<256, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        default: return (int)GPTQ_ERR_UNSUPPORTED;
+        }
+    };
+    args.tile0 = 0;
+    if (plan.ctas > 0) {
+        st = launch(args, plan.ctas);
+        if (st) return st;
     }
+    if (plan.tail_tiles > 0) {
+        // the last, partly filled wave: the same kernel on clusters that split K, starting at the first tile the
+        // main launch left out
+        UmmaArgs ta = args;
+        ta.tile0 = plan.ctas / plan.S;
+        ta.S = plan.tail_S;
+        ta.stages = plan.tail_stages;
+        st = launch(ta, plan.tail_tiles * plan.tail_S);
+    }
+    return st;
 }
 
 }  // namespace gptq

@@ -116,9 +116,19 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
         tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M < 256 else 256
         assert pl.m_tile == tok and pl.m_chunks == 1
         assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
-        assert pl.ctas == panels * -(-M // tok) * pl.cluster_size
+        tiles = panels * -(-M // tok)
+        cps_max = 1 if tok > 128 else 3 if tok <= 32 else 2
+        if pl.tail_ctas:                      # the partly filled last wave goes to a K-split second launch
+            tail_tiles = tiles % (sms * cps_max)
+            assert pl.cluster_size == 1 and tiles > sms * cps_max and tail_tiles > 0
+            assert pl.tail_cluster_size in (2, 4, 8) and pl.tail_cluster_size <= G
+            assert pl.tail_ctas == tail_tiles * pl.tail_cluster_size <= sms * cps_max
+            assert pl.ctas == tiles - tail_tiles
+        else:
+            assert pl.tail_cluster_size == 1
+            assert pl.ctas == tiles * pl.cluster_size
         assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
-        per_sm = min(-(-pl.ctas // sms), 1 if tok > 128 else 3 if tok <= 32 else 2)
+        per_sm = min(-(-tiles * pl.cluster_size // sms), cps_max)
         assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024
         # ring slots hold one K group (one K64 block for 128-token tiles): never more than the CTA has, unless the
         # ring must also hold the fp32 partial tile of the split-K exchange
