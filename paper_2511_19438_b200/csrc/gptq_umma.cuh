@@ -5,17 +5,25 @@
 // M = 128 rows, one TMEM lane per weight column) and a tile of TOK tokens (the MMA's N).  x[M, K]
 // row-major is already the K-major B operand, so it goes from global memory to swizzled shared
 // memory by TMA and is read by the tensor core through a shared-memory descriptor.  The weights
-// need arithmetic, so they take another road: TMA brings the packed K64 block of the panel (4 KB,
-// 64-byte swizzle) to shared memory, four dequant warps (one per 32 TMEM lanes) read the eight
-// words of "their" column, turn nibbles into fp16 with lop3 (1024+q / 64+q), subtract the zero
-// (exact integer) and multiply by the group scale as packed half2, and write the 64 fp16 values
-// with tcgen05.st into a ring of A-operand stages in tensor memory.  One thread issues
-// tcgen05.mma (kind::f16, A from TMEM, B from shared memory, fp32 accumulator in TMEM) and
-// tcgen05.commit hands ring slots back through mbarriers.  At the end of the K loop the dequant
-// warps read the accumulator with tcgen05.ld, round once to fp16 and store y.
+// need arithmetic, so they take another road: TMA brings the packed weights of a K group of the
+// panel (8 KB, 64-byte swizzle) to shared memory, two sets of four dequant warps (one warp per 32
+// TMEM lanes, the sets taking alternate groups) read the eight words of "their" column per K64
+// block, turn nibbles into fp16 with lop3 (1024+q / 64+q), subtract the zero (exact integer) and
+// multiply by the group scale as packed half2 (scale and zero come straight from L2, one group
+// ahead), and write the 64 fp16 values with tcgen05.st into a ring of A-operand stages in tensor
+// memory.  One thread issues tcgen05.mma (kind::f16, A from TMEM, B from shared memory, fp32
+// accumulator in TMEM); one tcgen05.commit per K64 block tells everybody that the block's ring
+// slot and A stage are free again.  At the end of the K loop the dequant warps read the
+// accumulator with tcgen05.ld, round once to fp16, turn each 32-token chunk around through the
+// idle ring and store whole lines of y.
 //
-// Two CTAs fit on an SM (256 TMEM columns and <= 110 KB of shared memory each), so one CTA's
-// epilogue overlaps the other's main loop.  Every wait is bounded.
+// The two single threads (TMA producer, MMA issue) pay 60-110 cycles for every instruction, so
+// both loops are kept short: a ring refill is one wait, one arrive-and-expect, one weight copy and
+// one 3-D x copy per K group; an MMA step is one wait, four MMAs and one commit per K64 block.
+//
+// Small problems split K over a thread-block cluster (partial tiles meet through distributed
+// shared memory in rank order); when the tiles fill the SMs more than once, the partly filled
+// last wave is launched separately with such a split.  Every wait is bounded.
 #pragma once
 #include "gptq_common.cuh"
 #include "gptq_tma.cuh"
