@@ -137,6 +137,23 @@ def test_gemm_token_count_boundaries(M, act, ws):
     assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
 
 
+@pytest.mark.parametrize("K,M,act", [(512, 2040, False), (768, 1300, True)])
+def test_gemm_tail_wave_launch(K, M, act, ws):
+    """More 256-token tiles than the GPU holds at once, with a short last wave: those tiles run in a second launch
+    that splits K over clusters (gptq_plan reports it).  Full compare, ragged last token tile."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    tok_tiles = -(-M // 256)
+    panels = sms // tok_tiles + 1              # tiles = sms + (1 .. tok_tiles): a nearly empty last wave
+    N = 128 * panels
+    st, pl = B.gptq_plan(M, N, K, 128, int(act), sms)
+    assert st == B.GPTQ_OK and pl.kernel == 2 and pl.m_tile == 256
+    assert pl.tail_ctas > 0 and pl.tail_cluster_size >= 2 and pl.ctas == sms
+    L = wl.make_linear(K, N, seed=wl.seed_for("tail", K, N, act), act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("tail-x", K, M))
+    y, _ = run_gemm(L, x, ws)
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+
+
 @pytest.mark.parametrize("K,N,M,act", [(512, 256, 256, False), (1024, 512, 300, False), (640, 256, 513, True),
                                         (4096, 4096, 1024, False)])
 def test_gemm_on_cta_pairs(K, N, M, act, ws):
