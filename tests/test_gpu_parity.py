@@ -413,6 +413,46 @@ def test_graph_replayed_step_matches_oracle(ws):
         sampled_check(L, x_np, y.cpu().numpy(), 2000, seed=x_np.shape[0])
 
 
+@pytest.mark.parametrize("M", [1, 40, 2040])
+def test_dependent_chain_in_a_graph(M, ws):
+    """Two matmuls where the second reads what the first wrote, captured in a CUDA graph and replayed: every kernel starts
+    before its predecessor has finished (programmatic dependent launch) and must wait before it touches x or y.  At
+    M = 2040 the first matmul takes a main and a tail launch, so the second one's wait has to cover both."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    K1, N1, N2 = 512, 128 * (sms // 8 + 1), 256          # at M = 2040: eight token tiles x (sms / 8 + 1) panels
+    if M == 2040:
+        st, pl = B.gptq_plan(M, N1, K1, 128, 0, sms)
+        assert st == B.GPTQ_OK and pl.tail_ctas > 0
+    L1 = wl.make_linear(K1, N1, seed=wl.seed_for("chain", 1, M))
+    L2 = wl.make_linear(N1, N2, seed=wl.seed_for("chain", 2, M))
+    D1, D2 = H.upload_and_repack(L1), H.upload_and_repack(L2)
+    x_np = wl.make_x(M, K1, wl.seed_for("chain-x", M))
+    x = H.to_device(x_np)
+    y1 = torch.zeros((M, N1), dtype=torch.float16, device="cuda")
+    y2 = torch.zeros((M, N2), dtype=torch.float16, device="cuda")
+    ws.ensure_for(M, D1)
+    ws.ensure_for(M, D2)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        H.gemm(x, D1, y1)
+        H.gemm(y1, D2, y2)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(3):                    # back to back: the next round's first kernel overwrites y1 early
+                H.gemm(x, D1, y1)
+                H.gemm(y1, D2, y2)
+        y1.zero_()
+        y2.zero_()
+        g.replay()
+        stream.synchronize()
+    assert B.gptq_check_status() == B.GPTQ_OK
+    y1_np = y1.cpu().numpy()
+    assert_close(y1_np, oracle.gemm_f64(x_np, L1.qweight, L1.qzeros, L1.scales, None, 128), K1)
+    # the second matmul against the oracle on the first one's fp16 output, so that errors do not compound
+    assert_close(y2.cpu().numpy(), oracle.gemm_f64(y1_np, L2.qweight, L2.qzeros, L2.scales, None, 128), N1)
+
+
 @pytest.mark.parametrize("M", wl.STEP_M)
 def test_config5_decode_step_layers(M, ws):
     """Layers 0 and 31 of the 32-layer step (distinct seeded weights per layer)."""
