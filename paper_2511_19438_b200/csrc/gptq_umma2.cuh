@@ -21,6 +21,7 @@ constexpr int kUmma2Threads = 320;     // TMA warp, MMA/TMEM warp, two sets of f
 constexpr int kUmma2Tok = 256;         // tokens per pair tile (128 loaded by each CTA)
 constexpr int kUmma2AStages = 8;
 constexpr uint32_t kUmma2Cols = 512;   // accumulator 256 + A ring 8 x 32
+constexpr int kUmma2StageBytes = 2 * (kUmma2Tok / 2) * 128 + 2 * kUmmaWBlockBytes;   // one K group: two x half-tiles + 8 KB of W
 
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_slot, uint32_t cols)
 {
@@ -67,14 +68,17 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
 {
     extern __shared__ uint8_t smem_raw[];
     constexpr int kHalfTok = kUmma2Tok / 2;                 // tokens whose x rows this CTA loads
-    constexpr int kStage = umma_stage_bytes(kHalfTok, 1);
-    constexpr int kOffW = kHalfTok * 128, kOffS = kOffW + kUmmaWBlockBytes, kOffZ = kOffS + kItemSBytes;
+    // ring slot = one K group: [x half-tile of block 0][x half-tile of block 1][8 KB of packed weights]
+    constexpr int kXTile = kHalfTok * 128, kStage = kUmma2StageBytes, kOffW = 2 * kXTile;
     constexpr uint32_t kAcol = kUmma2Tok;                  // accumulator first, then the A ring
     constexpr int NA = kUmma2AStages, SETS = 2;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bar_full = base, bar_empty = base + 128, bar_afull = base + 256, bar_aempty = base + 320;   // <= 16 stages
-    const uint32_t bar_dfull = base + 384, tmem_slot = base + 392;
+    // full[s]: this CTA's TMA data of ring slot s has landed; a_full (the leader's copy is used): the A stage of a block
+    // is in tensor memory in both CTAs; done[b mod 16] (in both CTAs, by a multicast commit): the pair's MMAs of block b
+    // have completed - the block's ring slot (with its group's second block) and its A stage may be overwritten
+    const uint32_t bar_full = base, bar_afull = base + 128, bar_done = base + 320;
+    const uint32_t bar_dfull = base + 256, tmem_slot = base + 264;
     const uint32_t ring = base + 1024;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NS = a.stages;
@@ -85,14 +89,11 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
     const int NB = a.K / kUmmaBlockK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, kUmmaDequantWarps + 1);       // this CTA's dequant warps + the pair's MMA
-        }
+        for (int s = 0; s < NS; ++s) mbar_init(bar_full + 8 * s, 1);
+        for (int s = 0; s < kUmmaDoneRing; ++s) mbar_init(bar_done + 8 * s, 1);
         for (int s = 0; s < NA; ++s) {
             mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);           // leader's copy is used: its four warps arrive, the
                                                                        // peer's four send 4 bytes each (transaction count)
-            mbar_init(bar_aempty + 8 * s, 1);
         }
         mbar_init(bar_dfull, 1);
         fence_barrier_init();
@@ -111,33 +112,35 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
     const uint32_t tmem_base = lds32(tmem_slot);
     pdl_launch_dependents();
 
+    const int G = a.G;
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (one thread per CTA)
         if (lane == 0) {
             tma_prefetch_descriptor(&w_map);
             tma_prefetch_descriptor(&x_map);
-            auto issue_w = [&](int b, int s) {
-                const uint32_t st = ring + s * kStage, bar = bar_full + 8 * s;
-                mbar_expect_tx(bar, kUmmaWBlockBytes + kItemSBytes + kItemZBytes);
-                tma_load_2d(st + kOffW, &w_map, 0, (2 * a.G * p + b) * 64, bar);
-                const size_t t = (size_t)p * a.G + (b >> 1);
-                bulk_g2s(st + kOffS, a.scales + t * kItemSBytes, kItemSBytes, bar);
-                bulk_g2s(st + kOffZ, a.qzeros + t * kItemZBytes, kItemZBytes, bar);
-            };
-            const int n_pre = NB < NS ? NB : NS;
-            for (int b = 0; b < n_pre; ++b) issue_w(b, b);   // weights do not depend on earlier kernels
+            constexpr uint32_t kWBytes = 2 * kUmmaWBlockBytes, kXBytes = 2 * kXTile;
+            const int n_pre = G < NS ? G : NS;
+            for (int i = 0; i < n_pre; ++i) {                // weights do not depend on earlier kernels
+                mbar_expect_tx(bar_full + 8 * i, kWBytes);
+                tma_load_2d(ring + i * kStage + kOffW, &w_map, 0, (2 * G * p + 2 * i) * 64, bar_full + 8 * i);
+            }
             pdl_wait();
-            int s = 0, round = 0;
-            for (int b = 0; b < NB; ++b) {
-                const uint32_t bar = bar_full + 8 * s;
-                if (b >= NS) {
-                    if (!mbar_wait(bar_empty + 8 * s, (uint32_t)((round - 1) & 1))) break;
-                    issue_w(b, s);
+            // as in the single-CTA kernel: a refill is one wait (the pair's MMAs of the slot's previous group are
+            // done, which also means its weights were read), one arrive-and-expect and two copies
+            int s = 0;
+            for (int i = 0; i < G; ++i) {
+                const uint32_t bar = bar_full + 8 * s, st = ring + s * kStage;
+                if (i >= NS) {
+                    const int c = 2 * (i - NS) + 1;
+                    if (!mbar_wait(bar_done + 8 * (c & (kUmmaDoneRing - 1)), (uint32_t)((c / kUmmaDoneRing) & 1))) break;
+                    mbar_arrive_expect_tx(bar, kXBytes + kWBytes);
+                    tma_load_2d(st + kOffW, &w_map, 0, (2 * G * p + 2 * i) * 64, bar);
+                } else {
+                    mbar_arrive_expect_tx(bar, kXBytes);
                 }
-                // this CTA's half of the token tile: rows m0 + 128 rank .. + 127 (rows >= M read as zero)
-                mbar_arrive_expect_tx(bar, (uint32_t)(kHalfTok * 128));
-                tma_load_2d(ring + s * kStage, &x_map, b * kUmmaBlockK, m0 + rank * kHalfTok, bar);
-                if (++s == NS) { s = 0; ++round; }
+                // this CTA's half of the token tile: rows m0 + 128 rank .. + 127 (rows >= M read as zero), both K64 tiles
+                tma_load_3d(st, &x_map, 0, m0 + rank * kHalfTok, 2 * i, bar);
+                if (++s == NS) s = 0;
             }
         }
     } else if (warp == 1) {
@@ -145,21 +148,21 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = umma_idesc_f16(256, kUmma2Tok);
             int s = 0, sa = 0;
-            uint32_t ph = 0, pha = 0;
+            uint32_t pha = 0;
             bool ok = true;
             for (int b = 0; b < NB && ok; ++b) {
-                // own x half landed; both CTAs' A stages written (which implies the peer's x half landed too)
-                ok = mbar_wait(bar_full + 8 * s, ph) && mbar_wait_cluster(bar_afull + 8 * sa, pha);
+                // both CTAs' A stages written - which implies that both halves of the x tile have landed, since the
+                // dequant warps waited for their slot before they wrote
+                ok = mbar_wait_cluster(bar_afull + 8 * sa, pha);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage);
+                const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage + (b & 1) * kXTile);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     umma_f16_ts_pair(tmem_base, tmem_base + kAcol + sa * 32 + kk * 8, bdesc + (uint64_t)(kk * 2), idesc,
                                      (uint32_t)((b | kk) != 0));
-                umma_commit_pair(bar_aempty + 8 * sa, 3);   // both CTAs: this A stage may be overwritten
-                umma_commit_pair(bar_empty + 8 * s, 3);     // both CTAs: and so may the x tile of this stage
-                if (++s == NS) { s = 0; ph ^= 1u; }
+                umma_commit_pair(bar_done + 8 * (b & (kUmmaDoneRing - 1)), 3);   // both CTAs: block b has been multiplied
+                if ((b & 1) && ++s == NS) s = 0;
                 if (++sa == NA) { sa = 0; pha ^= 1u; }
             }
             umma_commit_pair(bar_dfull, 3);
@@ -167,35 +170,51 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
     } else {
         // ---------------------------------------------------------------- dequant warps, then epilogue
         const int q = warp & 3;                 // the 32 TMEM lanes this warp may touch
-        const int set = (warp - 2) >> 2;        // which K64 blocks: set, set + 2, ...
+        const int set = (warp - 2) >> 2;        // which K groups: set, set + 2, ...
         const int n = 32 * q + lane;            // weight column inside the panel = TMEM lane
         const int u = n >> 4, g = n & 7, h = (n >> 3) & 1;
         uint32_t w_rd[4];
 #pragma unroll
         for (int t4 = 0; t4 < 4; ++t4) w_rd[t4] = kOffW + (u * 8 + g) * 64 + ((uint32_t)(t4 ^ (g >> 1)) << 4) + 8 * h;
-        const uint32_t s_rd = kOffS + (16 * u + 2 * g + h) * 2, z_rd = kOffZ + 8 * u + g;
+        // scale and zero point of the lane's column: straight from L2, one group ahead
+        const uint8_t *s_gl = a.scales + (size_t)p * G * kItemSBytes + (16 * u + 2 * g + h) * 2;
+        const uint8_t *z_gl = a.qzeros + (size_t)p * G * kItemZBytes + 8 * u + g;
+        auto load_sz = [&](int gg, uint32_t &sc, uint32_t &zb) {
+            sc = __ldcg(reinterpret_cast<const unsigned short *>(s_gl + (size_t)gg * kItemSBytes));
+            zb = __ldcg(z_gl + (size_t)gg * kItemZBytes);
+        };
+        uint32_t sc_next = 0, zb_next = 0;
+        if (set < G) load_sz(set, sc_next, zb_next);
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
         // The peer's warps signal the leader's a_full barrier with a fire-and-forget 4-byte st.async that is counted
         // on the barrier's transaction count (a remote mbarrier.arrive holds the issuing thread up for hundreds of
         // cycles); the leader's warp 0 of the set arms those 16 bytes with its own arrival.
         const uint32_t leader_afull = map_to_cluster_rank(bar_afull, 0);
         const uint32_t leader_slot = map_to_cluster_rank(base + 512 + 4 * warp, 0);
-        int s = set % NS, sa = set % NA;
-        uint32_t ph = (uint32_t)(set / NS) & 1u, pha = (uint32_t)(set / NA) & 1u;
+        int b = 2 * set;
+        int s = set % NS, sa = b % NA;
+        uint32_t ph = (uint32_t)(set / NS) & 1u;
+        uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
         bool ok = true;
-        for (int b = set; b < NB && ok; b += SETS) {
+        for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
-            if (!ok) break;
-            uint32_t sh;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sh) : "r"(st + s_rd));
-            const uint32_t s2 = sh * 0x00010001u;
-            const uint32_t zb = lds8(st + z_rd);
-            const uint32_t z = h ? (zb >> 4) : (zb & 15u);
-            const uint32_t zlo = (z * 0x00010001u) | MAGIC_LO, zhi = (z * 0x00100010u) | MAGIC_HI;
+            if ((b & 1) == 0) {
+                // a set skips the other set's slots: its parity wait on a slot is unambiguous once the slot's previous
+                // refill is known to have landed, i.e. that group's last block has been multiplied
+                const int c = b - 2 * NS + 1;
+                if (c > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * (c & (kUmmaDoneRing - 1)), (uint32_t)((c / kUmmaDoneRing) & 1)));
+                ok = ok && __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
+                if (!ok) break;
+                s2 = sc_next * 0x00010001u;
+                const uint32_t z = h ? (zb_next >> 4) : (zb_next & 15u);
+                zlo = (z * 0x00010001u) | MAGIC_LO;
+                zhi = (z * 0x00100010u) | MAGIC_HI;
+                if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next group
+            }
+            const uint32_t wb = st + (b & 1) * kUmmaWBlockBytes;
             uint2 wv[4];
 #pragma unroll
-            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(st + w_rd[t4]);
+            for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(wb + w_rd[t4]);
             uint32_t r[32];
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -209,8 +228,8 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
                     o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
                     o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
                 }
-            if (b >= NA) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_aempty + 8 * sa, pha ^ 1u));
+            if (b >= NA) {     // the stage's previous block b - NA must have been multiplied
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((b - NA) & (kUmmaDoneRing - 1)), (uint32_t)(((b - NA) / kUmmaDoneRing) & 1)));
                 if (!ok) break;
                 tc_fence_after_sync();
             }
@@ -226,12 +245,14 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
                 } else {
                     st_async_f32(leader_slot, 0.f, leader_afull + 8 * sa);
                 }
-                mbar_arrive(bar_empty + 8 * s);               // the packed weights of this stage have been read
             }
-            s += SETS;
-            if (s >= NS) { s -= NS; ph ^= 1u; }
-            sa += SETS;
-            if (sa >= NA) { sa -= NA; pha ^= 1u; }
+            const int step = (b & 1) ? 2 * SETS - 1 : 1;   // to this set's next block
+            if (b & 1) {                                   // and to its next group's ring slot
+                s += SETS;
+                while (s >= NS) { s -= NS; ph ^= 1u; }
+            }
+            sa += step;
+            while (sa >= NA) sa -= NA;
         }
         // ---- epilogue: lane n of this CTA's accumulator holds y[m0 .. m0+256, 128 p + n]
         pdl_wait();
@@ -293,10 +314,10 @@ inline bool umma2_applicable(int M, int N) { return M >= 256 && (N / kPanel) % 2
 inline Umma2Plan plan_umma2(int M, int N, int K)
 {
     Umma2Plan pl{};
-    const int stage = umma_stage_bytes(kUmma2Tok / 2, 1);
+    const int stage = kUmma2StageBytes;
     int stages = (227 * 1024 - 1024 - 2048) / stage;
-    if (stages > 16) stages = 16;
-    if (stages > K / kUmmaBlockK) stages = K / kUmmaBlockK;
+    if (stages > 7) stages = 7;                               // fewer than 16 blocks in the ring (the done barriers)
+    if (stages > K / kGroup) stages = K / kGroup;
     pl.stages = stages;
     pl.ctas = (N / kPanel) * ((M + kUmma2Tok - 1) / kUmma2Tok);
     pl.smem_bytes = 2048 + stages * stage;
@@ -320,12 +341,11 @@ int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const
     args.stages = plan.stages;
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
-    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 64,
+    int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 128,
                                 CU_TENSOR_MAP_SWIZZLE_64B);
     if (st) return st;
-    // x as [M rows, K halves]; a box is 64 k of one CTA's half (128 rows) of the token tile
-    st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
-                            (uint64_t)K * sizeof(__half), 64, kUmma2Tok / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    // x as K / 64 tiles of [M rows, 64 k]; a box is the two tiles of a K group, one CTA's half (128 rows) of the token tile
+    st = make_tensor_map_ktiles(&x_map, x, (uint64_t)K, (uint64_t)M, kUmma2Tok / 2, 2);
     if (st) return st;
     static int configured_smem[64] = {};
     int dev = 0;
