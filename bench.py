@@ -45,8 +45,8 @@ FALLBACK_TFLOPS = 1590.0
 # on (`--print-digest`); `traffic` is that ratio times the timed launches' algorithmic bytes, and
 # null once the sources have changed since the capture.
 NCU_TRAFFIC = {
-    "splitk_kernel<1>": {"digest": "abe6e8a34afd6ef7", "ratio": 1.0005},      # M = 1, the four 7B shapes
-    "umma_kernel<256,4,1,2>": {"digest": "abe6e8a34afd6ef7", "ratio": 0.732},  # qkv, M = 2048, main + tail launch (y partly still in L2)
+    "splitk_kernel<1>": {"digest": "ca9079fd443538ec", "ratio": 1.0005},      # M = 1, the four 7B shapes
+    "umma_kernel<256,4,1,2>": {"digest": "f0d5dd09bf44dc76", "ratio": 0.732},  # qkv, M = 2048, main + tail launch (y partly still in L2)
 }
 
 WORKLOADS = {
@@ -61,10 +61,19 @@ WORKLOADS = {
 }
 
 
-def kernel_source_digest() -> str:
+# the header files each captured kernel is built from (its own file and what that includes)
+KERNEL_SOURCES = {
+    "splitk_kernel<1>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh"),
+    "umma_kernel<256,4,1,2>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh", "gptq_umma.cuh"),
+}
+
+
+def kernel_source_digest(kernel: str | None = None) -> str:
+    """sha256 over the header files a kernel is built from (all kernel headers when the kernel is not listed)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2511_19438_b200", "csrc")
-    for name in sorted(n for n in os.listdir(csrc) if n.endswith(".cuh")):   # the kernels; the .cu holds dispatch only
+    names = KERNEL_SOURCES.get(kernel) or sorted(n for n in os.listdir(csrc) if n.endswith(".cuh"))
+    for name in names:                        # the kernels; the .cu holds dispatch only
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:16]
@@ -337,7 +346,8 @@ def main():
     ap.add_argument("--print-digest", action="store_true", help="print the kernel-source digest and exit")
     args = ap.parse_args()
     if args.print_digest:
-        print(kernel_source_digest())
+        for k in KERNEL_SOURCES:
+            print(k, kernel_source_digest(k))
         return
     spec = dict(WORKLOADS[args.workload])
     if args.ms:
@@ -513,7 +523,7 @@ def main():
         else:
             achieved = sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_s / 1e9
             peak, bound, runit = peaks["hbm_gbs"], "hbm", "GB/s"
-        digest = kernel_source_digest()
+        digest = kernel_source_digest(kname)
         traffic = None
         t = NCU_TRAFFIC.get(kname)
         if t and t.get("digest") == digest:
