@@ -113,7 +113,7 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
     G, panels = K // 128, N // 128
     assert pl.items == G * panels and pl.workspace_bytes == 0
     if pl.kernel == 2:                        # tcgen05 kernel: one launch, 16- to 128-token tiles
-        tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M < 256 else 256
+        tok = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M <= 128 else 256
         assert pl.m_tile == tok and pl.m_chunks == 1
         assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
         tiles = panels * -(-M // tok)
