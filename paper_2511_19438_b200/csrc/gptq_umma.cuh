@@ -519,6 +519,9 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
         for (int S = 1; S <= 8; S *= 2) {
             if (S > G || (pass == 1 && S > 1)) break;          // nothing fits at once: several waves, no split
+            // the exchange of the fp32 partial tiles grows with the tile: with 128 tokens and more an 8-way split measured
+            // slower than a 4-way one (o, M = 128: 16.2 vs 11.5 us; down: 24.5 vs 21.3)
+            if (tok >= 128 && S > 4) break;
             const long long ctas = (long long)tiles * S, ipc = (G + S - 1) / S;
             const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
             if (pass == 0 && on_busiest_sm > cps_max) continue;
@@ -554,7 +557,7 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     if (S == 1 && tiles > slots && tiles % slots != 0) {
         const int r = tiles % slots;
         int ts = 1;
-        while (ts * 2 <= 8 && ts * 2 <= G && r * ts * 2 <= slots) ts *= 2;
+        while (ts * 2 <= (tok >= 128 ? 4 : 8) && ts * 2 <= G && r * ts * 2 <= slots) ts *= 2;
         int tstages = stages;
         const int trefills = 2 * ((G + ts - 1) / ts) / umma_blocks_per_slot(tok);
         if (tstages > trefills) tstages = trefills;
