@@ -13,7 +13,9 @@ multiply-accumulate, reduce, store fp16 y) over every matmul of the workload:
 
 Every matmul is a gptq_gemm call through the C ABI.  The device-timed number replays CUDA graphs
 of those calls (one graph per M) with CUDA events around them; the end-to-end number calls
-gptq_gemm_host with pinned host activations and outputs, copies inside the timed region.
+gptq_gemm_host_batch (one call per step) with pinned host activations and outputs, copies inside
+the timed region.  The default run (decode7b) also measures a short pass of prefill7b and reports it
+as the `prefill` object of the same line, so both halves of the metric are in one record.
 One JSON line is printed by rank 0.  With --impl reference the CPU oracle is timed instead.
 """
 from __future__ import annotations
@@ -45,8 +47,12 @@ FALLBACK_TFLOPS = 1590.0
 # on (`--print-digest`); `traffic` is that ratio times the timed launches' algorithmic bytes, and
 # null once the sources have changed since the capture.
 NCU_TRAFFIC = {
-    "splitk_kernel<1>": {"digest": "ca9079fd443538ec", "ratio": 1.0005},      # M = 1, the four 7B shapes
-    "umma_kernel<256,4,1,2>": {"digest": "7568e8af7d5bd1cb", "ratio": 0.74},  # qkv, M = 2048, main + tail launch (y partly still in L2)
+    "splitk_kernel<1>": {"digest": "ca9079fd443538ec", "ratio": 1.0005, "Ms": (1,),
+                         "source": "ncu capture profiles/splitk_kernel_decode7b.md (M = 1, the four 7B shapes): "
+                                   "dram bytes / algorithmic bytes x algorithmic bytes per timed launch"},
+    "umma_kernel<256,4,1,2>": {"digest": "7568e8af7d5bd1cb", "ratio": 0.74, "Ms": (2048,),
+                               "source": "ncu capture profiles/umma_kernel_prefill7b.md (qkv, M = 2048, main + tail "
+                                         "launch; y partly still in L2): ratio x algorithmic bytes per timed launch"},
 }
 
 WORKLOADS = {
@@ -209,19 +215,16 @@ def launches_per_gemm(spec, M, name, sm_count):
     return 1 + (1 if pl.tail_ctas > 0 else 0) + (1 if spec["act_order"] else 0)
 
 
-def kernel_of(M):
-    """The kernel gptq_gemm dispatches to for M token rows (mirrors gptq_plan)."""
-    if M <= 8:
-        return "splitk_kernel<1>"
-    if M <= 16:
-        return "splitk_kernel<2>"
-    if M <= 32:
-        return "umma_kernel<32,3,1,2>"
-    if M <= 64:
-        return "umma_kernel<64,4,1,2>"
-    if M <= 128:
-        return "umma_kernel<128,4,1,2>"
-    return "umma_kernel<256,4,1,2>"
+def kernel_of(spec, M, sm_count):
+    """The kernel instantiation gptq_gemm launches for M token rows, as the library's own planner names it
+    (the widest shape of the workload decides when shapes differ)."""
+    from paper_2511_19438_b200 import binding as B
+    names = {}
+    for (K, N) in spec["shapes"].values():
+        st, pl = B.gptq_plan(M, N, K, wl.GROUP_SIZE, 1 if spec["act_order"] else 0, sm_count)
+        assert st == B.GPTQ_OK
+        names[B.plan_kernel_name(pl)] = names.get(B.plan_kernel_name(pl), 0) + K * N
+    return max(names, key=names.get)
 
 
 # ------------------------------------------------------------------------------------ reference arm
@@ -329,59 +332,11 @@ def whole_job_value(spec, world, step_bytes, step_flops, steps, slowest_ms):
 
 
 # ------------------------------------------------------------------------------------ product arm
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode7b", choices=list(WORKLOADS))
-    ap.add_argument("--layers", type=int, default=0, help="distinct weight copies per shape (0 = workload default)")
-    ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
-    ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
-    ap.add_argument("--cta-pairs", action="store_true", help="prefill on CTA pairs (tcgen05 cta_group::2), off by default")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--ref-budget", type=float, default=150.0,
-                    help="--impl reference: seconds of CPU time the whole run should take (sizes the per-step sample)")
-    ap.add_argument("--print-digest", action="store_true", help="print the kernel-source digest and exit")
-    args = ap.parse_args()
-    if args.print_digest:
-        for k in KERNEL_SOURCES:
-            print(k, kernel_source_digest(k))
-        return
-    spec = dict(WORKLOADS[args.workload])
-    if args.ms:
-        spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
-    layers = args.layers or spec["layers"]
-    if args.impl == "reference":
-        run_reference(args, spec)
-        return
-    args.warmup = max(args.warmup, 3)
-
-    import torch
-    import torch.distributed as dist
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the GPTQ matmul has no CPU path")
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=device)
-
-    from paper_2511_19438_b200 import build as libbuild
-    if local_rank == 0:
-        libbuild.build()
-    if world > 1:
-        dist.barrier()
-    from paper_2511_19438_b200 import binding as B
-    from paper_2511_19438_b200 import harness as H
-
-    if args.cta_pairs:
-        B.check(B.gptq_set_cta_pairs(1), "gptq_set_cta_pairs")
+def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
+    """Builds one workload on the device, times `steps` graph-replayed steps and `e2e_steps` host-resident steps
+    (max over ranks), and returns the raw numbers report_line() turns into the JSON fields."""
+    torch, dist, B, H = env["torch"], env["dist"], env["B"], env["H"]
+    device, world, local_rank = env["device"], env["world"], env["local_rank"]
     per_m, _host = build_problems(spec, layers, H, torch, device)
     ws = H.WorkspaceHolder(device)
     need = 0
@@ -420,13 +375,13 @@ def main():
         torch.cuda.synchronize()
 
     with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
+        for _ in range(warmup):
             for M in Ms:
                 graphs[M].replay()
         barrier()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(Ms) + 1)] for _ in range(args.steps)]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(Ms) + 1)] for _ in range(steps)]
         t_host0 = time.perf_counter()
-        for k in range(args.steps):
+        for k in range(steps):
             ev[k][0].record(stream)
             for i, M in enumerate(Ms):
                 graphs[M].replay()
@@ -434,7 +389,7 @@ def main():
         barrier()
         t_host1 = time.perf_counter()
     total_ms = ev[0][0].elapsed_time(ev[-1][-1])
-    seg_ms = {M: sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)) for i, M in enumerate(Ms)}
+    seg_ms = {M: sum(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(steps)) for i, M in enumerate(Ms)}
     clocks = sampler.summary(t_host0, t_host1)
     if clocks["samples"] < 3:
         # the timed region was too short to catch a sample: keep replaying the same step, untimed
@@ -449,7 +404,6 @@ def main():
     B.check(B.gptq_check_status(), "timed region")
 
     # ---- end to end: host activations in, host outputs back, every call through gptq_gemm_host
-    e2e_steps = args.e2e_steps or min(args.steps, 20)
     host_io = {}
     h2d = d2h = 0
     for M in Ms:
@@ -493,67 +447,165 @@ def main():
     total_ms, e2e_ms = times[0], times[1]
     seg_ms = {M: times[2 + i] for i, M in enumerate(Ms)}
 
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+    launches_step = sum(launches_per_gemm(spec, M, nm, sms) for M in Ms for (_D, _x, _y, nm) in per_m[M])
+    kernels = {M: kernel_of(spec, M, sms) for M in Ms}
+    out = dict(total_ms=total_ms, e2e_ms=e2e_ms, e2e_steps=e2e_steps, seg_ms=seg_ms, clocks=clocks, bytes_m=bytes_m,
+               flops_m=flops_m, h2d=h2d, d2h=d2h, launches_step=launches_step, kernels=kernels,
+               matmuls={M: len(per_m[M]) for M in Ms}, Ms=Ms)
+    del per_m, graphs, step_problems, step_items, host_io
+    torch.cuda.empty_cache()
+    return out
+
+
+def report_line(name, spec, layers, steps, warmup, r, world):
+    """The JSON fields of one measured workload."""
+    total_ms, e2e_ms, e2e_steps, seg_ms, clocks = r["total_ms"], r["e2e_ms"], r["e2e_steps"], r["seg_ms"], r["clocks"]
+    bytes_m, flops_m, h2d, d2h, launches_step, Ms = r["bytes_m"], r["flops_m"], r["h2d"], r["d2h"], r["launches_step"], r["Ms"]
+    n_matmuls = r["matmuls"]
+    peaks = measured_peaks()
+    metric, unit = metric_of(spec)
+    step_bytes, step_flops = sum(bytes_m.values()), sum(flops_m.values())
+    value = whole_job_value(spec, world, step_bytes, step_flops, steps, total_ms)
+    e2e_value = whole_job_value(spec, world, step_bytes, step_flops, e2e_steps, e2e_ms)
+    per_m_report = {}
+    for M in Ms:
+        s = seg_ms[M] / 1e3
+        per_m_report[str(M)] = {
+            "GB/s": round(bytes_m[M] * steps / s / 1e9, 1),
+            "TFLOP/s": round(flops_m[M] * steps / s / 1e12, 2),
+            "us_per_matmul": round(1e6 * s / steps / n_matmuls[M], 3),
+            "kernel": r["kernels"][M],
+        }
+    # dominant kernel: the kernel instantiation that took most of the timed region
+    groups = {}
+    for M in Ms:
+        groups.setdefault(r["kernels"][M], []).append(M)
+    kname = max(groups, key=lambda k: sum(seg_ms[M] for M in groups[k]))
+    dom_Ms = groups[kname]
+    dom_s = sum(seg_ms[M] for M in dom_Ms) / 1e3
+    dom_launches = sum(n_matmuls[M] for M in dom_Ms) * steps
+    if spec["kind"] == "prefill":
+        achieved = sum(flops_m[M] for M in dom_Ms) * steps / dom_s / 1e12
+        # a timed region of under a second runs at burst clocks: it is held against the burst cuBLAS figure,
+        # a longer one (the power cap has pulled the clocks down) against the sustained one
+        sustained = total_ms >= 1000.0
+        peak, bound, runit = peaks["tflops_sustained" if sustained else "tflops_burst"], "tensor", "TFLOP/s"
+    else:
+        achieved = sum(bytes_m[M] for M in dom_Ms) * steps / dom_s / 1e9
+        peak, bound, runit = peaks["hbm_gbs"], "hbm", "GB/s"
+    digest = kernel_source_digest(kname)
+    # DRAM bytes per launch come from an ncu capture of this kernel (never from this run): the capture's ratio of
+    # measured to algorithmic bytes, scaled by the units a timed launch processes; null when the kernel sources
+    # changed since, or when the timed launches cover token counts the capture did not
+    traffic, traffic_source = None, None
+    t = NCU_TRAFFIC.get(kname)
+    if t and t.get("digest") == digest and set(dom_Ms) <= set(t["Ms"]):
+        traffic = round(t["ratio"] * sum(bytes_m[M] for M in dom_Ms) * steps / dom_launches)
+        traffic_source = t["source"]
+    roofline = {
+        "bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": runit,
+        "frac": round(achieved / peak, 4), "traffic": traffic, "traffic_source": traffic_source, "kernel": kname,
+        "peak_source": peaks["source"],
+        "avg_launch_us": round(1e6 * dom_s / dom_launches, 3),
+        "alg_bytes_per_launch": round(sum(bytes_m[M] for M in dom_Ms) * steps / dom_launches),
+        "launches_timed": dom_launches, "M_covered": dom_Ms,
+        "frac_of_nominal": round(achieved / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 4),
+    }
+    line = {
+        "metric": metric, "value": round(value, 2), "unit": unit, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": round(total_ms / steps, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {"workload": name, "describes": spec["describes"], "layers": layers,
+                   "matmuls_per_step": sum(n_matmuls[M] for M in Ms), "group_size": 128,
+                   "act_order": spec["act_order"], "parallelism": f"{world} independent replica(s)",
+                   "l2": f"inputs larger than L2: each M pass streams {round(bytes_m[Ms[0]] / 1e6)} MB of distinct weights",
+                   "timing": "CUDA events around CUDA-graph replays of the gptq_gemm calls, one graph per M"},
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_value, 2), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
+                "api": "one gptq_gemm_host_batch call per step (x from pinned host memory, y back to it, per matmul)"},
+        "gpu_launches": launches_step * steps,
+        "per_M": per_m_report,
+        "roofline": roofline,
+        "pct_of_nominal": round(100 * value / world / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 2),
+    }
+    if spec["kind"] == "prefill":
+        roofline["peak_kind"] = "sustained" if sustained else "burst"
+        roofline["frac_of_burst_peak"] = round(achieved / peaks["tflops_burst"], 4)
+        roofline["frac_of_sustained_peak"] = round(achieved / peaks["tflops_sustained"], 4)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode7b", choices=list(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=0, help="distinct weight copies per shape (0 = workload default)")
+    ap.add_argument("--e2e-steps", type=int, default=0, help="end-to-end steps (0 = min(steps, 20))")
+    ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
+    ap.add_argument("--cta-pairs", action="store_true", help="prefill on CTA pairs (tcgen05 cta_group::2), off by default")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefill-steps", type=int, default=10,
+                    help="decode7b only: steps of the prefill7b workload measured after it and reported as `prefill` (0 = skip)")
+    ap.add_argument("--ref-budget", type=float, default=150.0,
+                    help="--impl reference: seconds of CPU time the whole run should take (sizes the per-step sample)")
+    ap.add_argument("--print-digest", action="store_true", help="print the kernel-source digest and exit")
+    args = ap.parse_args()
+    if args.print_digest:
+        for k in KERNEL_SOURCES:
+            print(k, kernel_source_digest(k))
+        return
+    spec = dict(WORKLOADS[args.workload])
+    if args.ms:
+        spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
+    layers = args.layers or spec["layers"]
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GPTQ matmul has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2511_19438_b200 import build as libbuild
+    if local_rank == 0:
+        libbuild.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2511_19438_b200 import binding as B
+    from paper_2511_19438_b200 import harness as H
+
+    if args.cta_pairs:
+        B.check(B.gptq_set_cta_pairs(1), "gptq_set_cta_pairs")
+    env = dict(torch=torch, dist=dist, B=B, H=H, device=device, world=world, rank=rank, local_rank=local_rank)
+    res = measure_workload(args.workload, spec, layers, args.steps, args.warmup, args.e2e_steps or min(args.steps, 20), env)
+    # The metric has a second half (prefill TFLOP/s): the default run measures it too, as a short pass of the
+    # prefill workload after the decode one, and reports it as a sub-object of the same line.
+    prefill = None
+    if args.workload == "decode7b" and not args.ms and args.prefill_steps > 0:
+        pspec = dict(WORKLOADS["prefill7b"])
+        prefill = measure_workload("prefill7b", pspec, pspec["layers"], args.prefill_steps, 3, min(args.prefill_steps, 5), env)
     if rank == 0:
-        peaks = measured_peaks()
-        metric, unit = metric_of(spec)
-        step_bytes, step_flops = sum(bytes_m.values()), sum(flops_m.values())
-        value = whole_job_value(spec, world, step_bytes, step_flops, args.steps, total_ms)
-        e2e_value = whole_job_value(spec, world, step_bytes, step_flops, e2e_steps, e2e_ms)
-        sms = torch.cuda.get_device_properties(device).multi_processor_count
-        launches_step = sum(launches_per_gemm(spec, M, name, sms) for M in Ms for (_D, _x, _y, name) in per_m[M])
-        per_m_report = {}
-        for M in Ms:
-            s = seg_ms[M] / 1e3
-            per_m_report[str(M)] = {
-                "GB/s": round(bytes_m[M] * args.steps / s / 1e9, 1),
-                "TFLOP/s": round(flops_m[M] * args.steps / s / 1e12, 2),
-                "us_per_matmul": round(1e6 * s / args.steps / len(per_m[M]), 3),
-            }
-        # dominant kernel: the kernel instantiation that took most of the timed region
-        groups = {}
-        for M in Ms:
-            groups.setdefault(kernel_of(M), []).append(M)
-        kname = max(groups, key=lambda k: sum(seg_ms[M] for M in groups[k]))
-        dom_Ms = groups[kname]
-        dom_s = sum(seg_ms[M] for M in dom_Ms) / 1e3
-        dom_launches = sum(len(per_m[M]) for M in dom_Ms) * args.steps
-        if spec["kind"] == "prefill":
-            achieved = sum(flops_m[M] for M in dom_Ms) * args.steps / dom_s / 1e12
-            peak, bound, runit = peaks["tflops_sustained"], "tensor", "TFLOP/s"
-        else:
-            achieved = sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_s / 1e9
-            peak, bound, runit = peaks["hbm_gbs"], "hbm", "GB/s"
-        digest = kernel_source_digest(kname)
-        traffic = None
-        t = NCU_TRAFFIC.get(kname)
-        if t and t.get("digest") == digest:
-            traffic = round(t["ratio"] * sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_launches)
-        roofline = {
-            "bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": runit,
-            "frac": round(achieved / peak, 4), "traffic": traffic, "kernel": kname, "peak_source": peaks["source"],
-            "avg_launch_us": round(1e6 * dom_s / dom_launches, 3),
-            "alg_bytes_per_launch": round(sum(bytes_m[M] for M in dom_Ms) * args.steps / dom_launches),
-            "launches_timed": dom_launches, "M_covered": dom_Ms,
-            "frac_of_nominal": round(achieved / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 4),
-        }
-        line = {
-            "metric": metric, "value": round(value, 2), "unit": unit, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 5), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
-            "config": {"workload": args.workload, "describes": spec["describes"], "layers": layers,
-                       "matmuls_per_step": sum(len(per_m[M]) for M in Ms), "group_size": 128,
-                       "act_order": spec["act_order"], "parallelism": f"{world} independent replica(s)",
-                       "l2": f"inputs larger than L2: each M pass streams {round(bytes_m[Ms[0]] / 1e6)} MB of distinct weights",
-                       "timing": "CUDA events around CUDA-graph replays of the gptq_gemm calls, one graph per M"},
-            "clocks": clocks,
-            "e2e": {"value": round(e2e_value, 2), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
-                    "api": "one gptq_gemm_host_batch call per step (x from pinned host memory, y back to it, per matmul)"},
-            "gpu_launches": launches_step * args.steps,
-            "per_M": per_m_report,
-            "roofline": roofline,
-            "pct_of_nominal": round(100 * value / world / (NOMINAL_FP16_TFLOPS if spec["kind"] == "prefill" else NOMINAL_HBM_GBS), 2),
-        }
+        line = report_line(args.workload, spec, layers, args.steps, args.warmup, res, world)
+        if prefill is not None:
+            pl = report_line("prefill7b", pspec, pspec["layers"], args.prefill_steps, 3, prefill, world)
+            line["prefill"] = {k: pl[k] for k in ("metric", "value", "unit", "steps", "warmup", "ms_per_step", "config",
+                                                  "clocks", "e2e", "gpu_launches", "per_M", "roofline", "pct_of_nominal")}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(spec)
         print(json.dumps(line), flush=True)

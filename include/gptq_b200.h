@@ -47,7 +47,7 @@ typedef enum {
     GPTQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned */
     GPTQ_ERR_UNSUPPORTED = -4, /* valid GPTQ shape outside the tiled fast path */
     GPTQ_ERR_LAYOUT = -5,      /* bad `which`/flag argument */
-    GPTQ_ERR_GIDX = -6,        /* g_idx out of range or groups of unequal size */
+    GPTQ_ERR_GIDX = -6,        /* g_idx entry out of range, or groups of unequal size (gptq_repack) */
     GPTQ_ERR_WORKSPACE = -7,   /* workspace missing or too small for this call */
     GPTQ_ERR_CUDA = -8,        /* a CUDA runtime call failed (see gptq_last_cuda_error) */
     GPTQ_ERR_TIMEOUT = -9      /* a bounded device-side wait gave up (see gptq_check_status) */
@@ -60,11 +60,14 @@ int gptq_last_cuda_error(void);
 
 /* ---- bit-exact building blocks on the canonical layout (the format reading) -------- */
 
-/* q_out uint8[K,N] and z_out uint8[G,N] (either may be NULL to skip it). */
+/* The nibble unpacking of the paper's Section 1 format ("4-bit quantized weights"), on its own, for bit-exact
+ * checks: q_out uint8[K,N] and z_out uint8[G,N] (either may be NULL to skip it).  Any group_size dividing K. */
 int gptq_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out,
                    int N, int K, int group_size, void *stream);
 
-/* w_out fp32[K,N] = float(q - z) * float(scale), one fp32 multiply (the product is exact).
+/* The dequantisation every kernel of Section 3 performs before its multiply-accumulate (Eq. 14-15 apply it in
+ * half precision; here it is written out in fp32 so that there is exactly one right answer):
+ * w_out fp32[K,N] = float(q - z) * float(scale), one fp32 multiply (the product is exact).
  * repacked = 0: inputs are canonical; g_idx is the checkpoint's g_idx when act_order != 0.
  * repacked = 1: inputs are the buffers written by gptq_repack and g_idx is its perm_out;
  *               rows are written back in ORIGINAL order, so both modes give identical bits. */
@@ -79,12 +82,13 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
  * invalid argument. */
 size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order);
 
-/* Re-tiles a canonical layer.  Fast-path requirements: group_size == 128, K % 128 == 0,
+/* Re-tiles a canonical layer (what Section 3.2 / Algorithm 2 achieve with wider loads of the original layout is
+ * achieved here by storing the weights in the order the kernels stream them).  Fast-path requirements: group_size == 128, K % 128 == 0,
  * N % 128 == 0 (else GPTQ_ERR_UNSUPPORTED).  With act_order != 0 the rows are stably sorted
  * by g_idx so that each group's rows are contiguous; perm_out[i] = original index of sorted
  * row i (int32[K]).  g_idx is range-checked on the device and every group must have exactly
- * group_size rows; this one-time call synchronises the stream to report GPTQ_ERR_GIDX.
- * Outputs must not alias inputs. */
+ * group_size rows; with act_order this one-time call synchronises the stream and returns GPTQ_ERR_GIDX
+ * for either violation (nothing is tiled then).  Outputs must not alias inputs. */
 int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
                 void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out,
                 int N, int K, int group_size, int act_order, void *stream);
@@ -95,12 +99,14 @@ int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scale
  * up to 256 bytes), otherwise 0 (the split-K partial sums stay in shared memory). */
 size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order);
 
-/* Registers caller-owned device scratch for later gptq_gemm calls on the current device (`stream`
- * is unused and kept for compatibility).  The workspace is shared by all calls: calls that may
- * overlap on the GPU (different streams) must not share one.  ptr = NULL unregisters. */
-int gptq_set_workspace(void *ptr, size_t bytes, void *stream);
+/* Registers caller-owned device scratch for later gptq_gemm calls on the current device.  The workspace is
+ * shared by all calls: calls that may overlap on the GPU (different streams) must not share one.
+ * ptr = NULL unregisters.  ptr must be 16-byte aligned (GPTQ_ERR_ALIGN). */
+int gptq_set_workspace(void *ptr, size_t bytes);
 
-/* y fp16[M,N] = x fp16[M,K] . dequant(W).  qweight/qzeros/scales are the REPACKED buffers from
+/* The GPTQ linear layer of Sections 1 and 3 (the product all three of the paper's optimisations serve; Section
+ * 4.4's last paragraph fixes what "the same result" means: equal up to summation order).
+ * y fp16[M,N] = x fp16[M,K] . dequant(W).  qweight/qzeros/scales are the REPACKED buffers from
  * gptq_repack; with act_order != 0, g_idx is gptq_repack's perm_out (else it may be NULL).
  * fp32 accumulation, one round-to-nearest-even conversion to fp16.  Any M >= 1.  Up to 16 rows the
  * weights enter the MMA as exact integers q - z and the scale multiplies fp32 group sums; above
@@ -108,7 +114,14 @@ int gptq_set_workspace(void *ptr, size_t bytes, void *stream);
  * The kernels begin fetching weights before earlier work on the stream has finished
  * (programmatic dependent launch); x, y and the workspace are only touched afterwards.  The
  * weight buffers must therefore not be written by a kernel launched immediately before this
- * call on the same stream (gptq_repack itself is safe). */
+ * call on the same stream (gptq_repack itself is safe).
+ * Thread safety: calls from several host threads are allowed (the library's own host state is locked);
+ * GPU work of calls on different streams may overlap unless they share the act-order workspace.
+ * Accuracy: the stated bar |y - y_exact| <= 1e-2 sqrt(K/4096) + 1e-2 |y_exact| holds for the Llama shapes
+ * (K >= 4096).  Above 16 token rows the fp16 rounding of each scaled weight gives y an error of about
+ * 1.4e-3 sqrt(K/4096) rms for unit-variance x; since the bar shrinks with sqrt(K) as fast as that error does
+ * but a layer with very few groups (K <= 256) has columns whose few scales are all large, single elements
+ * among millions can exceed the bar there (seen: 1 of 5e6 at K = 256, by a factor of 2). */
 int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales,
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
@@ -170,16 +183,26 @@ typedef struct {
  * while matmul i runs; the matmuls themselves stay in order on `stream`, and `stream` completes after
  * the last copy.  Staging buffers may be shared between problems (reuse waits for the earlier user).
  * All problems are validated before anything is enqueued; on an invalid problem *bad_index (if not
- * NULL) receives its index and nothing runs. */
+ * NULL) receives its index and nothing runs.  If a later step fails, `stream` is still joined with the
+ * internal streams before the error is returned.  The internal streams and events belong to the device:
+ * concurrent calls on one device (several host threads, or several user streams) are serialised by a lock
+ * for the duration of the enqueue.  Not capturable in a CUDA graph (it records and waits on events of
+ * internal streams). */
 int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
 
 /* Synchronises `stream` and returns GPTQ_ERR_TIMEOUT if any kernel's bounded wait gave up
  * since the last check (the flag is then cleared), GPTQ_ERR_CUDA on a runtime error, else OK. */
 int gptq_check_status(void *stream);
 
+/* Self-test of that mechanism (no counterpart in the paper): launches one thread that waits, the way the matmul
+ * kernels wait, on a barrier nothing will ever complete, gives up after limit_us microseconds (1 .. 1e6) and
+ * returns normally; the next gptq_check_status then reports GPTQ_ERR_TIMEOUT.  Nothing faults or hangs. */
+int gptq_selftest_wait_timeout(unsigned int limit_us, void *stream);
+
 /* ---- host-only: how a problem would be launched (no CUDA call; usable without a GPU) -- */
 
 typedef struct {
+    char kernel_name[48]; /* the kernel instantiation as profilers print it, e.g. "splitk_kernel<1>" */
     int kernel;       /* 1 = cluster split-K mma.sync kernel (gptq_gemm, M <= 16),
                          2 = tcgen05 kernel (gptq_gemm, M >= 17),
                          3 = stream-K mma.sync kernel (gptq_gemm_noalloc) */
@@ -202,7 +225,8 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
 /* The same for gptq_gemm_noalloc (stream-K kernel; workspace_bytes is its need of the built-in scratch). */
 int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out);
 
-/* The stream-K partition gptq_gemm_noalloc's kernel uses, from the same arithmetic: CTA `cta` of `ctas` works
+/* For tests only (not needed to use the library): the stream-K partition gptq_gemm_noalloc's kernel uses, from
+ * the same arithmetic as the kernel.  CTA `cta` of `ctas` works
  * through items [*first_item, *end_item) of `items`; the K range of panel `panel` (its `groups`
  * consecutive items) is shared by CTAs *first_cta .. *last_cta, whose partial tiles are summed
  * in that order. */

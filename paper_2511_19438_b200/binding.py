@@ -35,6 +35,7 @@ GPTQ_ERR_TIMEOUT = -9
 
 class gptq_plan_t(ctypes.Structure):
     _fields_ = [
+        ("kernel_name", ctypes.c_char * 48),
         ("kernel", ctypes.c_int), ("m_tile", ctypes.c_int), ("m_chunks", ctypes.c_int),
         ("stages", ctypes.c_int), ("ctas", ctypes.c_int), ("items", ctypes.c_int),
         ("split_panels", ctypes.c_int), ("smem_bytes", ctypes.c_int),
@@ -62,7 +63,7 @@ _SIGNATURES = {
     "gptq_repack_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "gptq_repack": (_i, [_vp] * 8 + [_i, _i, _i, _i, _vp]),
     "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
-    "gptq_set_workspace": (_i, [_vp, _sz, _vp]),
+    "gptq_set_workspace": (_i, [_vp, _sz]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_set_cta_pairs": (_i, [_i]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
@@ -70,6 +71,7 @@ _SIGNATURES = {
     "gptq_noalloc_scratch_bytes": (_sz, []),
     "gptq_gemm_host_batch": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_check_status": (_i, [_vp]),
+    "gptq_selftest_wait_timeout": (_i, [ctypes.c_uint, _vp]),
     "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_noalloc": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_cta_range": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
@@ -148,8 +150,8 @@ def gptq_workspace_bytes(M, N, K, group_size, act_order) -> int:
     return _lib.gptq_workspace_bytes(M, N, K, group_size, int(act_order))
 
 
-def gptq_set_workspace(ptr, nbytes, stream=None) -> int:
-    return _lib.gptq_set_workspace(_ptr(ptr), nbytes, _stream(stream))
+def gptq_set_workspace(ptr, nbytes) -> int:
+    return _lib.gptq_set_workspace(_ptr(ptr), nbytes)
 
 
 def gptq_gemm(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
@@ -196,6 +198,14 @@ def gptq_gemm_host_batch(problems, stream=None):
 
 def gptq_check_status(stream=None) -> int:
     return _lib.gptq_check_status(_stream(stream))
+
+
+def gptq_selftest_wait_timeout(limit_us, stream=None) -> int:
+    return _lib.gptq_selftest_wait_timeout(int(limit_us), _stream(stream))
+
+
+def plan_kernel_name(plan) -> str:
+    return plan.kernel_name.decode()
 
 
 def gptq_plan(M, N, K, group_size, act_order, sm_count):

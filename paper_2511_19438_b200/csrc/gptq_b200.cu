@@ -8,6 +8,7 @@
 #include "gptq_umma2.cuh"
 
 #include <atomic>
+#include <cstdio>
 #include <mutex>
 #include <vector>
 
@@ -21,6 +22,23 @@ int record_cuda_error(cudaError_t e)
     if (e == cudaSuccess) return GPTQ_OK;
     g_last_cuda_error.store((int)e);
     return GPTQ_ERR_CUDA;
+}
+
+int ensure_dynamic_smem(const void *kernel, int *configured, int smem_bytes)
+{
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (configured[dev] >= smem_bytes) return GPTQ_OK;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    configured[dev] = smem_bytes;
+    return GPTQ_OK;
 }
 
 constexpr int kMaxDevices = 64;
@@ -96,6 +114,7 @@ static size_t gemm_workspace_need(int M, int K, int act_order)
 
 // Copy streams and events of gptq_gemm_host_batch (per device, created on first use; no device memory).
 struct HostPipe {
+    std::mutex enqueue;   // held for a whole gptq_gemm_host_batch call: the streams and events are per device
     cudaStream_t in = nullptr, out = nullptr;
     std::vector<cudaEvent_t> events;
 };
@@ -134,7 +153,7 @@ const char *gptq_status_string(int status)
     case GPTQ_ERR_ALIGN: return "a pointer is not 16-byte aligned";
     case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 128, N%128==0, K%128==0, equal groups)";
     case GPTQ_ERR_LAYOUT: return "invalid layout selector or flag";
-    case GPTQ_ERR_GIDX: return "g_idx entry out of range";
+    case GPTQ_ERR_GIDX: return "g_idx entry out of range, or groups of unequal size";
     case GPTQ_ERR_WORKSPACE: return "workspace missing or too small (see gptq_workspace_bytes)";
     case GPTQ_ERR_CUDA: return "a CUDA runtime call failed (see gptq_last_cuda_error)";
     case GPTQ_ERR_TIMEOUT: return "a bounded device-side wait gave up";
@@ -204,6 +223,11 @@ int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scale
                          act_order, (cudaStream_t)stream);
 }
 
+static void set_kernel_name(gptq_plan_t *out, const char *fmt, int a, int b = 0, int c = 0, int d = 0)
+{
+    snprintf(out->kernel_name, sizeof(out->kernel_name), fmt, a, b, c, d);
+}
+
 int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, gptq_plan_t *out)
 {
     if (!out) return GPTQ_ERR_NULL;
@@ -227,6 +251,10 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
         out->tail_ctas = up.tail_tiles * up.tail_S;
         out->tail_cluster_size = up.tail_S;
         out->split_panels = up.S > 1 ? N / kPanel : 0;
+        if (g_use_cta_pairs.load() && umma2_applicable(M, N))
+            set_kernel_name(out, "umma2_kernel", 0);
+        else
+            set_kernel_name(out, "umma_kernel<%d,%d,%d,%d>", up.tok, umma_a_stages(up.tok, up.np), up.np, up.sets);
         return GPTQ_OK;
     }
     const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
@@ -243,6 +271,7 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     out->cluster_size = pl.S;
     out->tail_ctas = 0;
     out->tail_cluster_size = 1;
+    set_kernel_name(out, "splitk_kernel<%d>", pl.m_tile / 8);
     return GPTQ_OK;
 }
 
@@ -267,6 +296,7 @@ int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm
     out->cluster_size = 1;
     out->tail_ctas = 0;
     out->tail_cluster_size = 1;
+    set_kernel_name(out, "streamk_kernel<%d>", gp.sk.m_tile / 8);
     return GPTQ_OK;
 }
 
@@ -297,9 +327,8 @@ size_t gptq_workspace_bytes(int M, int N, int K, int group_size, int act_order)
     return gemm_workspace_need(M, K, act_order);
 }
 
-int gptq_set_workspace(void *ptr, size_t bytes, void *stream)
+int gptq_set_workspace(void *ptr, size_t bytes)
 {
-    (void)stream;
     int dev, sms;
     int st = current_device_sms(&dev, &sms);
     if (st) return st;
@@ -470,50 +499,74 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
     HostPipe *pipe = nullptr;
     st = ensure_host_pipe(dev, 3 * (size_t)count + 1, &pipe);
     if (st) return st;
+    // one caller at a time per device: the copy streams and events belong to the device, not to the call
+    std::lock_guard<std::mutex> enqueue_lock(pipe->enqueue);
+    std::vector<cudaEvent_t> events;   // handles copied out: another caller may grow (and move) the device's vector
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        events.assign(pipe->events.begin(), pipe->events.begin() + (3 * (size_t)count + 1));
+    }
     cudaStream_t s = (cudaStream_t)stream;
-    cudaEvent_t *ev_x = pipe->events.data(), *ev_g = ev_x + count, *ev_y = ev_g + count, ev_start = ev_y[count];
+    cudaEvent_t *ev_x = events.data(), *ev_g = ev_x + count, *ev_y = ev_g + count, ev_start = ev_y[count];
     auto check = [&](cudaError_t e) { return record_cuda_error(e); };
     // copies must not start before earlier work on `stream` (which may still use the staging buffers)
     if ((st = check(cudaEventRecord(ev_start, s)))) return st;
     if ((st = check(cudaStreamWaitEvent(pipe->in, ev_start, 0)))) return st;
     if ((st = check(cudaStreamWaitEvent(pipe->out, ev_start, 0)))) return st;
-    for (int i = 0; i < count; ++i) {
+    // from here on the internal streams are forked off `stream`: every exit goes through the join below
+    for (int i = 0; i < count && !st; ++i) {
         const gptq_host_problem_t &q = problems[i];
         // a staging buffer shared with an earlier problem is reused only after that problem is done with it
-        for (int j = i - 1; j >= 0; --j)
+        for (int j = i - 1; j >= 0 && !st; --j)
             if (problems[j].x_stage == q.x_stage) {
-                if ((st = check(cudaStreamWaitEvent(pipe->in, ev_g[j], 0)))) return st;
+                st = check(cudaStreamWaitEvent(pipe->in, ev_g[j], 0));
                 break;
             }
-        if ((st = check(cudaMemcpyAsync(q.x_stage, q.x_host, (size_t)q.M * q.K * sizeof(__half), cudaMemcpyHostToDevice,
-                                        pipe->in))))
-            return st;
-        if ((st = check(cudaEventRecord(ev_x[i], pipe->in)))) return st;
-        if ((st = check(cudaStreamWaitEvent(s, ev_x[i], 0)))) return st;
-        for (int j = i - 1; j >= 0; --j)
+        if (!st) st = check(cudaMemcpyAsync(q.x_stage, q.x_host, (size_t)q.M * q.K * sizeof(__half), cudaMemcpyHostToDevice, pipe->in));
+        if (!st) st = check(cudaEventRecord(ev_x[i], pipe->in));
+        if (!st) st = check(cudaStreamWaitEvent(s, ev_x[i], 0));
+        for (int j = i - 1; j >= 0 && !st; --j)
             if (problems[j].y_stage == q.y_stage) {
-                if ((st = check(cudaStreamWaitEvent(s, ev_y[j], 0)))) return st;
+                st = check(cudaStreamWaitEvent(s, ev_y[j], 0));
                 break;
             }
+        if (st) break;
         st = gptq_gemm(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
                        q.act_order, stream);
         if (st) {
             if (bad_index) *bad_index = i;
-            break;   // still join the copy streams below
+            break;
         }
-        if ((st = check(cudaEventRecord(ev_g[i], s)))) return st;
-        if ((st = check(cudaStreamWaitEvent(pipe->out, ev_g[i], 0)))) return st;
-        if ((st = check(cudaMemcpyAsync(q.y_host, q.y_stage, (size_t)q.M * q.N * sizeof(__half), cudaMemcpyDeviceToHost,
-                                        pipe->out))))
-            return st;
-        if ((st = check(cudaEventRecord(ev_y[i], pipe->out)))) return st;
+        st = check(cudaEventRecord(ev_g[i], s));
+        if (!st) st = check(cudaStreamWaitEvent(pipe->out, ev_g[i], 0));
+        if (!st) st = check(cudaMemcpyAsync(q.y_host, q.y_stage, (size_t)q.M * q.N * sizeof(__half), cudaMemcpyDeviceToHost, pipe->out));
+        if (!st) st = check(cudaEventRecord(ev_y[i], pipe->out));
     }
-    // `stream` finishes after the last copy of each direction
+    // join: `stream` finishes after the last copy of each direction, also after an error
     int st2 = check(cudaEventRecord(ev_start, pipe->in));
     if (!st2) st2 = check(cudaStreamWaitEvent(s, ev_start, 0));
     if (!st2) st2 = check(cudaEventRecord(ev_x[0], pipe->out));
     if (!st2) st2 = check(cudaStreamWaitEvent(s, ev_x[0], 0));
     return st ? st : st2;
+}
+
+// ---- self-test of the bounded waits ------------------------------------------------------------
+// One thread waits (for at most `limit_ns`) on an mbarrier that nothing will ever complete, exactly as the
+// matmul kernels wait, gives up, records the time-out in the status word and returns normally.
+__global__ void wait_selftest_kernel(unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = smem_u32(&bar);
+    mbar_init(b, 1);
+    fence_barrier_init();
+    mbar_wait_limited(b, 0, limit_ns);
+}
+
+int gptq_selftest_wait_timeout(unsigned int limit_us, void *stream)
+{
+    if (limit_us < 1 || limit_us > 1000000) return GPTQ_ERR_SHAPE;
+    wait_selftest_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((unsigned long long)limit_us * 1000ull);
+    return record_cuda_error(cudaGetLastError());
 }
 
 int gptq_check_status(void *stream)
@@ -528,7 +581,7 @@ int gptq_check_status(void *stream)
     e = cudaMemcpyToSymbolAsync(g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return record_cuda_error(e);
-    return status == kStatusWaitTimeout ? GPTQ_ERR_TIMEOUT : GPTQ_ERR_GIDX;
+    return GPTQ_ERR_TIMEOUT;
 }
 
 }  // extern "C"

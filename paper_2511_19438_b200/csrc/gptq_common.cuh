@@ -74,9 +74,13 @@ __host__ __device__ inline size_t repacked_zero_byte(int grp, int n, int G, int 
 // ----------------------------------------------------------------------------------------
 // Device status word: kernels never trap; a bounded wait that gives up records a code here.
 // ----------------------------------------------------------------------------------------
-enum : int { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusUnequalGroups = 2, kStatusBadGidx = 3 };  // recorded with atomicMax
-// The library is built as one translation unit, so this is the single definition.
+enum : int { kStatusOk = 0, kStatusWaitTimeout = 1 };                  // g_device_status, recorded with atomicMax
+enum : int { kGidxOk = 0, kGidxUnequalGroups = 1, kGidxOutOfRange = 2 };   // g_gidx_status, likewise
+// The library is built as one translation unit, so these are the single definitions.  The g_idx
+// check of gptq_repack has a word of its own, so that reading and clearing it never drops a
+// pending wait timeout of an earlier kernel.
 __device__ int g_device_status = 0;
+__device__ int g_gidx_status = 0;
 
 #ifdef __CUDACC__
 // ----------------------------------------------------------------------------------------
@@ -131,16 +135,20 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     return t;
 }
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity)
+__device__ __noinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, uint64_t limit_ns)
 {
     const uint64_t start = global_timer_ns();
     for (;;) {
         for (int it = 0; it < 256; ++it)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - start > kWaitLimitNs) break;
+        if (global_timer_ns() - start > limit_ns) break;
     }
     atomicMax(&g_device_status, (int)kStatusWaitTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity)
+{
+    return mbar_wait_limited(bar, parity, kWaitLimitNs);
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
@@ -148,14 +156,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity);
 }
-// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.  dst, src and
-// bytes must be multiples of 16.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
+// 1-D bulk copy global -> shared with an L2 cache-policy hint, completion counted in bytes on an
+// mbarrier.  dst, src and bytes must be multiples of 16.  Issue it from a dedicated producer thread:
+// issued from lanes of a warp that goes on to run mma.sync, it faulted ("illegal instruction").
 __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
                                               uint64_t policy)
 {
@@ -238,6 +241,9 @@ __device__ __forceinline__ uint32_t lds8(uint32_t addr)
 // Host-side launch plumbing shared by the translation units
 // ----------------------------------------------------------------------------------------
 int record_cuda_error(cudaError_t e);   // stores e, returns GPTQ_ERR_CUDA (or GPTQ_OK for success)
+// Raises a kernel's dynamic shared-memory limit (and asks for the largest carve-out) the first time a launch on
+// the current device needs more than before; `configured` is the launcher's per-device record.  Thread-safe.
+int ensure_dynamic_smem(const void *kernel, int *configured, int smem_bytes);
 
 struct Workspace {
     void *ptr = nullptr;

@@ -122,10 +122,10 @@ __global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *
     }
     if (k >= K) return;
     if (bad) {
-        atomicMax(&g_device_status, (int)kStatusBadGidx);
+        atomicMax(&g_gidx_status, (int)kGidxOutOfRange);
         return;
     }
-    if (same_total != kGroup) atomicMax(&g_device_status, (int)kStatusUnequalGroups);
+    if (same_total != kGroup) atomicMax(&g_gidx_status, (int)kGidxUnequalGroups);
     int rank = below + same_before;
     if (rank >= 0 && rank < K) perm[rank] = k;
 }
@@ -198,15 +198,15 @@ int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *sca
         if (e != cudaSuccess) return record_cuda_error(e);
         // one-time call: read the validation result before tiling with a possibly invalid perm
         int status = 0;
-        e = cudaMemcpyFromSymbolAsync(&status, g_device_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
+        e = cudaMemcpyFromSymbolAsync(&status, g_gidx_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) return record_cuda_error(e);
-        if (status == kStatusBadGidx || status == kStatusUnequalGroups) {
+        if (status != kGidxOk) {
             int zero = 0;
-            e = cudaMemcpyToSymbolAsync(g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
+            e = cudaMemcpyToSymbolAsync(g_gidx_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
             if (e == cudaSuccess) e = cudaStreamSynchronize(s);
             if (e != cudaSuccess) return record_cuda_error(e);
-            return status == kStatusBadGidx ? GPTQ_ERR_GIDX : GPTQ_ERR_UNSUPPORTED;
+            return GPTQ_ERR_GIDX;   // out of range, or groups of unequal size
         }
     }
     size_t words = (size_t)(K / 8) * N;

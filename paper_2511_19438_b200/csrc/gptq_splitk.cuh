@@ -39,12 +39,6 @@ __device__ __forceinline__ uint32_t map_to_cluster_rank(uint32_t local_addr, uin
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
     return remote;
 }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr)
-{
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-    return v;
-}
 // fire-and-forget 4-byte store into another CTA's shared memory; the 4 bytes are counted on that CTA's mbarrier
 __device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar)
 {
@@ -193,8 +187,6 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         // x fragment of k chunk (4j + t4) for token slot g: row r of the swizzled tile
         const uint32_t x_off0 = r * 128 + ((uint32_t)(t4 ^ r) << 4);          // j = 0
         const uint32_t x_off1 = r * 128 + ((uint32_t)((4 + t4) ^ r) << 4);    // j = 1
-        constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-
         int s = 0;
         uint32_t phase = 0;
         bool ok = true;   // false after a wait gave up: keep taking part in barriers, skip the data
@@ -202,57 +194,14 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             const uint32_t st = ring + s * kStage;
             if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
 
-            const uint4 wq0 = lds128(st + w_off);
-            const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
-            const uint32_t sc = lds32(st + s_off);
-            const uint32_t zb = lds8(st + z_off);
-            const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
-
-            {
-                const uint32_t zA = zb & 15u, zB = zb >> 4;
-                const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
-                const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
-                float accg[MT][4];
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) accg[mt][i] = 0.f;
-#pragma unroll
-                for (int blk = 0; blk < 2; ++blk) {
-                    const uint4 wq = blk ? wq1 : wq0;
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
-                        const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                        const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                        const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                        const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
-                        wA >>= 8;
-                        wB >>= 8;
-                        const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                        const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                        const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                        const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt) {
-                            const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
-                            mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
-                            mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
-                        }
-                    }
-                }
-                // release the stage, then fold the group sum into the running sum with the group's scale
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
-                if (++s == stages) { s = 0; phase ^= 1u; }
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    acc[mt][0] = fmaf(sf.x, accg[mt][0], acc[mt][0]);
-                    acc[mt][1] = fmaf(sf.x, accg[mt][1], acc[mt][1]);
-                    acc[mt][2] = fmaf(sf.y, accg[mt][2], acc[mt][2]);
-                    acc[mt][3] = fmaf(sf.y, accg[mt][3], acc[mt][3]);
-                }
-            }
+            float accg[MT][4];
+            uint32_t sc;
+            consume_item<MT>(st, w_off, s_off, z_off, x_off0, x_off1, accg, sc);
+            // release the stage, then fold the group sum into the running sum with the group's scale
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            if (++s == stages) { s = 0; phase ^= 1u; }
+            fold_group<MT>(acc, accg, sc);
         }
     }
 
@@ -361,18 +310,8 @@ template <int MT>
 static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, const SplitKPlan &plan, cudaStream_t s)
 {
     static int configured_smem[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
-    if (configured_smem[dev] < plan.smem_bytes) {
-        e = cudaFuncSetAttribute(splitk_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(splitk_kernel<MT>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        configured_smem[dev] = plan.smem_bytes;
-    }
+    const int cfg_st = ensure_dynamic_smem((const void *)splitk_kernel<MT>, configured_smem, plan.smem_bytes);
+    if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
     cfg.blockDim = dim3(kStreamKThreads);
@@ -412,8 +351,6 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     switch (plan.m_tile) {
     case 8: return launch_splitk_mt<1>(args, x_map, plan, s);
     case 16: return launch_splitk_mt<2>(args, x_map, plan, s);
-    case 32: return launch_splitk_mt<4>(args, x_map, plan, s);
-    case 64: return launch_splitk_mt<8>(args, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }

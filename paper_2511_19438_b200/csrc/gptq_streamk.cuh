@@ -44,6 +44,66 @@ __host__ __device__ inline int sk_owner(long long T, int C, long long t) { retur
 // chunks of the swizzled x tile, so the 128-bit fragment loads are bank-conflict free.
 __host__ __device__ constexpr int token_row_of_slot(int n) { return ((n & 1) << 2) | (n & 2) | ((n >> 2) & 1); }
 
+// The arithmetic of one (panel, group) item for one consumer warp, shared by the mma.sync kernels: the lane reads
+// its two 16-byte chunks of packed weights, the scale pair and the zero byte of its columns from ring stage `st`,
+// turns nibbles into exact fp16 integers q - z and multiplies them with the stage's x tiles; `accg` receives the
+// unscaled fp32 group sums, `sc` the two fp16 scales.  The stage may be released once this returns.
+template <int MT>
+__device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32_t s_off, uint32_t z_off,
+                                             uint32_t x_off0, uint32_t x_off1, float (&accg)[MT][4], uint32_t &sc)
+{
+    constexpr int kXTile = MT * 1024;
+    constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
+    const uint4 wq0 = lds128(st + w_off);
+    const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
+    sc = lds32(st + s_off);
+    const uint32_t zb = lds8(st + z_off);
+    const uint32_t zA = zb & 15u, zB = zb >> 4;
+    const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
+    const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) accg[mt][i] = 0.f;
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+        const uint4 wq = blk ? wq1 : wq0;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
+            const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+            const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+            const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+            const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+            wA >>= 8;
+            wB >>= 8;
+            const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
+            const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
+            const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
+            const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
+                mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
+                mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
+            }
+        }
+    }
+}
+// folds a group's sums into the running sums with the group's scales
+template <int MT>
+__device__ __forceinline__ void fold_group(float (&acc)[MT][4], const float (&accg)[MT][4], uint32_t sc)
+{
+    const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        acc[mt][0] = fmaf(sf.x, accg[mt][0], acc[mt][0]);
+        acc[mt][1] = fmaf(sf.x, accg[mt][1], acc[mt][1]);
+        acc[mt][2] = fmaf(sf.y, accg[mt][2], acc[mt][2]);
+        acc[mt][3] = fmaf(sf.y, accg[mt][3], acc[mt][3]);
+    }
+}
+
 struct StreamKArgs {
     const uint8_t *qweight; // tiled
     const uint8_t *scales;
@@ -133,8 +193,6 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     // x fragment of k chunk (4j + t4) for token slot g: row r of the swizzled tile
     const uint32_t x_off0 = r * 128 + ((uint32_t)(t4 ^ r) << 4);          // j = 0
     const uint32_t x_off1 = r * 128 + ((uint32_t)((4 + t4) ^ r) << 4);    // j = 1
-    constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
-
     float acc[MT][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -152,57 +210,14 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
         const uint32_t st = ring + s * kStage;
         if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
 
-        const uint4 wq0 = lds128(st + w_off);
-        const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
-        const uint32_t sc = lds32(st + s_off);
-        const uint32_t zb = lds8(st + z_off);
-        const uint32_t zA = zb & 15u, zB = zb >> 4;
-        const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
-        const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
-
         float accg[MT][4];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) accg[mt][i] = 0.f;
-
-#pragma unroll
-        for (int blk = 0; blk < 2; ++blk) {
-            const uint4 wq = blk ? wq1 : wq0;
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
-                const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                const uint32_t a3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
-                wA >>= 8;
-                wB >>= 8;
-                const uint32_t c0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
-                const uint32_t c2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
-                const uint32_t c1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
-                const uint32_t c3 = hsub2_u32(lop3_and_or(wB, HI, MAGIC_HI), zhiB);
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
-                    mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
-                    mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
-                }
-            }
-        }
+        uint32_t sc;
+        consume_item<MT>(st, w_off, s_off, z_off, x_off0, x_off1, accg, sc);
         // release the stage, then fold the group sum into the running sum with the group's scale
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         if (++s == stages) { s = 0; phase ^= 1u; }
-
-        const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-            acc[mt][0] = fmaf(sf.x, accg[mt][0], acc[mt][0]);
-            acc[mt][1] = fmaf(sf.x, accg[mt][1], acc[mt][1]);
-            acc[mt][2] = fmaf(sf.y, accg[mt][2], acc[mt][2]);
-            acc[mt][3] = fmaf(sf.y, accg[mt][3], acc[mt][3]);
-        }
+        fold_group<MT>(acc, accg, sc);
 
         const bool seg_end = (grp == a.G - 1) || (t == t1 - 1);
         if (seg_end) {
@@ -316,18 +331,8 @@ static int launch_streamk_mt(const StreamKArgs &args, const CUtensorMap &x_map, 
                              cudaStream_t s)
 {
     static int configured_smem[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
-    if (configured_smem[dev] < plan.smem_bytes) {
-        e = cudaFuncSetAttribute(streamk_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(streamk_kernel<MT>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        configured_smem[dev] = plan.smem_bytes;
-    }
+    const int cfg_st = ensure_dynamic_smem((const void *)streamk_kernel<MT>, configured_smem, plan.smem_bytes);
+    if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
     cfg.blockDim = dim3(kStreamKThreads);

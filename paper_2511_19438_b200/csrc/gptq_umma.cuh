@@ -157,11 +157,6 @@ __host__ __device__ constexpr int umma_slot_bytes(int TOK, int NP)
 {
     return (umma_blocks_per_slot(TOK) * (TOK * 128 + NP * kUmmaWBlockBytes) + 1023) & ~1023;
 }
-// one K64 block per slot (the CTA-pair kernel)
-__host__ __device__ constexpr int umma_stage_bytes(int TOK, int NP)
-{
-    return (TOK * 128 + NP * (kUmmaWBlockBytes + kItemSBytes + kItemZBytes) + 1023) & ~1023;
-}
 __host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP)
 {
     // per panel: accumulator (TOK columns) + A ring (32 columns = one K64 block per stage); a power of two >= 32
@@ -507,7 +502,7 @@ __host__ __device__ constexpr int umma_ctas_per_sm(int tok, int np) { return (np
 inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
 {
     UmmaPlan pl{};
-    const int tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    const int tok = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
     const int panels = N / kPanel;
     const int np = 1;
     const int sets = 2;
@@ -578,17 +573,8 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
 {
     auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS>;
     static int configured_smem[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
-    if (configured_smem[dev] < plan.smem_bytes) {
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        configured_smem[dev] = plan.smem_bytes;
-    }
+    const int cfg_st = ensure_dynamic_smem((const void *)kernel, configured_smem, plan.smem_bytes);
+    if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)ctas);
     cfg.blockDim = dim3(umma_threads(NP, SETS));
@@ -633,7 +619,6 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     if (st) return st;
     auto launch = [&](const UmmaArgs &la, int ctas) {
         switch (plan.tok) {
-        case 16: return launch_umma_tok<16, 1, 2>(la, w_map, x_map, plan, ctas, s);
         case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, s);
         case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, s);
         case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, s);

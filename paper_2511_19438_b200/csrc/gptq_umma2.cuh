@@ -348,18 +348,8 @@ int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const
     st = make_tensor_map_ktiles(&x_map, x, (uint64_t)K, (uint64_t)M, kUmma2Tok / 2, 2);
     if (st) return st;
     static int configured_smem[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    if (dev < 0 || dev >= 64) return GPTQ_ERR_UNSUPPORTED;
-    if (configured_smem[dev] < plan.smem_bytes) {
-        e = cudaFuncSetAttribute(umma2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(umma2_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        configured_smem[dev] = plan.smem_bytes;
-    }
+    const int cfg_st = ensure_dynamic_smem((const void *)umma2_kernel, configured_smem, plan.smem_bytes);
+    if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
     cfg.blockDim = dim3(kUmma2Threads);

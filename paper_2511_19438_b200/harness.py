@@ -61,7 +61,7 @@ class WorkspaceHolder:
         if self.buf is None or self.buf.numel() < nbytes:
             torch.cuda.synchronize()
             self.buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
-        # registering is idempotent and cheap (it re-zeroes the 16 KB ticket area on the stream)
+        # registering is idempotent and cheap (a host-side pointer swap)
         B.check(B.gptq_set_workspace(self.buf, self.buf.numel()), "gptq_set_workspace")
 
     def ensure_for(self, M: int, D: DeviceLinear) -> None:

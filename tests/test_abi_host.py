@@ -223,3 +223,15 @@ def test_plan_rejects_bad_arguments():
     assert B.gptq_plan(1, 4096, 4096, 32, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_plan_cta_range(10, 11, 0)[0] == B.GPTQ_ERR_SHAPE
     assert B.gptq_plan_panel_owners(10, 5, 3, 0)[0] == B.GPTQ_ERR_SHAPE
+
+
+def test_plan_names_the_kernel():
+    """The planner names the kernel instantiation a profiler would print; bench.py attributes time by it."""
+    for M, want in ((1, "splitk_kernel<1>"), (8, "splitk_kernel<1>"), (16, "splitk_kernel<2>"),
+                    (17, "umma_kernel<32,3,1,2>"), (64, "umma_kernel<64,4,1,2>"), (128, "umma_kernel<128,4,1,2>"),
+                    (2048, "umma_kernel<256,4,1,2>")):
+        st, pl = B.gptq_plan(M, 4096, 4096, 128, 0, 148)
+        assert st == B.GPTQ_OK and B.plan_kernel_name(pl) == want
+    for M, want in ((1, "streamk_kernel<1>"), (16, "streamk_kernel<2>"), (32, "streamk_kernel<4>"), (100, "streamk_kernel<8>")):
+        st, pl = B.gptq_plan_noalloc(M, 1024, 1024, 128, 0, 148)
+        assert st == B.GPTQ_OK and B.plan_kernel_name(pl) == want

@@ -104,8 +104,8 @@ def test_repack_rejects_bad_g_idx():
     L_un = wl.QuantLinear(L.K, L.N, 128, L.qweight, L.qzeros, L.scales, uneven, 0)
     with pytest.raises(B.GptqError) as e:
         H.upload_and_repack(L_un)
-    assert e.value.status == B.GPTQ_ERR_UNSUPPORTED
-    assert B.gptq_check_status() == B.GPTQ_OK     # the flag was cleared
+    assert e.value.status == B.GPTQ_ERR_GIDX      # one code for both violations, as the header says
+    assert B.gptq_check_status() == B.GPTQ_OK     # the g_idx check has a status word of its own
     H.upload_and_repack(L)                        # and a valid layer still works
 
 
@@ -339,44 +339,97 @@ def test_config1_full_compare(ws):
     assert abs(y.astype(np.float64).std() / math.sqrt(K * 42.5 * es2) - 1) < 0.05
 
 
+def full_check(L, x, y, M=None):
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128), L.K, M)
+
+
+def slab_check(L, x, y, n_rows, seed):
+    """A seeded set of whole rows of y (all N columns each) against the oracle: rows of a matmul are independent,
+    so this is an element-by-element compare of those rows, including every panel and the last column."""
+    M = x.shape[0]
+    r = np.random.default_rng(seed)
+    rows = np.unique(np.concatenate([[0, M - 1], r.integers(0, M, n_rows - 2)]))
+    want = oracle.gemm_f64(np.ascontiguousarray(x[rows]), L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert_close(y[rows], want, L.K, M)
+
+
 @pytest.mark.parametrize("name", list(wl.SHAPES_7B))
 def test_config2_llama7b_decode(name, ws):
+    """configs[1] in full: every output of the four 7B shapes at M = 1, 4, 8, 16."""
     K, N = wl.SHAPES_7B[name]
     L = wl.make_linear(K, N, seed=wl.seed_for("config2", name))
     D = H.upload_and_repack(L)
     for M in wl.DECODE_M:
         x = wl.make_x(M, K, wl.seed_for("config2-x", name, M))
         ws.ensure_for(M, D)
-        y = H.gemm(H.to_device(x), D).cpu().numpy()
-        sampled_check(L, x, y, 3000, seed=M)
-        if M == 1 and name in ("o", "down"):
-            assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128), K)
+        full_check(L, x, H.gemm(H.to_device(x), D).cpu().numpy())
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
 @pytest.mark.parametrize("name", list(wl.SHAPES_13B))
 def test_config3_act_order(name, ws):
+    """configs[2] in full: the 13B shapes with act-order at M = 1 and 8."""
     K, N = wl.SHAPES_13B[name]
     L = wl.make_linear(K, N, seed=wl.seed_for("config3", name), act_order=True)
     D = H.upload_and_repack(L)
     for M in wl.ACT_ORDER_M:
         x = wl.make_x(M, K, wl.seed_for("config3-x", name, M))
         ws.ensure_for(M, D)
-        y = H.gemm(H.to_device(x), D).cpu().numpy()
-        sampled_check(L, x, y, 3000, seed=M)
+        full_check(L, x, H.gemm(H.to_device(x), D).cpu().numpy())
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
-@pytest.mark.parametrize("name,M,act", [("o", 512, False), ("qkv", 1024, False), ("down", 2048, True),
-                                        ("gate_up", 4096, False), ("o", 4096, True)])
-def test_config4_prefill_sampled(name, M, act, ws):
+@pytest.mark.parametrize("act", [False, True])
+@pytest.mark.parametrize("name", list(wl.SHAPES_7B))
+def test_config4_prefill(name, act, ws):
+    """configs[3]: every (shape, M, act-order) combination.  M = 512 is compared in full; above that the oracle
+    would take minutes per case, so 64 seeded whole rows (all N columns) are compared instead."""
     K, N = wl.SHAPES_7B[name]
     L = wl.make_linear(K, N, seed=wl.seed_for("config4", name, act), act_order=act)
     D = H.upload_and_repack(L)
-    x = wl.make_x(M, K, wl.seed_for("config4-x", name, M))
-    ws.ensure_for(M, D)
-    y = H.gemm(H.to_device(x), D).cpu().numpy()
-    sampled_check(L, x, y, 4000, seed=M)
+    for M in wl.PREFILL_M:
+        x = wl.make_x(M, K, wl.seed_for("config4-x", name, M))
+        ws.ensure_for(M, D)
+        y = H.gemm(H.to_device(x), D).cpu().numpy()
+        if M == 512:
+            full_check(L, x, y)
+        else:
+            slab_check(L, x, y, 64, seed=M)
+    assert B.gptq_check_status() == B.GPTQ_OK
+
+
+def test_few_groups_tolerance_limit(ws):
+    """The documented limit of the stated tolerance (see gptq_gemm in the header): with K = 256 there are two groups
+    per column, the bar 1e-2 sqrt(K/4096) is a quarter of its value at K = 4096, and a column whose two scales are
+    both large can put single elements of a many-token product just outside it.  The shape is the one where that was
+    first seen; the test counts: almost all of the 5 million outputs are inside the bar, none is far outside."""
+    K, N, M = 256, 2432, 2040
+    L = wl.make_linear(K, N, seed=wl.seed_for("tail", K, N, False))
+    x = wl.make_x(M, K, wl.seed_for("tail-x", K, M))
+    y, _ = run_gemm(L, x, ws)
+    y64 = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 128)
+    err = np.abs(y.astype(np.float64) - y64)
+    bar = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64)
+    outside = int((err > bar).sum())
+    assert outside <= 8, f"{outside} of {err.size} outputs outside the stated tolerance"
+    assert np.all(err <= 3 * bar), f"worst error {np.max(err / bar):.2f} x the stated tolerance"
+    # the rms error is what the fp16 rounding of the scaled weights predicts (about 1.4e-3 sqrt(K/4096))
+    assert np.sqrt(np.mean(err ** 2)) < 2.5e-3 * math.sqrt(K / 4096) + 2.0 ** -11 * np.sqrt(np.mean(y64 ** 2))
+
+
+def test_bounded_wait_reports_timeout():
+    """A wait that nothing satisfies gives up after its limit, the kernel returns normally, and the status word
+    turns into GPTQ_ERR_TIMEOUT exactly once; the context stays usable."""
+    assert B.gptq_check_status() == B.GPTQ_OK
+    B.check(B.gptq_selftest_wait_timeout(200), "selftest launch")          # 200 microseconds
+    assert B.gptq_check_status() == B.GPTQ_ERR_TIMEOUT
+    assert "wait" in B.gptq_status_string(B.GPTQ_ERR_TIMEOUT)
+    assert B.gptq_check_status() == B.GPTQ_OK                               # cleared by the read
+    assert B.gptq_selftest_wait_timeout(0) == B.GPTQ_ERR_SHAPE
+    L = wl.make_linear(256, 128, seed=3)                                    # and matmuls still run
+    x = wl.make_x(2, 256, 4)
+    D = H.upload_and_repack(L)
+    full_check(L, x, H.gemm(H.to_device(x), D).cpu().numpy())
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
@@ -453,15 +506,16 @@ def test_dependent_chain_in_a_graph(M, ws):
     assert_close(y2.cpu().numpy(), oracle.gemm_f64(y1_np, L2.qweight, L2.qzeros, L2.scales, None, 128), N1)
 
 
-@pytest.mark.parametrize("M", wl.STEP_M)
-def test_config5_decode_step_layers(M, ws):
-    """Layers 0 and 31 of the 32-layer step (distinct seeded weights per layer)."""
-    for layer in (0, 31):
-        for name, (K, N) in wl.SHAPES_7B.items():
-            L = wl.make_linear(K, N, seed=wl.seed_for("config5", layer, name))
-            D = H.upload_and_repack(L)
+@pytest.mark.parametrize("layer", range(32))
+def test_config5_decode_step_layer(layer, ws):
+    """configs[4]: all 128 matmuls of the 32-layer step (distinct seeded weights per layer) in full at M = 1 and 8;
+    at M = 32 and 64 layers 0 and 31 in full."""
+    Ms = wl.STEP_M if layer in (0, 31) else tuple(M for M in wl.STEP_M if M <= 8)
+    for name, (K, N) in wl.SHAPES_7B.items():
+        L = wl.make_linear(K, N, seed=wl.seed_for("config5", layer, name))
+        D = H.upload_and_repack(L)
+        for M in Ms:
             x = wl.make_x(M, K, wl.seed_for("config5-x", layer, name, M))
             ws.ensure_for(M, D)
-            y = H.gemm(H.to_device(x), D).cpu().numpy()
-            sampled_check(L, x, y, 1500, seed=layer * 100 + M)
+            full_check(L, x, H.gemm(H.to_device(x), D).cpu().numpy())
     assert B.gptq_check_status() == B.GPTQ_OK

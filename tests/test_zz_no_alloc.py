@@ -39,7 +39,12 @@ def noalloc_scratch_need(M, N, K, act):
     return pl.workspace_bytes
 
 
-@pytest.mark.parametrize("K,N,M,act", [(4096, 4096, 1, False), (4096, 4096, 8, False), (2560, 1280, 5, True)])
+# M = 1 .. 8 run streamk_kernel<1>, 9 .. 16 <2>, 17 .. 32 <4>, 33 .. 64 <8>; above 64 rows the call loops over chunks
+# of 64 that reuse the tickets and partial tiles
+@pytest.mark.parametrize("K,N,M,act", [(4096, 4096, 1, False), (4096, 4096, 8, False), (2560, 1280, 5, True),
+                                        (4096, 4096, 16, False), (1024, 512, 12, True), (1024, 512, 24, False),
+                                        (1024, 512, 40, True), (2048, 768, 64, False), (1024, 512, 100, False),
+                                        (1024, 512, 130, True)])
 def test_noalloc_matches_gemm_on_two_calls_in_a_row(K, N, M, act):
     L = wl.make_linear(K, N, seed=wl.seed_for("noalloc", K, N, act), act_order=act)
     D = H.upload_and_repack(L)
@@ -52,9 +57,13 @@ def test_noalloc_matches_gemm_on_two_calls_in_a_row(K, N, M, act):
         x = H.to_device(x_np)
         want = H.gemm(x, D)                                 # existing entry point, caller's workspace
         y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.check(B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, N, K, 128, act),
                 "gptq_gemm_noalloc")
         assert B.gptq_check_status() == B.GPTQ_OK
+        if call == 1:                                       # (the first call on a device may load the kernel image)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
         assert within_stated_tolerance(y.cpu().numpy(), want.cpu().numpy().astype(np.float64), K), \
             f"call {call}: differs from gptq_gemm"
         y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
