@@ -38,7 +38,7 @@ def _load():
         lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
         lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
-                     "oracle_gemm_f64", "oracle_gemm_f64_at"):
+                     "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -89,8 +89,9 @@ def unpack_z(qzeros: np.ndarray) -> np.ndarray:
     return out
 
 
-def dequant_f32(qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
-    """fp32[K, N] dequantised weights; ``g_idx`` None means no act-order."""
+def dequant_f32(qweight, qzeros, scales, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp32[K, N] dequantised weights; ``g_idx`` None means no act-order.  With ``zeros_minus_one`` the stored
+    zero-point nibble is z - 1 (older checkpoints) and a separate oracle function is called."""
     qweight = _i32(qweight)
     R, N = qweight.shape
     K = R * 8
@@ -99,13 +100,14 @@ def dequant_f32(qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
     scales = _f16(scales, (G, N))
     g = None if g_idx is None else _i32(g_idx, (K,))
     out = np.empty((K, N), dtype=np.float32)
-    _load().oracle_dequant_f32(_p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(K),
+    fn = _load().oracle_dequant_f32_v1 if zeros_minus_one else _load().oracle_dequant_f32
+    fn(_p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(K),
                                ctypes.c_int(N), ctypes.c_int(group_size), _p(out))
     return out
 
 
-def gemm_f64(x, qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
-    """fp64[M, N] = x[M, K] . dequant(W)[K, N], k ascending."""
+def gemm_f64(x, qweight, qzeros, scales, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp64[M, N] = x[M, K] . dequant(W)[K, N], k ascending (``zeros_minus_one``: see dequant_f32)."""
     qweight = _i32(qweight)
     R, N = qweight.shape
     K = R * 8
@@ -117,7 +119,8 @@ def gemm_f64(x, qweight, qzeros, scales, g_idx, group_size: int) -> np.ndarray:
     scales = _f16(scales, (G, N))
     g = None if g_idx is None else _i32(g_idx, (K,))
     out = np.empty((M, N), dtype=np.float64)
-    _load().oracle_gemm_f64(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M),
+    fn = _load().oracle_gemm_f64_v1 if zeros_minus_one else _load().oracle_gemm_f64
+    fn(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M),
                             ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size), _p(out))
     return out
 

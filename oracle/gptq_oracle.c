@@ -152,3 +152,44 @@ void oracle_gemm_f64_at(const uint16_t *x, const int32_t *qweight, const int32_t
         y_out[i] = acc;
     }
 }
+
+/* ---- format variant: zero points stored minus one -------------------------------------------
+ * Older GPTQ checkpoints store z - 1 in the zero-point nibble and the kernels that read them add
+ * the one back; the paper (Section 1, Section 4.2) does not say which of the two conventions its
+ * checkpoints use, so both are defined.  The functions above take the stored nibble as the zero
+ * point; the two below take stored + 1 (1..16), everything else unchanged. */
+static inline float dequant_one_v1(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                                   const int32_t *g_idx, int N, int group_size, int k, int n)
+{
+    int g = group_of(g_idx, k, group_size);
+    int q = (int)nibble(qweight[(size_t)(k >> 3) * N + n], k & 7);
+    int z = (int)nibble(qzeros[(size_t)g * (N / 8) + (n >> 3)], n & 7) + 1;
+    float s = oracle_half_to_float(scales[(size_t)g * N + n]);
+    return (float)(q - z) * s;
+}
+
+void oracle_dequant_f32_v1(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                           const int32_t *g_idx, int K, int N, int group_size, float *w_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            w_out[(size_t)k * N + n] = dequant_one_v1(qweight, qzeros, scales, g_idx, N, group_size, k, n);
+}
+
+void oracle_gemm_f64_v1(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                        const uint16_t *scales, const int32_t *g_idx,
+                        int M, int N, int K, int group_size, double *y_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; n++) {
+        for (int m = 0; m < M; m++) {
+            double acc = 0.0;
+            for (int k = 0; k < K; k++) {
+                float w = dequant_one_v1(qweight, qzeros, scales, g_idx, N, group_size, k, n);
+                acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+            }
+            y_out[(size_t)m * N + n] = acc;
+        }
+    }
+}

@@ -276,3 +276,48 @@ def test_generator_distributions():
     assert np.array_equal(np.bincount(L.g_idx, minlength=8), np.full(8, 128))
     s = L.scales.astype(np.float64)
     assert s.min() >= 0.002 - 1e-5 and abs(s.mean() - (0.002 + 0.01 * math.sqrt(2 / math.pi))) < 2e-4
+
+
+# --------------------------------------------------------------------------- zero points stored minus one
+def test_v1_zeros_hand_values(tiny):
+    """The hand-packed layer read with the older convention (stored nibble = z - 1): every zero point is one
+    larger than the hand table, so every weight is one scale smaller; the stored 15 of group 1, column 7 means 16."""
+    q, z, s, gs = tiny["q"], tiny["z"], tiny["scales"].astype(np.float64), tiny["gs"]
+    w = oracle.dequant_f32(tiny["qweight"], tiny["qzeros"], tiny["scales"], None, gs, zeros_minus_one=True)
+    for k in range(16):
+        for n in range(8):
+            assert float(w[k, n]) == float((q[k, n] - (z[k // gs, n] + 1)) * s[k // gs, n]), (k, n)
+    assert w[0, 0] == -2.0          # (0 - (1 + 1)) * 1
+    assert w[7, 5] == 1.0           # (15 - (6 + 1)) * 0.125
+    assert w[15, 7] == -0.1875      # (13 - (15 + 1)) * 0.0625: the stored 15 is the zero point 16
+    assert w[8, 3] == 2.0           # (15 - (13 + 1)) * 2
+
+
+def test_v1_zeros_repacked_by_hand_equal_plain_reading(tiny):
+    """Pack z - 1 digit by digit (test-local packer) where every z >= 1: the older reading of those words must give
+    bit for bit what the plain reading gives on the original words."""
+    z = tiny["z"].copy()
+    z[z == 0] = 1                                   # the hand table has one zero point equal to 0
+    qz_plain = local_pack_n(z)
+    qz_minus_one = local_pack_n(z - 1)
+    a = oracle.dequant_f32(tiny["qweight"], qz_plain, tiny["scales"], tiny["g_idx"], tiny["gs"])
+    b = oracle.dequant_f32(tiny["qweight"], qz_minus_one, tiny["scales"], tiny["g_idx"], tiny["gs"], zeros_minus_one=True)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_v1_gemm_is_plain_gemm_minus_scaled_group_sums_of_x():
+    """(q - z - 1) s = (q - z) s - s, so y_v1 = y_plain - sum_g s[g, n] * sum_{k in g} x[m, k]: an identity that ties the
+    second matmul function to the first through a computation done here in numpy fp64."""
+    K, N, M, gs = 256, 24, 3, 32
+    L = wl.make_linear(K, N, seed=91, group_size=gs, act_order=True)
+    x = wl.make_x(M, K, 92)
+    y_plain = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs)
+    y_v1 = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=True)
+    xs = np.zeros((M, K // gs))
+    for k in range(K):
+        xs[:, L.g_idx[k]] += x[:, k].astype(np.float64)
+    corr = xs @ L.scales.astype(np.float64)
+    assert np.allclose(y_v1, y_plain - corr, rtol=0, atol=1e-9 * np.abs(y_plain).max())
+    # and it is the matmul of its own dequantised weights
+    w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=True).astype(np.float64)
+    assert np.allclose(y_v1, x.astype(np.float64) @ w, rtol=1e-13, atol=1e-12)
