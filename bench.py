@@ -47,10 +47,10 @@ FALLBACK_TFLOPS = 1590.0
 # on (`--print-digest`); `traffic` is that ratio times the timed launches' algorithmic bytes, and
 # null once the sources have changed since the capture.
 NCU_TRAFFIC = {
-    "splitk_kernel<1>": {"digest": "ca9079fd443538ec", "ratio": 1.0005, "Ms": (1,),
+    "splitk_kernel<1,1>": {"digest": "ca9079fd443538ec", "ratio": 1.0005, "Ms": (1,),
                          "source": "ncu capture profiles/splitk_kernel_decode7b.md (M = 1, the four 7B shapes): "
                                    "dram bytes / algorithmic bytes x algorithmic bytes per timed launch"},
-    "umma_kernel<256,4,1,2>": {"digest": "7568e8af7d5bd1cb", "ratio": 0.74, "Ms": (2048,),
+    "umma_kernel<256,4,1,2,1>": {"digest": "7568e8af7d5bd1cb", "ratio": 0.74, "Ms": (2048,),
                                "source": "ncu capture profiles/umma_kernel_prefill7b.md (qkv, M = 2048, main + tail "
                                          "launch; y partly still in L2): ratio x algorithmic bytes per timed launch"},
 }
@@ -69,8 +69,8 @@ WORKLOADS = {
 
 # the header files each captured kernel is built from (its own file and what that includes)
 KERNEL_SOURCES = {
-    "splitk_kernel<1>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh"),
-    "umma_kernel<256,4,1,2>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh", "gptq_umma.cuh"),
+    "splitk_kernel<1,1>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh"),
+    "umma_kernel<256,4,1,2,1>": ("gptq_common.cuh", "gptq_tma.cuh", "gptq_streamk.cuh", "gptq_splitk.cuh", "gptq_umma.cuh"),
 }
 
 

@@ -75,15 +75,30 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
                      float *w_out, int N, int K, int group_size, int act_order, int repacked,
                      void *stream);
 
+/* Format variants.  The paper (Section 1, Section 4.2) names 4-bit GPTQ without fixing the checkpoint conventions,
+ * and checkpoints of the same family differ in two of them:
+ *   - group_size: 128 (all of the paper's models), 64 or 32 rows per scale / zero point.  Every tiled entry point
+ *     accepts these three; gptq_gemm_noalloc and the CTA-pair switch accept 128 only.
+ *   - the zero point: stored as is (default), or stored minus one (older checkpoints: the kernels add the one
+ *     back, so a stored 15 means 16).  Pass GPTQ_FORMAT_ZEROS_MINUS_ONE to the _format entry points below.
+ * gptq_repack_format records the flag in a 16-byte trailer behind the tiled zero points (counted in
+ * gptq_repack_bytes(1, ...)), so gptq_gemm and gptq_dequant_f32(repacked = 1) need no format argument. */
+#define GPTQ_FORMAT_ZEROS_MINUS_ONE 1
+/* gptq_dequant_f32 with a format for canonical inputs (repacked = 0); with repacked = 1 the trailer decides and
+ * `format` must be 0 or equal to what the layer was repacked with. */
+int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                            float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
+                            void *stream);
+
 /* ---- one-time repack into the tiled layout the matmul kernels stream ---------------- */
 
 /* Byte size of each gptq_repack output: which = 0 qweight_out, 1 qzeros_out, 2 scales_out,
- * 3 perm_out (0 bytes unless act_order).  Sizes equal the canonical ones.  Returns 0 for an
- * invalid argument. */
+ * 3 perm_out (0 bytes unless act_order).  Sizes equal the canonical ones, plus 16 bytes of format trailer
+ * behind the zero points.  Returns 0 for an invalid argument. */
 size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order);
 
 /* Re-tiles a canonical layer (what Section 3.2 / Algorithm 2 achieve with wider loads of the original layout is
- * achieved here by storing the weights in the order the kernels stream them).  Fast-path requirements: group_size == 128, K % 128 == 0,
+ * achieved here by storing the weights in the order the kernels stream them).  Fast-path requirements: group_size 128, 64 or 32, K % 128 == 0,
  * N % 128 == 0 (else GPTQ_ERR_UNSUPPORTED).  With act_order != 0 the rows are stably sorted
  * by g_idx so that each group's rows are contiguous; perm_out[i] = original index of sorted
  * row i (int32[K]).  g_idx is range-checked on the device and every group must have exactly
@@ -92,6 +107,10 @@ size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order)
 int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
                 void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out,
                 int N, int K, int group_size, int act_order, void *stream);
+/* The same with a format (see above); gptq_repack is format 0. */
+int gptq_repack_format(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                       void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out,
+                       int N, int K, int group_size, int act_order, int format, void *stream);
 
 /* ---- the matmul ---------------------------------------------------------------------- */
 

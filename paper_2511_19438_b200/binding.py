@@ -21,6 +21,7 @@ if not os.path.exists(LIB_PATH):
 
 _lib = ctypes.CDLL(LIB_PATH)
 
+GPTQ_FORMAT_ZEROS_MINUS_ONE = 1
 GPTQ_OK = 0
 GPTQ_ERR_NULL = -1
 GPTQ_ERR_SHAPE = -2
@@ -60,7 +61,9 @@ _SIGNATURES = {
     "gptq_last_cuda_error": (_i, []),
     "gptq_unpack_u8": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "gptq_dequant_f32": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "gptq_dequant_f32_format": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp]),
     "gptq_repack_bytes": (_sz, [_i, _i, _i, _i, _i]),
+    "gptq_repack_format": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_repack": (_i, [_vp] * 8 + [_i, _i, _i, _i, _vp]),
     "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "gptq_set_workspace": (_i, [_vp, _sz]),
@@ -133,6 +136,19 @@ def gptq_dequant_f32(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, ac
                      stream=None) -> int:
     return _lib.gptq_dequant_f32(_ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(w_out), N, K,
                                  group_size, int(act_order), int(repacked), _stream(stream))
+
+
+def gptq_dequant_f32_format(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked, fmt,
+                            stream=None) -> int:
+    return _lib.gptq_dequant_f32_format(_ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(w_out), N, K,
+                                        group_size, int(act_order), int(repacked), int(fmt), _stream(stream))
+
+
+def gptq_repack_format(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
+                       group_size, act_order, fmt, stream=None) -> int:
+    return _lib.gptq_repack_format(_ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(qweight_out),
+                                   _ptr(qzeros_out), _ptr(scales_out), _ptr(perm_out), N, K, group_size,
+                                   int(act_order), int(fmt), _stream(stream))
 
 
 def gptq_repack_bytes(which, N, K, group_size, act_order) -> int:

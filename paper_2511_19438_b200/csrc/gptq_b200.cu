@@ -63,7 +63,8 @@ static int check_shape(int M, int N, int K, int group_size)
 }
 static int check_fast_path(int N, int K, int group_size)
 {
-    if (group_size != kGroup || N % kPanel || K % kGroup) return GPTQ_ERR_UNSUPPORTED;
+    if ((group_size != 128 && group_size != 64 && group_size != 32) || N % kPanel || K % kGroup)
+        return GPTQ_ERR_UNSUPPORTED;
     if (N / kPanel > (int)(kTicketAreaBytes / sizeof(int))) return GPTQ_ERR_UNSUPPORTED;
     return GPTQ_OK;
 }
@@ -151,7 +152,7 @@ const char *gptq_status_string(int status)
     case GPTQ_ERR_NULL: return "a required pointer is NULL";
     case GPTQ_ERR_SHAPE: return "invalid shape (need M>=1, K%8==0, N%8==0, K%group_size==0)";
     case GPTQ_ERR_ALIGN: return "a pointer is not 16-byte aligned";
-    case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 128, N%128==0, K%128==0, equal groups)";
+    case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 128, 64 or 32, N%128==0, K%128==0)";
     case GPTQ_ERR_LAYOUT: return "invalid layout selector or flag";
     case GPTQ_ERR_GIDX: return "g_idx entry out of range, or groups of unequal size";
     case GPTQ_ERR_WORKSPACE: return "workspace missing or too small (see gptq_workspace_bytes)";
@@ -181,6 +182,14 @@ int gptq_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out
 int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
                      float *w_out, int N, int K, int group_size, int act_order, int repacked, void *stream)
 {
+    return gptq_dequant_f32_format(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked, 0, stream);
+}
+
+int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                            float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
+                            void *stream)
+{
+    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !w_out || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
     if (st) return st;
@@ -189,7 +198,7 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
         st = check_fast_path(N, K, group_size);
         if (st) return st;
     }
-    return launch_dequant_f32(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked,
+    return launch_dequant_f32(qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, repacked, format,
                               (cudaStream_t)stream);
 }
 
@@ -199,7 +208,7 @@ size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order)
     const size_t G = (size_t)(K / group_size);
     switch (which) {
     case 0: return (size_t)K / 8 * N * 4;
-    case 1: return G * (N / 8) * 4;
+    case 1: return G * (N / 8) * 4 + kTrailerBytes;   // + the format trailer
     case 2: return G * N * 2;
     case 3: return act_order ? (size_t)K * 4 : 0;
     default: return 0;
@@ -210,6 +219,15 @@ int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scale
                 void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
                 int group_size, int act_order, void *stream)
 {
+    return gptq_repack_format(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
+                              group_size, act_order, 0, stream);
+}
+
+int gptq_repack_format(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                       void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
+                       int group_size, int act_order, int format, void *stream)
+{
+    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out) return GPTQ_ERR_NULL;
     if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
@@ -220,7 +238,7 @@ int gptq_repack(const int32_t *qweight, const int32_t *qzeros, const void *scale
     if (qweight_out == (const void *)qweight || qzeros_out == (const void *)qzeros || scales_out == scales)
         return GPTQ_ERR_LAYOUT;
     return launch_repack(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
-                         act_order, (cudaStream_t)stream);
+                         group_size, act_order, format, (cudaStream_t)stream);
 }
 
 static void set_kernel_name(gptq_plan_t *out, const char *fmt, int a, int b = 0, int c = 0, int d = 0)
@@ -251,14 +269,15 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
         out->tail_ctas = up.tail_tiles * up.tail_S;
         out->tail_cluster_size = up.tail_S;
         out->split_panels = up.S > 1 ? N / kPanel : 0;
-        if (g_use_cta_pairs.load() && umma2_applicable(M, N))
+        if (g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup)
             set_kernel_name(out, "umma2_kernel", 0);
         else
-            set_kernel_name(out, "umma_kernel<%d,%d,%d,%d>", up.tok, umma_a_stages(up.tok, up.np), up.np, up.sets);
+            snprintf(out->kernel_name, sizeof(out->kernel_name), "umma_kernel<%d,%d,%d,%d,%d>", up.tok,
+                     umma_a_stages(up.tok, up.np), up.np, up.sets, kGroup / group_size);
         return GPTQ_OK;
     }
     const int rows = M < kStreamKMaxRows ? M : kStreamKMaxRows;
-    const SplitKPlan pl = plan_splitk(rows, N, K, sm_count);
+    const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sm_count);
     out->kernel = 1;
     out->m_tile = pl.m_tile;
     out->m_chunks = (M + kStreamKMaxRows - 1) / kStreamKMaxRows;
@@ -271,7 +290,7 @@ int gptq_plan(int M, int N, int K, int group_size, int act_order, int sm_count, 
     out->cluster_size = pl.S;
     out->tail_ctas = 0;
     out->tail_cluster_size = 1;
-    set_kernel_name(out, "splitk_kernel<%d>", pl.m_tile / 8);
+    set_kernel_name(out, "splitk_kernel<%d,%d>", pl.m_tile / 8, pl.sub);
     return GPTQ_OK;
 }
 
@@ -282,6 +301,7 @@ int gptq_plan_noalloc(int M, int N, int K, int group_size, int act_order, int sm
     if (st) return st;
     st = check_fast_path(N, K, group_size);
     if (st) return st;
+    if (group_size != kGroup) return GPTQ_ERR_UNSUPPORTED;   // the stream-K kernel is built for group size 128 only
     if (sm_count < 1) return GPTQ_ERR_SHAPE;
     const StreamKGemmPlan gp = make_streamk_plan(M, N, K, act_order, sm_count);
     out->kernel = 3;
@@ -368,17 +388,17 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
         xin = x_perm;
     }
     if (M >= kUmmaMinTokens) {
-        if (g_use_cta_pairs.load() && umma2_applicable(M, N)) {
+        if (g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
             const Umma2Plan p2 = plan_umma2(M, N, K);
             return launch_umma2(xin, qweight, qzeros, scales, (__half *)y, M, N, K, p2, s);
         }
         // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
-        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, pl, s);
+        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
-        const SplitKPlan pl = plan_splitk(rows, N, K, sms);
+        const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sms);
         st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
                            pl, s);
         if (st) return st;
@@ -438,6 +458,7 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
         return GPTQ_ERR_ALIGN;
     st = check_fast_path(N, K, group_size);
     if (st) return st;
+    if (group_size != kGroup) return GPTQ_ERR_UNSUPPORTED;   // the stream-K kernel is built for group size 128 only
     int dev, sms;
     st = current_device_sms(&dev, &sms);
     if (st) return st;

@@ -32,14 +32,28 @@ namespace gptq {
 //  * tcgen05 kernel: the thread that owns column n (TMEM lane) reads 8 bytes (h fixed, j=0,1)
 //    from each of the four chunks 4g+t4: 64 consecutive rows of its column.
 //
-// Scales of an item: fp16[128] at position 16u + 2g + h  <- column 128p + 16u + g + 8h.
-// Zeros of an item: 64 bytes, byte 8u + g = z[col g] | z[col g+8] << 4.
+// Scales of an item: per quantisation group inside its 128 rows (SUB = 128 / group_size of them: 1, 2 or 4)
+// fp16[128] at position 16u + 2g + h  <- column 128p + 16u + g + 8h; the SUB blocks follow each other.
+// Zeros of an item: per group 64 bytes, byte 8u + g = z[col g] | z[col g+8] << 4.
+// qzeros_out ends with a 16-byte trailer {magic, flags, group_size, 0} (see TiledTrailer): the tiled buffers
+// describe themselves, so gptq_gemm needs no format argument.
 // ----------------------------------------------------------------------------------------
-constexpr int kGroup = 128;          // rows per group (fast path)
+constexpr int kGroup = 128;          // rows per item (one quantisation group at group_size 128, two at 64, four at 32)
 constexpr int kPanel = 128;          // columns per panel
 constexpr int kItemWBytes = 8192;    // packed weights of one item
-constexpr int kItemSBytes = 256;     // scales of one item
-constexpr int kItemZBytes = 64;      // packed zeros of one item
+constexpr int kItemSBytes = 256;     // scales of one group of one item
+constexpr int kItemZBytes = 64;      // packed zeros of one group of one item
+constexpr int kTrailerBytes = 16;
+constexpr uint32_t kTrailerMagic = 0x51545047u;   // "GPTQ"
+constexpr uint32_t kFormatZerosMinusOne = 1u;     // == GPTQ_FORMAT_ZEROS_MINUS_ONE
+struct TiledTrailer {
+    uint32_t magic, flags, group_size, reserved;
+};
+// bytes of the tiled zero points without the trailer
+__host__ __device__ inline size_t tiled_zero_bytes(int N, int K, int group_size)
+{
+    return (size_t)(K / group_size) * (size_t)(N / 2);
+}
 constexpr int kBlockWBytes = 4096;   // one K64 block of one panel
 constexpr int kUnitBytes = 512;
 
@@ -56,19 +70,20 @@ __host__ __device__ inline size_t repacked_word_offset(int i, int n, int G, int 
     size_t item = (size_t)p * G + grp;
     return item * kItemWBytes + (size_t)blk * kBlockWBytes + u * kUnitBytes + (4 * g + t4) * 16 + (j + 2 * h) * 4;
 }
-__host__ __device__ inline size_t repacked_scale_index(int grp, int n, int G)
+// grp counts quantisation groups (K / group_size of them, `groups` per column panel)
+__host__ __device__ inline size_t repacked_scale_index(int grp, int n, int groups)
 {
     int p = n / kPanel, nn = n % kPanel;
     int u = nn / 16, c16 = nn % 16, g = c16 & 7, h = c16 >> 3;
-    return ((size_t)p * G + grp) * kPanel + 16 * u + 2 * g + h;
+    return ((size_t)p * groups + grp) * kPanel + 16 * u + 2 * g + h;
 }
 // byte index and nibble (0 = low) of the zero point of (grp, n)
-__host__ __device__ inline size_t repacked_zero_byte(int grp, int n, int G, int *hi)
+__host__ __device__ inline size_t repacked_zero_byte(int grp, int n, int groups, int *hi)
 {
     int p = n / kPanel, nn = n % kPanel;
     int u = nn / 16, c16 = nn % 16, g = c16 & 7;
     *hi = c16 >> 3;
-    return ((size_t)p * G + grp) * kItemZBytes + 8 * u + g;
+    return ((size_t)p * groups + grp) * kItemZBytes + 8 * u + g;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -266,10 +281,11 @@ StreamKPlan plan_streamk(int m_rows, int N, int K, int sm_count);
 int launch_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_out, uint8_t *z_out, int N, int K,
                      int G, cudaStream_t s);
 int launch_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
-                       float *w_out, int N, int K, int group_size, int act_order, int repacked, cudaStream_t s);
+                       float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
+                       cudaStream_t s);
 int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
                   void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
-                  int act_order, cudaStream_t s);
+                  int group_size, int act_order, int format, cudaStream_t s);
 int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, int K, cudaStream_t s);
 int launch_streamk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
                    int M, int N, int K, const StreamKPlan &plan, float *partials, int *tickets, cudaStream_t s);

@@ -49,58 +49,63 @@ int launch_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_o
 // One thread per (k, n).  float(q - z) * float(s): a single fp32 multiply whose result is exact.
 __global__ void dequant_canonical_kernel(const int32_t *__restrict__ qweight, const int32_t *__restrict__ qzeros,
                                          const __half *__restrict__ scales, const int32_t *__restrict__ g_idx,
-                                         float *__restrict__ w_out, int N, int K, int group_size)
+                                         float *__restrict__ w_out, int N, int K, int group_size, int z_add)
 {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)K * N) return;
     int k = (int)(idx / N), n = (int)(idx % N);
     int g = g_idx ? g_idx[k] : k / group_size;
     int q = (int)(((uint32_t)qweight[(size_t)(k >> 3) * N + n] >> (4 * (k & 7))) & 15u);
-    int z = (int)(((uint32_t)qzeros[(size_t)g * (N / 8) + (n >> 3)] >> (4 * (n & 7))) & 15u);
+    int z = (int)(((uint32_t)qzeros[(size_t)g * (N / 8) + (n >> 3)] >> (4 * (n & 7))) & 15u) + z_add;
     w_out[idx] = __fmul_rn((float)(q - z), __half2float(scales[(size_t)g * N + n]));
 }
 
 // Tiled layout: thread per (sorted row i, column n); the row goes back to its original index.
 __global__ void dequant_tiled_kernel(const uint8_t *__restrict__ qweight, const uint8_t *__restrict__ qzeros,
                                      const __half *__restrict__ scales, const int32_t *__restrict__ perm,
-                                     float *__restrict__ w_out, int N, int K)
+                                     float *__restrict__ w_out, int N, int K, int group_size)
 {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)K * N) return;
     int i = (int)(idx / N), n = (int)(idx % N);
-    int G = K / kGroup, grp = i / kGroup;
+    int groups = K / group_size, grp = i / group_size;
     int slot, hi;
-    size_t off = repacked_word_offset(i, n, G, &slot);
+    size_t off = repacked_word_offset(i, n, K / kGroup, &slot);
     uint32_t word = *reinterpret_cast<const uint32_t *>(qweight + off);
     int q = (int)((word >> (4 * slot)) & 15u);
-    uint8_t zb = qzeros[repacked_zero_byte(grp, n, G, &hi)];
-    int z = hi ? (zb >> 4) : (zb & 15);
-    float s = __half2float(scales[repacked_scale_index(grp, n, G)]);
+    // the trailer says whether the stored zero points are one too small
+    const TiledTrailer *tr = reinterpret_cast<const TiledTrailer *>(qzeros + tiled_zero_bytes(N, K, group_size));
+    uint8_t zb = qzeros[repacked_zero_byte(grp, n, groups, &hi)];
+    int z = (hi ? (zb >> 4) : (zb & 15)) + (int)(tr->flags & kFormatZerosMinusOne);
+    float s = __half2float(scales[repacked_scale_index(grp, n, groups)]);
     int k = perm ? perm[i] : i;
     w_out[(size_t)k * N + n] = __fmul_rn((float)(q - z), s);
 }
 
 int launch_dequant_f32(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
-                       float *w_out, int N, int K, int group_size, int act_order, int repacked, cudaStream_t s)
+                       float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
+                       cudaStream_t s)
 {
     const int T = 256;
     size_t total = (size_t)K * N;
     unsigned blocks = (unsigned)((total + T - 1) / T);
     if (repacked)
         dequant_tiled_kernel<<<blocks, T, 0, s>>>((const uint8_t *)qweight, (const uint8_t *)qzeros,
-                                                  (const __half *)scales, act_order ? g_idx : nullptr, w_out, N, K);
+                                                  (const __half *)scales, act_order ? g_idx : nullptr, w_out, N, K,
+                                                  group_size);
     else
         dequant_canonical_kernel<<<blocks, T, 0, s>>>((const int32_t *)qweight, (const int32_t *)qzeros,
                                                       (const __half *)scales, act_order ? g_idx : nullptr, w_out,
-                                                      N, K, group_size);
+                                                      N, K, group_size, (format & (int)kFormatZerosMinusOne) ? 1 : 0);
     return record_cuda_error(cudaGetLastError());
 }
 
 // ------------------------------------------------------------------------------ act-order sort
 // perm = stable argsort(g_idx).  Thread k counts the keys that sort before its own:
 // rank(k) = #{k' : g[k'] < g[k]} + #{k' < k : g[k'] == g[k]}.  O(K^2) compares, one-time, K <= ~16k.
-// Also checks 0 <= g[k] < G and that every group has exactly 128 rows.
-__global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *__restrict__ perm, int K, int G)
+// Also checks 0 <= g[k] < G and that every group has exactly group_size rows.
+__global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *__restrict__ perm, int K, int G,
+                                    int group_size)
 {
     extern __shared__ int32_t tile[];
     int k = blockIdx.x * blockDim.x + threadIdx.x;
@@ -125,7 +130,7 @@ __global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *
         atomicMax(&g_gidx_status, (int)kGidxOutOfRange);
         return;
     }
-    if (same_total != kGroup) atomicMax(&g_gidx_status, (int)kGidxUnequalGroups);
+    if (same_total != group_size) atomicMax(&g_gidx_status, (int)kGidxUnequalGroups);
     int rank = below + same_before;
     if (rank >= 0 && rank < K) perm[rank] = k;
 }
@@ -163,11 +168,16 @@ __global__ void repack_weights_kernel(const int32_t *__restrict__ qweight, const
 }
 
 // One thread per (group, column): scale to its tiled position; thread with h == 0 also writes the
-// zero byte of its column pair.
+// zero byte of its column pair.  Thread 0 writes the trailer behind the zero points.
 __global__ void repack_meta_kernel(const int32_t *__restrict__ qzeros, const __half *__restrict__ scales,
-                                   uint8_t *__restrict__ z_out, __half *__restrict__ s_out, int N, int G)
+                                   uint8_t *__restrict__ z_out, __half *__restrict__ s_out, int N, int G,
+                                   int group_size, uint32_t flags)
 {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx == 0) {
+        TiledTrailer tr{kTrailerMagic, flags, (uint32_t)group_size, 0u};
+        *reinterpret_cast<TiledTrailer *>(z_out + (size_t)G * (N / 2)) = tr;
+    }
     if (idx >= (size_t)G * N) return;
     int grp = (int)(idx / N), n = (int)(idx % N);
     s_out[repacked_scale_index(grp, n, G)] = scales[idx];
@@ -187,13 +197,13 @@ __global__ void repack_fence_kernel() {}
 
 int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
                   void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
-                  int act_order, cudaStream_t s)
+                  int group_size, int act_order, int format, cudaStream_t s)
 {
     const int T = 256;
-    int G = K / kGroup;
+    int G = K / group_size;
     if (act_order) {
         int blocks = (K + T - 1) / T;
-        argsort_gidx_kernel<<<blocks, T, T * sizeof(int32_t), s>>>(g_idx, perm_out, K, G);
+        argsort_gidx_kernel<<<blocks, T, T * sizeof(int32_t), s>>>(g_idx, perm_out, K, G, group_size);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return record_cuda_error(e);
         // one-time call: read the validation result before tiling with a possibly invalid perm
@@ -214,7 +224,8 @@ int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *sca
                                                                         (uint32_t *)qweight_out, N, K);
     size_t meta = (size_t)G * N;
     repack_meta_kernel<<<(unsigned)((meta + T - 1) / T), T, 0, s>>>(qzeros, (const __half *)scales,
-                                                                    (uint8_t *)qzeros_out, (__half *)scales_out, N, G);
+                                                                    (uint8_t *)qzeros_out, (__half *)scales_out, N, G,
+                                                                    group_size, (uint32_t)format);
     repack_fence_kernel<<<1, 32, 0, s>>>();
     return record_cuda_error(cudaGetLastError());
 }

@@ -90,24 +90,26 @@ struct SplitKArgs {
     int M, N, K, G;
     int S;                  // CTAs per panel = cluster size
     int stages;
+    const TiledTrailer *trailer;   // behind the tiled zero points
 };
 
 struct SplitKPlan {
-    int m_tile;     // 8, 16, 32 or 64
+    int m_tile;     // 8 or 16
+    int sub;        // quantisation groups per 128-row item: 128 / group_size
     int S;
     int stages;
     int ctas;       // panels * S
     int smem_bytes;
 };
 
-template <int MT>
-__global__ void __launch_bounds__(kStreamKThreads, MT <= 2 ? 3 : 1)
+template <int MT, int SUB>
+__global__ void __launch_bounds__(kStreamKThreads, 3)
 splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
-    constexpr int kStage = streamk_stage_bytes(MT);
+    constexpr int kStage = streamk_stage_bytes(MT, SUB);
     constexpr int kXTile = MT * 1024;                       // one K64 tile of x
-    constexpr int kOffW = streamk_x_bytes(MT), kOffS = kOffW + kItemWBytes, kOffZ = kOffS + kItemSBytes;
+    constexpr int kOffW = streamk_x_bytes(MT), kOffS = kOffW + kItemWBytes, kOffZ = kOffS + SUB * kItemSBytes;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_base;                  // stages x 8 B
@@ -149,14 +151,14 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         if (lane == 0) {
             const uint64_t policy = l2_policy_evict_first();
             tma_prefetch_descriptor(&x_map);
-            const uint32_t meta_bytes = kItemWBytes + kItemSBytes + kItemZBytes;
+            const uint32_t meta_bytes = kItemWBytes + SUB * (kItemSBytes + kItemZBytes);
             const int n_pre = n_items < stages ? n_items : stages;
             auto issue_weights = [&](int t, int s) {
                 const uint32_t dst = ring + s * kStage, bar = bar_full + 8 * s;
                 mbar_expect_tx(bar, meta_bytes);
                 bulk_g2s_hint(dst + kOffW, a.qweight + (size_t)t * kItemWBytes, kItemWBytes, bar, policy);
-                bulk_g2s_hint(dst + kOffS, a.scales + (size_t)t * kItemSBytes, kItemSBytes, bar, policy);
-                bulk_g2s_hint(dst + kOffZ, a.qzeros + (size_t)t * kItemZBytes, kItemZBytes, bar, policy);
+                bulk_g2s_hint(dst + kOffS, a.scales + (size_t)t * (SUB * kItemSBytes), SUB * kItemSBytes, bar, policy);
+                bulk_g2s_hint(dst + kOffZ, a.qzeros + (size_t)t * (SUB * kItemZBytes), SUB * kItemZBytes, bar, policy);
             };
             // weights never depend on earlier work in the stream: fill the ring before waiting on it
             for (int i = 0; i < n_pre; ++i) issue_weights(t0 + i, i);
@@ -179,6 +181,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
+        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // weights-side data: no need to wait
         pdl_wait();
         const int r = token_row_of_slot(g);
         const uint32_t w_off = kOffW + warp * kUnitBytes + lane * 16;
@@ -194,14 +197,13 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             const uint32_t st = ring + s * kStage;
             if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
 
-            float accg[MT][4];
-            uint32_t sc;
-            consume_item<MT>(st, w_off, s_off, z_off, x_off0, x_off1, accg, sc);
-            // release the stage, then fold the group sum into the running sum with the group's scale
+            ItemSums<MT, SUB> sums;
+            consume_item<MT, SUB>(st, w_off, s_off, z_off, x_off0, x_off1, z_add, sums);
+            // release the stage, then fold the group sums into the running sums with the groups' scales
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
             if (++s == stages) { s = 0; phase ^= 1u; }
-            fold_group<MT>(acc, accg, sc);
+            fold_item<MT, SUB>(acc, sums);
         }
     }
 
@@ -259,7 +261,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 
 // Resident CTAs per SM by token tile: registers and ring size are set so that three CTAs of the
 // narrowest tile fit, which lets the next kernel's first CTAs start (and prefetch weights) early.
-__host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT <= 2 ? 3 : 1; }
+__host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return 3; }
 
 // Picks the cluster size S in {1, 2, 4, 8} with the smallest estimated time among those whose
 // panels * S CTAs are all resident at once (falling back to all S if none is).  The estimate is
@@ -267,12 +269,13 @@ __host__ __device__ constexpr int splitk_ctas_per_sm(int MT) { return MT <= 2 ? 
 // serial rate, plus the cluster reduction when S > 1 (hundredths of a microsecond; only ratios
 // matter).  Shared memory is then padded so that exactly ceil(CTAs / SMs) CTAs fit on an SM: the
 // cluster scheduler otherwise packs three CTAs onto some SMs and leaves others empty.
-SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
+SplitKPlan plan_splitk(int m_rows, int N, int K, int group_size, int sm_count)
 {
     SplitKPlan pl{};
     const int MT = streamk_m_tile(m_rows);
     const int G = K / kGroup, panels = N / kPanel;
-    const int stage = streamk_stage_bytes(MT);
+    pl.sub = kGroup / group_size;
+    const int stage = streamk_stage_bytes(MT, pl.sub);
     const int cps_max = splitk_ctas_per_sm(MT);
     int best_S = 1;
     long long best_t = -1;
@@ -306,11 +309,11 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int sm_count)
     return pl;
 }
 
-template <int MT>
+template <int MT, int SUB>
 static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, const SplitKPlan &plan, cudaStream_t s)
 {
     static int configured_smem[64] = {};
-    const int cfg_st = ensure_dynamic_smem((const void *)splitk_kernel<MT>, configured_smem, plan.smem_bytes);
+    const int cfg_st = ensure_dynamic_smem((const void *)splitk_kernel<MT, SUB>, configured_smem, plan.smem_bytes);
     if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
@@ -326,7 +329,7 @@ static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, co
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return record_cuda_error(cudaLaunchKernelEx(&cfg, splitk_kernel<MT>, args, x_map));
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, splitk_kernel<MT, SUB>, args, x_map));
 }
 
 int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
@@ -343,14 +346,19 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
+    args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;
     int st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
                                 (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.m_tile, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st) return st;
-    switch (plan.m_tile) {
-    case 8: return launch_splitk_mt<1>(args, x_map, plan, s);
-    case 16: return launch_splitk_mt<2>(args, x_map, plan, s);
+    switch (plan.m_tile * 10 + plan.sub) {
+    case 81: return launch_splitk_mt<1, 1>(args, x_map, plan, s);
+    case 82: return launch_splitk_mt<1, 2>(args, x_map, plan, s);
+    case 84: return launch_splitk_mt<1, 4>(args, x_map, plan, s);
+    case 161: return launch_splitk_mt<2, 1>(args, x_map, plan, s);
+    case 162: return launch_splitk_mt<2, 2>(args, x_map, plan, s);
+    case 164: return launch_splitk_mt<2, 4>(args, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }

@@ -28,9 +28,9 @@ constexpr int kRingOffset = 1024;   // barriers live below the ring; the ring is
 // A ring stage: [x: two K64 tiles of MT*8 token rows x 128 B, 128-byte swizzled by the tensor-map load]
 //               [8192 B packed weights][256 B scales][64 B zeros], rounded up to 1024 B.
 __host__ __device__ constexpr int streamk_x_bytes(int MT) { return MT * 2048; }
-__host__ __device__ constexpr int streamk_stage_bytes(int MT)
+__host__ __device__ constexpr int streamk_stage_bytes(int MT, int SUB = 1)
 {
-    return (streamk_x_bytes(MT) + kItemWBytes + kItemSBytes + kItemZBytes + 1023) & ~1023;
+    return (streamk_x_bytes(MT) + kItemWBytes + SUB * (kItemSBytes + kItemZBytes) + 1023) & ~1023;
 }
 
 // Stream-K index arithmetic (shared by the kernel, the planner and the host-side introspection
@@ -44,32 +44,46 @@ __host__ __device__ inline int sk_owner(long long T, int C, long long t) { retur
 // chunks of the swizzled x tile, so the 128-bit fragment loads are bank-conflict free.
 __host__ __device__ constexpr int token_row_of_slot(int n) { return ((n & 1) << 2) | (n & 2) | ((n >> 2) & 1); }
 
-// The arithmetic of one (panel, group) item for one consumer warp, shared by the mma.sync kernels: the lane reads
-// its two 16-byte chunks of packed weights, the scale pair and the zero byte of its columns from ring stage `st`,
-// turns nibbles into exact fp16 integers q - z and multiplies them with the stage's x tiles; `accg` receives the
-// unscaled fp32 group sums, `sc` the two fp16 scales.  The stage may be released once this returns.
-template <int MT>
+// The arithmetic of one (panel, 128-row) item for one consumer warp, shared by the mma.sync kernels.  The lane reads
+// its two 16-byte chunks of packed weights from ring stage `st`; for each of the item's SUB quantisation groups
+// (128 / group_size: the whole item, a K64 block, or half of one) it reads the scale pair and the zero byte of its
+// columns, turns nibbles into exact fp16 integers q - z (z_add = 1 when the stored zero points are one too small),
+// multiplies them with the stage's x tiles and folds the fp32 group sums into `acc` with the group's scales.
+// The stage may be released once `consume_item` has returned; `fold_item` needs registers only.
+template <int MT, int SUB>
+struct ItemSums {
+    float g[SUB][MT][4];
+    uint32_t sc[SUB];
+};
+template <int MT, int SUB>
 __device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32_t s_off, uint32_t z_off,
-                                             uint32_t x_off0, uint32_t x_off1, float (&accg)[MT][4], uint32_t &sc)
+                                             uint32_t x_off0, uint32_t x_off1, uint32_t z_add, ItemSums<MT, SUB> &out)
 {
     constexpr int kXTile = MT * 1024;
     constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
     const uint4 wq0 = lds128(st + w_off);
     const uint4 wq1 = lds128(st + kBlockWBytes + w_off);
-    sc = lds32(st + s_off);
-    const uint32_t zb = lds8(st + z_off);
-    const uint32_t zA = zb & 15u, zB = zb >> 4;
-    const uint32_t zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
-    const uint32_t zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+    uint32_t zloA = 0, zhiA = 0, zloB = 0, zhiB = 0;
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int sub = 0; sub < SUB; ++sub)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) accg[mt][i] = 0.f;
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) out.g[sub][mt][i] = 0.f;
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk) {
         const uint4 wq = blk ? wq1 : wq0;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
+            const int q4 = blk * 2 + j;              // quarter of the item: 32 rows
+            const int sub = q4 * SUB / 4;
+            if (q4 * SUB % 4 == 0) {                 // first quarter of a group
+                out.sc[sub] = lds32(st + s_off + sub * kItemSBytes);
+                const uint32_t zb = lds8(st + z_off + sub * kItemZBytes);
+                const uint32_t zA = (zb & 15u) + z_add, zB = (zb >> 4) + z_add;   // up to 16: still exact below
+                zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
+                zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+            }
             uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
             const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
             const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
@@ -84,23 +98,26 @@ __device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) {
                 const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
-                mma_m16n8k16(accg[mt], a0, a1, a2, a3, xb.x, xb.y);
-                mma_m16n8k16(accg[mt], c0, c1, c2, c3, xb.z, xb.w);
+                mma_m16n8k16(out.g[sub][mt], a0, a1, a2, a3, xb.x, xb.y);
+                mma_m16n8k16(out.g[sub][mt], c0, c1, c2, c3, xb.z, xb.w);
             }
         }
     }
 }
-// folds a group's sums into the running sums with the group's scales
-template <int MT>
-__device__ __forceinline__ void fold_group(float (&acc)[MT][4], const float (&accg)[MT][4], uint32_t sc)
+// folds the item's group sums into the running sums with each group's scales
+template <int MT, int SUB>
+__device__ __forceinline__ void fold_item(float (&acc)[MT][4], const ItemSums<MT, SUB> &it)
 {
-    const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&sc));
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        acc[mt][0] = fmaf(sf.x, accg[mt][0], acc[mt][0]);
-        acc[mt][1] = fmaf(sf.x, accg[mt][1], acc[mt][1]);
-        acc[mt][2] = fmaf(sf.y, accg[mt][2], acc[mt][2]);
-        acc[mt][3] = fmaf(sf.y, accg[mt][3], acc[mt][3]);
+    for (int sub = 0; sub < SUB; ++sub) {
+        const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&it.sc[sub]));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            acc[mt][0] = fmaf(sf.x, it.g[sub][mt][0], acc[mt][0]);
+            acc[mt][1] = fmaf(sf.x, it.g[sub][mt][1], acc[mt][1]);
+            acc[mt][2] = fmaf(sf.y, it.g[sub][mt][2], acc[mt][2]);
+            acc[mt][3] = fmaf(sf.y, it.g[sub][mt][3], acc[mt][3]);
+        }
     }
 }
 
@@ -114,6 +131,7 @@ struct StreamKArgs {
     int M, N, K, G;
     int items;              // T = panels * G
     int stages;
+    const TiledTrailer *trailer;   // behind the tiled zero points: says whether the stored zero points are one too small
 };
 
 template <int MT>
@@ -184,6 +202,7 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     }
 
     // -------------------------------------------------------------------- consumer warps
+    const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // weights-side data: no need to wait
     pdl_wait();
     const int g = lane >> 2, t4 = lane & 3;
     const int r = token_row_of_slot(g);
@@ -210,14 +229,13 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
         const uint32_t st = ring + s * kStage;
         if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
 
-        float accg[MT][4];
-        uint32_t sc;
-        consume_item<MT>(st, w_off, s_off, z_off, x_off0, x_off1, accg, sc);
+        ItemSums<MT, 1> sums;
+        consume_item<MT, 1>(st, w_off, s_off, z_off, x_off0, x_off1, z_add, sums);
         // release the stage, then fold the group sum into the running sum with the group's scale
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty + 8 * s);
         if (++s == stages) { s = 0; phase ^= 1u; }
-        fold_group<MT>(acc, accg, sc);
+        fold_item<MT, 1>(acc, sums);
 
         const bool seg_end = (grp == a.G - 1) || (t == t1 - 1);
         if (seg_end) {
@@ -362,6 +380,7 @@ int launch_streamk(const __half *x, const void *qweight, const void *qzeros, con
     args.G = K / kGroup;
     args.items = plan.items;
     args.stages = plan.stages;
+    args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;
     int st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,

@@ -146,6 +146,7 @@ struct UmmaArgs {
     int S;                  // CTAs that share one output tile along K (cluster size)
     int tile0;              // first output tile of this launch (a matmul may take a main and a tail launch)
     int stages;             // shared-memory ring depth
+    const TiledTrailer *trailer;   // behind the tiled zero points
 };
 
 // K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
@@ -165,7 +166,7 @@ __host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP)
     return c;
 }
 
-template <int TOK, int NA, int NP, int SETS>
+template <int TOK, int NA, int NP, int SETS, int SUB>
 __global__ void __launch_bounds__(umma_threads(NP, SETS), (NP > 1 || TOK > 128) ? 1 : TOK <= 32 ? 3 : 2)
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
@@ -310,22 +311,31 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // The column's scale and zero point of a group come straight from global memory (2 bytes and a nibble per
         // lane: 64 + 16 bytes per warp), fetched one group ahead into registers, which spares the producer thread two
         // copies per group.  In the tiled layout the pair (column, column + 8) is adjacent.
-        const uint8_t *s_gl = a.scales + ((size_t)p * a.G + g0) * kItemSBytes + (16 * u + 2 * g + h) * 2;
-        const uint8_t *z_gl = a.qzeros + ((size_t)p * a.G + g0) * kItemZBytes + 8 * u + g;
-        auto load_sz = [&](int gg, uint32_t &sc, uint32_t &zb) {
+        // A 128-row item holds SUB quantisation groups (128 / group_size), each with its own scales and zeros.
+        const uint8_t *s_gl = a.scales + ((size_t)p * a.G + g0) * (SUB * kItemSBytes) + (16 * u + 2 * g + h) * 2;
+        const uint8_t *z_gl = a.qzeros + ((size_t)p * a.G + g0) * (SUB * kItemZBytes) + 8 * u + g;
+        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // stored zero points one too small
+        auto load_sz = [&](int gg, uint32_t (&sc)[SUB], uint32_t (&zb)[SUB]) {
             // through L2 only: this kernel may start while its predecessor still runs, and the buffers may have been
             // rewritten since an earlier kernel left lines of them in this SM's L1
-            sc = __ldcg(reinterpret_cast<const unsigned short *>(s_gl + (size_t)gg * kItemSBytes));
-            zb = __ldcg(z_gl + (size_t)gg * kItemZBytes);
+#pragma unroll
+            for (int sub = 0; sub < SUB; ++sub) {
+                sc[sub] = __ldcg(reinterpret_cast<const unsigned short *>(s_gl + ((size_t)gg * SUB + sub) * kItemSBytes));
+                zb[sub] = __ldcg(z_gl + ((size_t)gg * SUB + sub) * kItemZBytes);
+            }
         };
-        uint32_t sc_next = 0, zb_next = 0;
+        uint32_t sc_next[SUB], zb_next[SUB];
+#pragma unroll
+        for (int sub = 0; sub < SUB; ++sub) sc_next[sub] = zb_next[sub] = 0;
         if (2 * set < NB) load_sz(set, sc_next, zb_next);
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
         // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1; block b lives in ring refill b / BPS
         int b = 2 * set;
         int s = (b / BPS) % NS, sa = b % NA;
         uint32_t ph = (uint32_t)((b / BPS) / NS) & 1u;
-        uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
+        uint32_t s2[SUB], zlo[SUB], zhi[SUB];
+#pragma unroll
+        for (int sub = 0; sub < SUB; ++sub) s2[sub] = 0, zlo[sub] = MAGIC_LO, zhi[sub] = MAGIC_HI;
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
@@ -338,16 +348,31 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 if (!ok) break;
             }
             if ((b & 1) == 0) {
-                s2 = sc_next * 0x00010001u;
-                const uint32_t z = h ? (zb_next >> 4) : (zb_next & 15u);
-                zlo = (z * 0x00010001u) | MAGIC_LO;
-                zhi = (z * 0x00100010u) | MAGIC_HI;
-                if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next group
+#pragma unroll
+                for (int sub = 0; sub < SUB; ++sub) {
+                    s2[sub] = sc_next[sub] * 0x00010001u;
+                    const uint32_t z = (h ? (zb_next[sub] >> 4) : (zb_next[sub] & 15u)) + z_add;   // up to 16: still exact
+                    zlo[sub] = (z * 0x00010001u) | MAGIC_LO;
+                    zhi[sub] = (z * 0x00100010u) | MAGIC_HI;
+                }
+                if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next item
             }
             const uint32_t wb = st + (b % BPS) * kUmmaWBlockBytes;
             uint2 wv[4];
 #pragma unroll
             for (int t4 = 0; t4 < 4; ++t4) wv[t4] = lds64(wb + w_rd[t4]);
+            // constants of the two 32-row halves of this block: the item's group (SUB = 1), the block's (2) or the
+            // half's own (4); picked with selects so that the arrays stay in registers
+            uint32_t s2_b[2], zlo_b[2], zhi_b[2];
+            const bool odd = (b & 1) != 0;
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+                constexpr int kLast = SUB - 1;
+                const int lo = SUB == 4 ? jj : 0, hi = SUB == 4 ? 2 + jj : kLast;   // even / odd block of the item
+                s2_b[jj] = odd ? s2[hi] : s2[lo];
+                zlo_b[jj] = odd ? zlo[hi] : zlo[lo];
+                zhi_b[jj] = odd ? zhi[hi] : zhi[lo];
+            }
             uint32_t r[32];
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -355,11 +380,11 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 for (int t4 = 0; t4 < 4; ++t4) {
                     uint32_t w = jj ? wv[t4].y : wv[t4].x;       // rows 32 jj + 8 t4 + (0..7), TMEM columns 16 jj + 4 t4 + (0..3)
                     uint32_t *o = r + 16 * jj + 4 * t4;
-                    o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
-                    o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                    o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo_b[jj]), s2_b[jj]);
+                    o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi_b[jj]), s2_b[jj]);
                     w >>= 8;
-                    o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo), s2);
-                    o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi), s2);
+                    o[2] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo_b[jj]), s2_b[jj]);
+                    o[3] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi_b[jj]), s2_b[jj]);
                 }
             if (b >= NA) {     // the stage's previous block b - NA must have been multiplied
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((b - NA) & (kUmmaDoneRing - 1)), (uint32_t)(((b - NA) / kUmmaDoneRing) & 1)));
@@ -567,11 +592,11 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     return pl;
 }
 
-template <int TOK, int NP, int SETS>
-static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
+template <int TOK, int NP, int SETS, int SUB>
+static int launch_umma_sub(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
                            const UmmaPlan &plan, int ctas, cudaStream_t s)
 {
-    auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS>;
+    auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS, SUB>;
     static int configured_smem[64] = {};
     const int cfg_st = ensure_dynamic_smem((const void *)kernel, configured_smem, plan.smem_bytes);
     if (cfg_st) return cfg_st;
@@ -592,8 +617,20 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
     return record_cuda_error(cudaLaunchKernelEx(&cfg, kernel, args, w_map, x_map));
 }
 
+template <int TOK, int NP, int SETS>
+static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
+                           const UmmaPlan &plan, int ctas, int sub, cudaStream_t s)
+{
+    switch (sub) {
+    case 1: return launch_umma_sub<TOK, NP, SETS, 1>(args, w_map, x_map, plan, ctas, s);
+    case 2: return launch_umma_sub<TOK, NP, SETS, 2>(args, w_map, x_map, plan, ctas, s);
+    case 4: return launch_umma_sub<TOK, NP, SETS, 4>(args, w_map, x_map, plan, ctas, s);
+    default: return GPTQ_ERR_UNSUPPORTED;
+    }
+}
+
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
-                int K, const UmmaPlan &plan, cudaStream_t s)
+                int K, int group_size, const UmmaPlan &plan, cudaStream_t s)
 {
     UmmaArgs args;
     args.scales = (const uint8_t *)scales;
@@ -605,6 +642,8 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
+    args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, group_size));
+    const int sub = kGroup / group_size;
     if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;
     // packed weights as rows of 64 bytes (16 words); a box is one ring slot's K64 blocks of a panel (64 rows each)
     CUtensorMap w_map, x_map;
@@ -619,10 +658,10 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     if (st) return st;
     auto launch = [&](const UmmaArgs &la, int ctas) {
         switch (plan.tok) {
-        case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, s);
-        case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, s);
-        case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, s);
-        case 256: return launch_umma_tok<256, 1, 2>(la, w_map, x_map, plan, ctas, s);
+        case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
+        case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
+        case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
+        case 256: return launch_umma_tok<256, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
         default: return (int)GPTQ_ERR_UNSUPPORTED;
         }
     };

@@ -195,6 +195,7 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         int s = set % NS, sa = b % NA;
         uint32_t ph = (uint32_t)(set / NS) & 1u;
         uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
+        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // stored zero points one too small
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
@@ -206,7 +207,7 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
                 ok = ok && __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph));   // warp-uniform
                 if (!ok) break;
                 s2 = sc_next * 0x00010001u;
-                const uint32_t z = h ? (zb_next >> 4) : (zb_next & 15u);
+                const uint32_t z = (h ? (zb_next >> 4) : (zb_next & 15u)) + z_add;
                 zlo = (z * 0x00010001u) | MAGIC_LO;
                 zhi = (z * 0x00100010u) | MAGIC_HI;
                 if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next group
@@ -339,6 +340,7 @@ int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const
     args.G = K / kGroup;
     args.S = 1;
     args.stages = plan.stages;
+    args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup));
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;
     int st = make_tensor_map_2d(&w_map, CU_TENSOR_MAP_DATA_TYPE_UINT32, qweight, 16, w_rows, 64, 16, 128,

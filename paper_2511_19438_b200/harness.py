@@ -42,7 +42,9 @@ def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda
     qz_t = torch.empty(B.gptq_repack_bytes(1, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     sc_t = torch.empty(B.gptq_repack_bytes(2, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     perm = torch.empty(L.K, dtype=torch.int32, device=device) if L.act_order else None
-    B.check(B.gptq_repack(qw, qz, sc, gi, qw_t, qz_t, sc_t, perm, L.N, L.K, L.group_size, L.act_order), "gptq_repack")
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0
+    B.check(B.gptq_repack_format(qw, qz, sc, gi, qw_t, qz_t, sc_t, perm, L.N, L.K, L.group_size, L.act_order, fmt),
+            "gptq_repack_format")
     torch.cuda.current_stream().synchronize()
     canonical = (qw, qz, sc, gi) if keep_canonical else None
     return DeviceLinear(L.K, L.N, L.group_size, L.act_order, qw_t, qz_t, sc_t, perm, canonical)

@@ -92,6 +92,7 @@ class QuantLinear:
     scales: np.ndarray           # float16[G, N]
     g_idx: np.ndarray | None     # int32[K] or None
     seed: int
+    zeros_minus_one: bool = False   # the stored zero-point nibble is z - 1 (older checkpoints)
 
     @property
     def act_order(self) -> bool:
@@ -114,9 +115,11 @@ def make_g_idx(K: int, group_size: int, seed: int) -> np.ndarray:
 
 
 def make_linear(K: int, N: int, seed: int, group_size: int = GROUP_SIZE,
-                act_order: bool = False) -> QuantLinear:
+                act_order: bool = False, zeros_minus_one: bool = False) -> QuantLinear:
     """Random GPTQ layer.  Packed words are drawn directly as uniform 32-bit
-    integers, which makes every nibble uniform on 0..15 and independent."""
+    integers, which makes every nibble uniform on 0..15 and independent.
+    ``zeros_minus_one`` only labels the layer: the same stored nibbles are then
+    to be read as zero point minus one."""
     assert K % 8 == 0 and N % 8 == 0 and K % group_size == 0
     G = K // group_size
     r = _rng(seed)
@@ -124,7 +127,7 @@ def make_linear(K: int, N: int, seed: int, group_size: int = GROUP_SIZE,
     qzeros = r.integers(0, 1 << 32, size=(G, N // 8), dtype=np.uint32).view(np.int32)
     scales = make_scales(G, N, seed ^ 0x5CA1E5)
     g_idx = make_g_idx(K, group_size, seed ^ 0x61D7) if act_order else None
-    return QuantLinear(K, N, group_size, qweight, qzeros, scales, g_idx, seed)
+    return QuantLinear(K, N, group_size, qweight, qzeros, scales, g_idx, seed, zeros_minus_one)
 
 
 def make_linear_from_values(q: np.ndarray, z: np.ndarray, scales: np.ndarray,

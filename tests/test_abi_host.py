@@ -56,7 +56,8 @@ def test_gemm_validation_order_without_gpu():
     assert call(group_size=0) == B.GPTQ_ERR_SHAPE
     assert call(x=A16 + 8) == B.GPTQ_ERR_ALIGN
     assert call(qw=A16 + 4) == B.GPTQ_ERR_ALIGN
-    assert call(group_size=64) == B.GPTQ_ERR_UNSUPPORTED
+    assert call(group_size=16) == B.GPTQ_ERR_UNSUPPORTED   # 128, 64 and 32 have a tiled layout
+    assert call(group_size=256) == B.GPTQ_ERR_UNSUPPORTED
     assert call(N=4096 + 64) == B.GPTQ_ERR_UNSUPPORTED
 
 
@@ -68,7 +69,10 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_dequant_f32(A16, A16, A16, None, A16, 64, 128, 128, 0, 1, stream=0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack(A16, A16, A16, None, A16 + 16, None, A16, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_repack(A16, A16, A16, None, A16, A16 + 16, A16 + 32, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_LAYOUT
-    assert B.gptq_repack(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 16, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack_format(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, 2, stream=0) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_repack_bytes(1, 256, 512, 32, 0) == (512 // 32) * 256 // 2 + 16    # zero points + format trailer
+    assert B.gptq_plan_noalloc(4, 128, 512, 64, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack(A16, A16, A16, A16, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_gemm_host(None, A16, A16, A16, None, A16, A16, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
 
@@ -89,11 +93,11 @@ def test_host_batch_validates_every_problem_before_running():
     assert B._lib.gptq_gemm_host_batch(arr, 0, 0, None) == B.GPTQ_OK      # an empty step is fine
 
 
-def test_repack_bytes_equal_canonical_sizes():
+def test_repack_bytes_equal_canonical_sizes_plus_trailer():
     for (K, N) in list(wl.SHAPES_7B.values()) + list(wl.SHAPES_13B.values()):
         G = K // 128
         assert B.gptq_repack_bytes(0, N, K, 128, 0) == K * N // 2
-        assert B.gptq_repack_bytes(1, N, K, 128, 0) == G * N // 2
+        assert B.gptq_repack_bytes(1, N, K, 128, 0) == G * N // 2 + 16     # + the 16-byte format trailer
         assert B.gptq_repack_bytes(2, N, K, 128, 0) == G * N * 2
         assert B.gptq_repack_bytes(3, N, K, 128, 0) == 0
         assert B.gptq_repack_bytes(3, N, K, 128, 1) == 4 * K
@@ -220,18 +224,21 @@ def test_plan_act_order_adds_gathered_x():
 
 def test_plan_rejects_bad_arguments():
     assert B.gptq_plan(1, 4096, 4096, 128, 0, 0)[0] == B.GPTQ_ERR_SHAPE
-    assert B.gptq_plan(1, 4096, 4096, 32, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_plan(1, 4096, 4096, 16, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_plan(1, 4096, 4096, 32, 0, 148)[0] == B.GPTQ_OK
     assert B.gptq_plan_cta_range(10, 11, 0)[0] == B.GPTQ_ERR_SHAPE
     assert B.gptq_plan_panel_owners(10, 5, 3, 0)[0] == B.GPTQ_ERR_SHAPE
 
 
 def test_plan_names_the_kernel():
     """The planner names the kernel instantiation a profiler would print; bench.py attributes time by it."""
-    for M, want in ((1, "splitk_kernel<1>"), (8, "splitk_kernel<1>"), (16, "splitk_kernel<2>"),
-                    (17, "umma_kernel<32,3,1,2>"), (64, "umma_kernel<64,4,1,2>"), (128, "umma_kernel<128,4,1,2>"),
-                    (2048, "umma_kernel<256,4,1,2>")):
+    for M, want in ((1, "splitk_kernel<1,1>"), (8, "splitk_kernel<1,1>"), (16, "splitk_kernel<2,1>"),
+                    (17, "umma_kernel<32,3,1,2,1>"), (64, "umma_kernel<64,4,1,2,1>"), (128, "umma_kernel<128,4,1,2,1>"),
+                    (2048, "umma_kernel<256,4,1,2,1>")):
         st, pl = B.gptq_plan(M, 4096, 4096, 128, 0, 148)
         assert st == B.GPTQ_OK and B.plan_kernel_name(pl) == want
+    assert B.plan_kernel_name(B.gptq_plan(4, 4096, 4096, 32, 0, 148)[1]) == "splitk_kernel<1,4>"     # four groups per item
+    assert B.plan_kernel_name(B.gptq_plan(512, 4096, 4096, 64, 0, 148)[1]) == "umma_kernel<256,4,1,2,2>"
     for M, want in ((1, "streamk_kernel<1>"), (16, "streamk_kernel<2>"), (32, "streamk_kernel<4>"), (100, "streamk_kernel<8>")):
         st, pl = B.gptq_plan_noalloc(M, 1024, 1024, 128, 0, 148)
         assert st == B.GPTQ_OK and B.plan_kernel_name(pl) == want

@@ -417,6 +417,75 @@ def test_few_groups_tolerance_limit(ws):
     assert np.sqrt(np.mean(err ** 2)) < 2.5e-3 * math.sqrt(K / 4096) + 2.0 ** -11 * np.sqrt(np.mean(y64 ** 2))
 
 
+# ------------------------------------------------------------------------------- format variants
+VARIANTS = [(32, False, False), (64, False, False), (32, True, False), (64, True, True), (128, False, True),
+            (128, True, True), (32, False, True)]
+
+
+@pytest.mark.parametrize("gs,act,zm1", VARIANTS)
+def test_variant_dequant_bit_exact(gs, act, zm1):
+    """Group sizes 32 and 64 and zero points stored minus one: canonical and tiled dequantisation give the oracle's
+    bits (the tiled buffers carry the format in their trailer)."""
+    K, N = 512, 256
+    L = wl.make_linear(K, N, seed=wl.seed_for("variant-dq", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    want = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    gi = H.to_device(L.g_idx) if act else None
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if zm1 else 0
+    B.check(B.gptq_dequant_f32_format(H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales), gi, w,
+                                      N, K, gs, act, 0, fmt), "dequant canonical")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    D = H.upload_and_repack(L)
+    w.zero_()
+    B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert B.gptq_dequant_f32_format(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 2) == B.GPTQ_ERR_LAYOUT
+
+
+@pytest.mark.parametrize("gs,act,zm1", VARIANTS)
+@pytest.mark.parametrize("M", [1, 8, 13, 40, 200, 600])
+def test_variant_gemm(gs, act, zm1, M, ws):
+    """The matmul on every kernel family (M = 1 .. 16 mma.sync, above tcgen05 with 32- to 256-token tiles)."""
+    K, N = 1024, 384
+    L = wl.make_linear(K, N, seed=wl.seed_for("variant", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    x = wl.make_x(M, K, wl.seed_for("variant-x", M))
+    y, _ = run_gemm(L, x, ws)
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1), K)
+
+
+def test_variant_zero_point_sixteen_is_exact(ws):
+    """Every stored zero point 15 read as 16, scales 1, small-integer x: q - 16 is a negative integer and the product is
+    exact in fp16 wherever |y| <= 2048 - a wrong wrap-around of the nibble would show at once."""
+    K, N = 512, 128
+    r = np.random.default_rng(5)
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    L = wl.make_linear_from_values(q, np.full((K // 32, N), 15, np.uint8), np.ones((K // 32, N), np.float16), 32)
+    L.zeros_minus_one = True
+    for M in (2, 50):
+        x = r.integers(-2, 3, (M, K)).astype(np.float16)
+        y, _ = run_gemm(L, x, ws)
+        want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, None, 32, zeros_minus_one=True)
+        small = np.abs(want) <= 2048
+        assert np.array_equal(y.astype(np.float64)[small], want[small])
+        assert np.allclose(want, x.astype(np.float64) @ (q.astype(np.float64) - 16.0))
+
+
+def test_variants_unsupported_entry_points():
+    """gptq_gemm_noalloc is built for group size 128 only; other group sizes (and sizes the format has no tiling for)
+    are refused before any launch."""
+    K, N = 512, 128
+    L = wl.make_linear(K, N, seed=11, group_size=64)
+    D = H.upload_and_repack(L)
+    x = H.to_device(wl.make_x(4, K, 1))
+    y = torch.zeros((4, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 4, N, K, 64, 0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 4, N, K, 16, 0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack_format(D.qweight_t, D.qzeros_t, D.scales_t, None, D.qweight_t, D.qzeros_t, D.scales_t, None,
+                                N, K, 64, 0, 4) == B.GPTQ_ERR_LAYOUT
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(y) == 0
+
+
 def test_bounded_wait_reports_timeout():
     """A wait that nothing satisfies gives up after its limit, the kernel returns normally, and the status word
     turns into GPTQ_ERR_TIMEOUT exactly once; the context stays usable."""
