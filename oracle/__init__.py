@@ -25,7 +25,7 @@ def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".{os.getpid()}.tmp"
         subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11",
-                               "-o", tmp, _SRC])
+                               "-o", tmp, _SRC, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -38,7 +38,7 @@ def _load():
         lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
         lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
-                     "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1"):
+                     "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -146,4 +146,14 @@ def gemm_f64_at(x, qweight, qzeros, scales, g_idx, group_size: int, rows, cols) 
     _load().oracle_gemm_f64_at(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M),
                                ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size),
                                _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
+    return out
+
+
+def silu_mul_f64(y: np.ndarray) -> np.ndarray:
+    """out[M, I] = silu(y[:, :I]) * y[:, I:] in fp64 for the [gate | up] columns of a gate_up projection."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    M, N = y.shape
+    assert N % 2 == 0
+    out = np.empty((M, N // 2), dtype=np.float64)
+    _load().oracle_silu_mul_f64(_p(y), ctypes.c_int(M), ctypes.c_int(N // 2), _p(out))
     return out

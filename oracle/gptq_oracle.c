@@ -28,6 +28,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <string.h>
+#include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -192,4 +193,18 @@ void oracle_gemm_f64_v1(const uint16_t *x, const int32_t *qweight, const int32_t
             y_out[(size_t)m * N + n] = acc;
         }
     }
+}
+
+/* ---- the gated-MLP neighbour of the gate_up projection ---------------------------------------
+ * In the Llama-class models the paper serves (Section 4.1), the columns of the fused gate_up projection are
+ * [gate | up] and the next operation is out[m][i] = silu(gate[m][i]) * up[m][i], silu(t) = t / (1 + exp(-t)).
+ * The paper's kernels stop at the matmul; the library can fuse this step into the matmul's epilogue, and this
+ * is its definition: y is the fp64 matmul result [M, 2 I], out is [M, I]. */
+void oracle_silu_mul_f64(const double *y, int M, int I, double *out)
+{
+    for (int m = 0; m < M; m++)
+        for (int i = 0; i < I; i++) {
+            double g = y[(size_t)m * 2 * I + i], u = y[(size_t)m * 2 * I + I + i];
+            out[(size_t)m * I + i] = g / (1.0 + exp(-g)) * u;
+        }
 }

@@ -321,3 +321,28 @@ def test_v1_gemm_is_plain_gemm_minus_scaled_group_sums_of_x():
     # and it is the matmul of its own dequantised weights
     w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=True).astype(np.float64)
     assert np.allclose(y_v1, x.astype(np.float64) @ w, rtol=1e-13, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- silu(gate) * up
+def test_silu_mul_special_values():
+    y = np.array([[0.0, 1.0, -1.0, 40.0, -40.0, 2.0,      # gate
+                   3.0, 2.0, 2.0, 0.5, 7.0, -1.5]])       # up
+    out = oracle.silu_mul_f64(y)[0]
+    assert out[0] == 0.0                                   # silu(0) = 0
+    assert abs(out[1] - 2 * 0.7310585786300049) < 1e-15    # silu(1) = 1 / (1 + e^-1)
+    assert abs(out[2] - 2 * -0.2689414213699951) < 1e-15   # silu(-1) = -1 / (1 + e)
+    assert abs(out[3] - 20.0) < 1e-12                      # silu(t) -> t for large t
+    assert abs(out[4]) < 1e-14                             # silu(t) -> 0 for very negative t
+    assert abs(out[5] - (-1.5) * 2 / (1 + math.exp(-2))) < 1e-15
+
+
+def test_silu_mul_against_the_tanh_form_and_its_symmetry():
+    r = np.random.default_rng(3)
+    y = r.normal(0, 4, (5, 64))
+    out = oracle.silu_mul_f64(y)
+    g, u = y[:, :32], y[:, 32:]
+    assert np.allclose(out, g * 0.5 * (1 + np.tanh(g / 2)) * u, rtol=1e-13, atol=1e-15)   # sigmoid(t) = (1 + tanh(t/2)) / 2
+    neg = oracle.silu_mul_f64(np.concatenate([-g, u], axis=1))
+    assert np.allclose(out - neg, g * u, rtol=1e-13, atol=1e-13)                           # silu(t) - silu(-t) = t
+    # gate columns first, up columns second: swapping the halves is a different function
+    assert not np.allclose(out, oracle.silu_mul_f64(np.concatenate([u, g], axis=1)))
