@@ -46,7 +46,7 @@ typedef enum {
     GPTQ_ERR_SHAPE = -2,       /* M<1, K%8, N%8, K%group_size, group_size<=0 ... */
     GPTQ_ERR_ALIGN = -3,       /* a pointer is not 16-byte aligned */
     GPTQ_ERR_UNSUPPORTED = -4, /* valid GPTQ shape outside the tiled fast path */
-    GPTQ_ERR_LAYOUT = -5,      /* bad `which`/flag argument */
+    GPTQ_ERR_LAYOUT = -5,      /* bad `which`/flag argument; from gptq_check_status: a layer's tiling does not fit the call */
     GPTQ_ERR_GIDX = -6,        /* g_idx entry out of range, or groups of unequal size (gptq_repack) */
     GPTQ_ERR_WORKSPACE = -7,   /* workspace missing or too small for this call */
     GPTQ_ERR_CUDA = -8,        /* a CUDA runtime call failed (see gptq_last_cuda_error) */
@@ -84,8 +84,14 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
  * gptq_repack_format records the flag in a 16-byte trailer behind the tiled zero points (counted in
  * gptq_repack_bytes(1, ...)), so gptq_gemm and gptq_dequant_f32(repacked = 1) need no format argument. */
 #define GPTQ_FORMAT_ZEROS_MINUS_ONE 1
-/* gptq_dequant_f32 with a format for canonical inputs (repacked = 0); with repacked = 1 the trailer decides and
- * `format` must be 0 or equal to what the layer was repacked with. */
+/* A third flag concerns the tiled layout only, not the checkpoint: GPTQ_FORMAT_GATE_UP tiles a layer whose N columns
+ * are [gate | up] (N / 2 each, the merged first projection of a Llama MLP block - the models of Section 4.1) so that
+ * each 128-column panel holds 64 gate columns and the 64 matching up columns; gptq_gemm_silu_mul needs that order and
+ * gptq_gemm refuses it.  gptq_dequant_f32(repacked = 1) undoes it: its output is in checkpoint column order. */
+#define GPTQ_FORMAT_GATE_UP 2
+/* gptq_dequant_f32 with a format for canonical inputs (repacked = 0; GPTQ_FORMAT_GATE_UP is refused there with
+ * GPTQ_ERR_LAYOUT); with repacked = 1 the trailer decides and `format` must be 0 or equal to what the layer was
+ * repacked with.  Unknown flag bits: GPTQ_ERR_LAYOUT. */
 int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
                             float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
                             void *stream);
@@ -144,6 +150,18 @@ int gptq_set_workspace(void *ptr, size_t bytes);
 int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales,
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
+
+/* (No counterpart in the paper: an epilogue fused into the product of Sections 1 and 3.)
+ * out fp16[M, N / 2] = silu(y[:, :N/2]) * y[:, N/2:], silu(g) = g / (1 + exp(-g)), for y = x . dequant(W) of a layer
+ * repacked with GPTQ_FORMAT_GATE_UP: the activation of a Llama MLP block applied before the product leaves the chip,
+ * so y itself is never written.  Other arguments as for gptq_gemm; N counts both halves.  Up to 16 token rows the
+ * two factors are the fp32 sums; above that each is rounded to fp16 first unless the K range was split across CTAs;
+ * silu and the product are evaluated in fp32 (fast exponential, relative error ~1e-6), then rounded to fp16 once.
+ * A layer repacked without the flag (or a flagged layer given to gptq_gemm / gptq_gemm_noalloc) stores nothing and
+ * makes the next gptq_check_status return GPTQ_ERR_LAYOUT.  The CTA-pair switch below does not apply to it. */
+int gptq_gemm_silu_mul(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                       const int32_t *g_idx, void *out, int M, int N, int K, int group_size, int act_order,
+                       void *stream);
 
 /* Process-wide switch: with enable != 0, gptq_gemm runs problems with M >= 256 and an even number
  * of 128-column panels on CTA pairs (tcgen05.mma.cta_group::2: two SMs share one 256 x 256 x 16 MMA and
@@ -209,8 +227,9 @@ typedef struct {
  * internal streams). */
 int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
 
-/* Synchronises `stream` and returns GPTQ_ERR_TIMEOUT if any kernel's bounded wait gave up
- * since the last check (the flag is then cleared), GPTQ_ERR_CUDA on a runtime error, else OK. */
+/* Synchronises `stream` and returns GPTQ_ERR_LAYOUT if a kernel since the last check met a layer whose tiling does
+ * not fit the call (see GPTQ_FORMAT_GATE_UP), GPTQ_ERR_TIMEOUT if a kernel's bounded wait gave up (the flag is
+ * cleared either way), GPTQ_ERR_CUDA on a runtime error, else OK. */
 int gptq_check_status(void *stream);
 
 /* Self-test of that mechanism (no counterpart in the paper): launches one thread that waits, the way the matmul

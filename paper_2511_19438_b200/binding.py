@@ -22,6 +22,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 GPTQ_FORMAT_ZEROS_MINUS_ONE = 1
+GPTQ_FORMAT_GATE_UP = 2
 GPTQ_OK = 0
 GPTQ_ERR_NULL = -1
 GPTQ_ERR_SHAPE = -2
@@ -68,6 +69,7 @@ _SIGNATURES = {
     "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "gptq_set_workspace": (_i, [_vp, _sz]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_silu_mul": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_set_cta_pairs": (_i, [_i]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
@@ -184,6 +186,11 @@ def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_st
     return _lib.gptq_gemm_host(_ptr(x_host), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx),
                                _ptr(y_host), _ptr(x_stage), _ptr(y_stage), M, N, K, group_size,
                                int(act_order), _stream(stream))
+
+
+def gptq_gemm_silu_mul(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, stream=None) -> int:
+    return _lib.gptq_gemm_silu_mul(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(out), M, N,
+                                   K, group_size, int(act_order), _stream(stream))
 
 
 def gptq_gemm_noalloc(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:

@@ -189,11 +189,12 @@ int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void 
                             float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
                             void *stream)
 {
-    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
+    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP)) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !w_out || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
     if (st) return st;
     if (repacked != 0 && repacked != 1) return GPTQ_ERR_LAYOUT;
+    if (!repacked && (format & GPTQ_FORMAT_GATE_UP)) return GPTQ_ERR_LAYOUT;   // a property of the tiled layout only
     if (repacked) {
         st = check_fast_path(N, K, group_size);
         if (st) return st;
@@ -227,7 +228,7 @@ int gptq_repack_format(const int32_t *qweight, const int32_t *qzeros, const void
                        void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
                        int group_size, int act_order, int format, void *stream)
 {
-    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
+    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP)) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out) return GPTQ_ERR_NULL;
     if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
@@ -359,8 +360,11 @@ int gptq_set_workspace(void *ptr, size_t bytes)
     return GPTQ_OK;
 }
 
-int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
-              void *y, int M, int N, int K, int group_size, int act_order, void *stream)
+} // extern "C"
+
+// y = x W (fuse == 0, y is [M, N]) or silu(gate) * up of y's column halves (fuse == 1, y is [M, N / 2])
+static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                         void *y, int M, int N, int K, int group_size, int act_order, int fuse, void *stream)
 {
     if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(M, N, K, group_size);
@@ -387,23 +391,39 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
         if (st) return st;
         xin = x_perm;
     }
+    const size_t ldy = fuse ? (size_t)N / 2 : (size_t)N;
     if (M >= kUmmaMinTokens) {
-        if (g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
+        if (!fuse && g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
             const Umma2Plan p2 = plan_umma2(M, N, K);
             return launch_umma2(xin, qweight, qzeros, scales, (__half *)y, M, N, K, p2, s);
         }
         // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
-        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, s);
+        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, fuse, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
         const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sms);
-        st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * N, rows, N, K,
-                           pl, s);
+        st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * ldy, rows, N, K,
+                           pl, fuse, s);
         if (st) return st;
     }
     return GPTQ_OK;
+}
+
+extern "C" {
+
+int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+              void *y, int M, int N, int K, int group_size, int act_order, void *stream)
+{
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, stream);
+}
+
+int gptq_gemm_silu_mul(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                       const int32_t *g_idx, void *out, int M, int N, int K, int group_size, int act_order,
+                       void *stream)
+{
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, stream);
 }
 
 int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, const void *scales,
@@ -602,7 +622,7 @@ int gptq_check_status(void *stream)
     e = cudaMemcpyToSymbolAsync(g_device_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return record_cuda_error(e);
-    return GPTQ_ERR_TIMEOUT;
+    return status == kStatusLayoutMismatch ? GPTQ_ERR_LAYOUT : GPTQ_ERR_TIMEOUT;
 }
 
 }  // extern "C"

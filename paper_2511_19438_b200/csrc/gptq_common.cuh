@@ -46,6 +46,19 @@ constexpr int kItemZBytes = 64;      // packed zeros of one group of one item
 constexpr int kTrailerBytes = 16;
 constexpr uint32_t kTrailerMagic = 0x51545047u;   // "GPTQ"
 constexpr uint32_t kFormatZerosMinusOne = 1u;     // == GPTQ_FORMAT_ZEROS_MINUS_ONE
+constexpr uint32_t kFormatGateUp = 2u;            // == GPTQ_FORMAT_GATE_UP: column halves interleaved per panel
+// With kFormatGateUp a layer's columns are [gate | up] (N / 2 each) and tiled panel p holds gate columns
+// 64 p .. 64 p + 63 in its first half and the matching up columns in its second, so that one CTA sees both.
+__host__ __device__ inline int gate_up_source_column(int nt, int N)      // tiled column -> checkpoint column
+{
+    const int p = nt / kPanel, c = nt % kPanel;
+    return (c / 64) * (N / 2) + 64 * p + (c % 64);
+}
+__host__ __device__ inline int gate_up_tiled_column(int n, int N)        // checkpoint column -> tiled column
+{
+    const int half = n / (N / 2), rem = n % (N / 2);
+    return (rem / 64) * kPanel + half * 64 + (rem % 64);
+}
 struct TiledTrailer {
     uint32_t magic, flags, group_size, reserved;
 };
@@ -89,7 +102,7 @@ __host__ __device__ inline size_t repacked_zero_byte(int grp, int n, int groups,
 // ----------------------------------------------------------------------------------------
 // Device status word: kernels never trap; a bounded wait that gives up records a code here.
 // ----------------------------------------------------------------------------------------
-enum : int { kStatusOk = 0, kStatusWaitTimeout = 1 };                  // g_device_status, recorded with atomicMax
+enum : int { kStatusOk = 0, kStatusWaitTimeout = 1, kStatusLayoutMismatch = 2 };   // g_device_status, recorded with atomicMax
 enum : int { kGidxOk = 0, kGidxUnequalGroups = 1, kGidxOutOfRange = 2 };   // g_gidx_status, likewise
 // The library is built as one translation unit, so these are the single definitions.  The g_idx
 // check of gptq_repack has a word of its own, so that reading and clearing it never drops a

@@ -70,14 +70,15 @@ __global__ void dequant_tiled_kernel(const uint8_t *__restrict__ qweight, const 
     int i = (int)(idx / N), n = (int)(idx % N);
     int groups = K / group_size, grp = i / group_size;
     int slot, hi;
-    size_t off = repacked_word_offset(i, n, K / kGroup, &slot);
+    // the trailer says whether the stored zero points are one too small and whether the column halves are interleaved
+    const TiledTrailer *tr = reinterpret_cast<const TiledTrailer *>(qzeros + tiled_zero_bytes(N, K, group_size));
+    const int nt = (tr->flags & kFormatGateUp) ? gate_up_tiled_column(n, N) : n;
+    size_t off = repacked_word_offset(i, nt, K / kGroup, &slot);
     uint32_t word = *reinterpret_cast<const uint32_t *>(qweight + off);
     int q = (int)((word >> (4 * slot)) & 15u);
-    // the trailer says whether the stored zero points are one too small
-    const TiledTrailer *tr = reinterpret_cast<const TiledTrailer *>(qzeros + tiled_zero_bytes(N, K, group_size));
-    uint8_t zb = qzeros[repacked_zero_byte(grp, n, groups, &hi)];
+    uint8_t zb = qzeros[repacked_zero_byte(grp, nt, groups, &hi)];
     int z = (hi ? (zb >> 4) : (zb & 15)) + (int)(tr->flags & kFormatZerosMinusOne);
-    float s = __half2float(scales[repacked_scale_index(grp, n, groups)]);
+    float s = __half2float(scales[repacked_scale_index(grp, nt, groups)]);
     int k = perm ? perm[i] : i;
     w_out[(size_t)k * N + n] = __fmul_rn((float)(q - z), s);
 }
@@ -138,7 +139,7 @@ __global__ void argsort_gidx_kernel(const int32_t *__restrict__ g_idx, int32_t *
 // ------------------------------------------------------------------------------ repack
 // One thread per output word of the tiled layout.
 __global__ void repack_weights_kernel(const int32_t *__restrict__ qweight, const int32_t *__restrict__ perm,
-                                      uint32_t *__restrict__ out, int N, int K)
+                                      uint32_t *__restrict__ out, int N, int K, int gate_up)
 {
     size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     size_t words = (size_t)(K / 8) * N;
@@ -150,6 +151,7 @@ __global__ void repack_weights_kernel(const int32_t *__restrict__ qweight, const
     int p = (int)(item / G), grp = (int)(item % G);
     int g = lane >> 2, t4 = lane & 3, j = c & 1, h = c >> 1;
     int n = p * kPanel + 16 * u + g + 8 * h;
+    if (gate_up) n = gate_up_source_column(n, N);
     int i0 = grp * kGroup + blk * 64 + j * 32 + t4 * 8;
     uint32_t word = 0;
     if (perm == nullptr) {
@@ -179,15 +181,18 @@ __global__ void repack_meta_kernel(const int32_t *__restrict__ qzeros, const __h
         *reinterpret_cast<TiledTrailer *>(z_out + (size_t)G * (N / 2)) = tr;
     }
     if (idx >= (size_t)G * N) return;
-    int grp = (int)(idx / N), n = (int)(idx % N);
-    s_out[repacked_scale_index(grp, n, G)] = scales[idx];
-    if (((n % 16) >> 3) == 0) {
+    // one thread per (group, tiled column nt); its values come from checkpoint column n
+    int grp = (int)(idx / N), nt = (int)(idx % N);
+    const bool gate_up = (flags & kFormatGateUp) != 0;
+    int n = gate_up ? gate_up_source_column(nt, N) : nt;
+    s_out[repacked_scale_index(grp, nt, G)] = scales[(size_t)grp * N + n];
+    if (((nt % 16) >> 3) == 0) {
         const int32_t *zrow = qzeros + (size_t)grp * (N / 8);
         uint32_t za = ((uint32_t)zrow[n >> 3] >> (4 * (n & 7))) & 15u;
-        int nb = n + 8;
+        int nb = n + 8;     // the partner column: eight further in both numberings (halves are multiples of 64)
         uint32_t zb = ((uint32_t)zrow[nb >> 3] >> (4 * (nb & 7))) & 15u;
         int hi;
-        z_out[repacked_zero_byte(grp, n, G, &hi)] = (uint8_t)(za | (zb << 4));
+        z_out[repacked_zero_byte(grp, nt, G, &hi)] = (uint8_t)(za | (zb << 4));
     }
 }
 
@@ -221,7 +226,8 @@ int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *sca
     }
     size_t words = (size_t)(K / 8) * N;
     repack_weights_kernel<<<(unsigned)((words + T - 1) / T), T, 0, s>>>(qweight, act_order ? perm_out : nullptr,
-                                                                        (uint32_t *)qweight_out, N, K);
+                                                                        (uint32_t *)qweight_out, N, K,
+                                                                        (format & (int)kFormatGateUp) ? 1 : 0);
     size_t meta = (size_t)G * N;
     repack_meta_kernel<<<(unsigned)((meta + T - 1) / T), T, 0, s>>>(qzeros, (const __half *)scales,
                                                                     (uint8_t *)qzeros_out, (__half *)scales_out, N, G,

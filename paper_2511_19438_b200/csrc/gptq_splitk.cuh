@@ -91,7 +91,11 @@ struct SplitKArgs {
     int S;                  // CTAs per panel = cluster size
     int stages;
     const TiledTrailer *trailer;   // behind the tiled zero points
+    int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
 };
+
+// silu(g) * u in fp32
+__device__ __forceinline__ float silu_mul(float g, float u) { return g / (1.f + __expf(-g)) * u; }
 
 struct SplitKPlan {
     int m_tile;     // 8 or 16
@@ -145,6 +149,10 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
     const int g = lane >> 2, t4 = lane & 3;
+    // a layer tiled for the fused gate/up epilogue must be used with it, and only with it: otherwise nothing is
+    // stored and the status word says so
+    const bool layout_ok = ((__ldg(&a.trailer->flags) & kFormatGateUp) != 0) == (a.fuse != 0);
+    if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------------ producer (one thread)
@@ -211,15 +219,44 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     const int col = warp * 16 + g;
     const int m_lo = token_row_of_slot(2 * t4), m_hi = token_row_of_slot(2 * t4 + 1);
     if (S == 1) {
-        if (warp < kConsumerWarps) {
-            __half *yp = a.y + (size_t)p * kPanel + col;
+        if (warp < kConsumerWarps && layout_ok) {
+            if (!a.fuse) {
+                __half *yp = a.y + (size_t)p * kPanel + col;
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
+                for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
-                    if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
+                    for (int i = 0; i < 4; ++i) {
+                        const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
+                        if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
+                    }
+            } else {
+                // warps 4-7 hold the up columns of the gate columns of warps 0-3: hand them over through the
+                // (unused) receive buffer, [token][64 columns] floats
+                const uint32_t hand = ring + (uint32_t)a.stages * kStage;
+                if (warp >= 4) {
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
+                            if (m < a.M) sts_f32(hand + (uint32_t)(m * 64 + col - 64 + 8 * (i >> 1)) * 4u, acc[mt][i]);
+                        }
                 }
+                named_bar_sync(1, kConsumerThreads);
+                if (warp < 4) {
+                    __half *yp = a.y + (size_t)p * 64 + col;
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
+                            if (m < a.M) {
+                                const float up = lds_f32(hand + (uint32_t)(m * 64 + col + 8 * (i >> 1)) * 4u);
+                                yp[(size_t)m * (a.N / 2) + 8 * (i >> 1)] = __float2half_rn(silu_mul(acc[mt][i], up));
+                            }
+                        }
+                }
+            }
         }
         return;
     }
@@ -236,24 +273,41 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             for (int i = 0; i < 4; ++i) {
                 const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                 if (m < a.M) {
-                    const int c = col + 8 * (i >> 1), q = c / width;
-                    const uint32_t off = (uint32_t)((rank * a.M + m) * width + (c - q * width)) * 4u;
+                    // owner q gets columns [q width, (q + 1) width); with the fused epilogue the first half of its
+                    // slice are gate columns [q width / 2, ...) and the second half the matching up columns
+                    const int c = col + 8 * (i >> 1);
+                    const int half_w = width >> 1, cc = c & 63;
+                    const int q = a.fuse ? cc / half_w : c / width;
+                    const int pos = a.fuse ? (c >> 6) * half_w + (cc - q * half_w) : c - q * width;
+                    const uint32_t off = (uint32_t)((rank * a.M + m) * width + pos) * 4u;
                     st_async_f32(map_to_cluster_rank(recv + off, (uint32_t)q), acc[mt][i],
                                  map_to_cluster_rank(bar_recv, (uint32_t)q));
                 }
             }
-        if (mbar_wait_cluster(bar_recv, 0)) {
-            const int c_lo = rank * width;
-            for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
-                const int m = idx / width, cc = idx - m * width;
+        if (mbar_wait_cluster(bar_recv, 0) && layout_ok) {
+            auto slice_sum = [&](int m, int cc) {   // rank order
                 float v[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
                     v[q] = q < S ? lds_f32(recv + (uint32_t)((q * a.M + m) * width + cc) * 4u) : 0.f;
                 float sum = 0.f;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) sum += v[q];   // rank order
-                a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(sum);
+                for (int q = 0; q < 8; ++q) sum += v[q];
+                return sum;
+            };
+            if (!a.fuse) {
+                const int c_lo = rank * width;
+                for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
+                    const int m = idx / width, cc = idx - m * width;
+                    a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(slice_sum(m, cc));
+                }
+            } else {
+                const int half_w = width >> 1;
+                for (int idx = threadIdx.x; idx < a.M * half_w; idx += kConsumerThreads) {
+                    const int m = idx / half_w, cc = idx - m * half_w;
+                    a.y[(size_t)m * (a.N / 2) + (size_t)p * 64 + rank * half_w + cc] =
+                        __float2half_rn(silu_mul(slice_sum(m, cc), slice_sum(m, half_w + cc)));
+                }
             }
         }
     }
@@ -333,7 +387,7 @@ static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, co
 }
 
 int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
-                  int M, int N, int K, const SplitKPlan &plan, cudaStream_t s)
+                  int M, int N, int K, const SplitKPlan &plan, int fuse, cudaStream_t s)
 {
     SplitKArgs args;
     args.qweight = (const uint8_t *)qweight;
@@ -346,6 +400,7 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
+    args.fuse = fuse;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;

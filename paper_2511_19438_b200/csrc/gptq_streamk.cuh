@@ -153,6 +153,11 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     const int t0 = sk_range_begin(T, C, c), t1 = sk_range_begin(T, C, c + 1);
     const int stages = a.stages;
     __shared__ int s_last;
+    // this kernel has no fused gate/up epilogue: a layer tiled for one is refused by every CTA before any barrier exists
+    if (__ldg(&a.trailer->flags) & kFormatGateUp) {
+        if (threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
+        return;
+    }
 
     if (threadIdx.x == kConsumerThreads) {
         for (int s = 0; s < stages; ++s) {

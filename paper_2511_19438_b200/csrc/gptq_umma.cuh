@@ -147,6 +147,7 @@ struct UmmaArgs {
     int tile0;              // first output tile of this launch (a matmul may take a main and a tail launch)
     int stages;             // shared-memory ring depth
     const TiledTrailer *trailer;   // behind the tiled zero points
+    int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
 };
 
 // K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
@@ -222,6 +223,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     tc_fence_after_sync();
     const uint32_t tmem_base = lds32(tmem_slot);
     pdl_launch_dependents();
+    // a layer tiled for the fused gate/up epilogue must be used with it, and only with it (else: nothing is stored)
+    const bool layout_ok = ((__ldg(&a.trailer->flags) & kFormatGateUp) != 0) == (a.fuse != 0);
+    if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (one thread)
@@ -407,6 +411,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         pdl_wait();
         ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
         if (ok) tc_fence_after_sync();
+        ok = ok && layout_ok;
         if (S == 1) {
             // The accumulator holds a column of y per TMEM lane, so a thread's 32 values of a chunk belong to 32
             // different rows of y.  The four warps of a set turn their 32-token x 128-column chunk around through
@@ -429,7 +434,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                         sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
                 }
                 named_bar_sync(bar_id, 128);
-                if (ok) {
+                if (ok && !a.fuse) {
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
                         const int piece = tq + 128 * t, row = piece >> 4, c16 = piece & 15;   // 16 pieces per row
@@ -437,6 +442,29 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                         if (m < a.M && c0 + row < TOK) {
                             const uint4 v = lds128(stg + (uint32_t)piece * 16u);
                             *reinterpret_cast<uint4 *>(a.y + (size_t)m * a.N + (size_t)p * kPanel + c16 * 8) = v;
+                        }
+                    }
+                } else if (ok) {
+                    // fused gate/up epilogue: the first 64 staged columns of a row are gate, the last 64 the matching up
+                    // columns (both already rounded to fp16); eight outputs (16 bytes of the N / 2 wide row) per piece
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const int piece = tq + 128 * t, row = piece >> 3, c8 = piece & 7;     // 8 output pieces per row
+                        const int m = m0 + c0 + row;
+                        if (m < a.M && c0 + row < TOK) {
+                            const uint4 gv = lds128(stg + (uint32_t)(row * 256 + c8 * 16));
+                            const uint4 uv = lds128(stg + (uint32_t)(row * 256 + 128 + c8 * 16));
+                            const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
+                            uint32_t ow[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 gf = __half22float2(*reinterpret_cast<const __half2 *>(&gw[e]));
+                                const float2 uf = __half22float2(*reinterpret_cast<const __half2 *>(&uw[e]));
+                                const __half2 o = __floats2half2_rn(silu_mul(gf.x, uf.x), silu_mul(gf.y, uf.y));
+                                ow[e] = *reinterpret_cast<const uint32_t *>(&o);
+                            }
+                            *reinterpret_cast<uint4 *>(a.y + (size_t)m * (a.N / 2) + (size_t)p * 64 + c8 * 8) =
+                                make_uint4(ow[0], ow[1], ow[2], ow[3]);
                         }
                     }
                 }
@@ -462,13 +490,11 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         __syncwarp();
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (warp >= 2) {
+        if (warp >= 2 && layout_ok) {
             const int p = p0;   // split-K runs with one panel per CTA (NP == 1)
             const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
-            const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;
-            const int w4 = width >> 2;      // width is 16, 32 or 64: four columns (16 bytes) per thread and step
-            for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
-                const int m = idx / w4, cc = c_lo + 4 * (idx - m * w4);
+            // four columns of token row m, starting at tile column cc, summed over the cluster in rank order
+            auto sum4 = [&](int m, int cc) {
                 const uint32_t local = ring + (uint32_t)(m * kPanel + cc) * 4u;
                 float4 v[8];
 #pragma unroll
@@ -476,17 +502,38 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     v[qq] = qq < S ? ld_cluster_f32x4(map_to_cluster_rank(local, (uint32_t)qq)) : make_float4(0.f, 0.f, 0.f, 0.f);
                 float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int qq = 0; qq < 8; ++qq) {   // rank order
+                for (int qq = 0; qq < 8; ++qq) {
                     sum.x += v[qq].x;
                     sum.y += v[qq].y;
                     sum.z += v[qq].z;
                     sum.w += v[qq].w;
                 }
-                const __half2 lo = __floats2half2_rn(sum.x, sum.y), hi = __floats2half2_rn(sum.z, sum.w);
+                return sum;
+            };
+            auto store4 = [&](__half *dst, float4 v) {
+                const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
                 uint2 out;
                 out.x = *reinterpret_cast<const uint32_t *>(&lo);
                 out.y = *reinterpret_cast<const uint32_t *>(&hi);
-                *reinterpret_cast<uint2 *>(a.y + (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc) = out;
+                *reinterpret_cast<uint2 *>(dst) = out;
+            };
+            const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;   // width is 16, 32 or 64
+            if (!a.fuse) {
+                const int w4 = width >> 2;      // four columns (16 bytes) per thread and step
+                for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
+                    const int m = idx / w4, cc = c_lo + 4 * (idx - m * w4);
+                    store4(a.y + (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc, sum4(m, cc));
+                }
+            } else {
+                // this CTA finishes gate columns [rank width / 2, ...) of the tile and the matching up columns 64 further
+                const int half_w = width >> 1, w4 = half_w >> 2;
+                for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
+                    const int m = idx / w4, cc = rank * half_w + 4 * (idx - m * w4);
+                    const float4 gsum = sum4(m, cc), usum = sum4(m, 64 + cc);
+                    store4(a.y + (size_t)(m0 + m) * (a.N / 2) + (size_t)p * 64 + cc,
+                           make_float4(silu_mul(gsum.x, usum.x), silu_mul(gsum.y, usum.y), silu_mul(gsum.z, usum.z),
+                                       silu_mul(gsum.w, usum.w)));
+                }
             }
         }
         // no CTA may exit (and free its shared memory) while a peer can still read its tile
@@ -630,7 +677,7 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
 }
 
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
-                int K, int group_size, const UmmaPlan &plan, cudaStream_t s)
+                int K, int group_size, const UmmaPlan &plan, int fuse, cudaStream_t s)
 {
     UmmaArgs args;
     args.scales = (const uint8_t *)scales;
@@ -642,6 +689,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.G = K / kGroup;
     args.S = plan.S;
     args.stages = plan.stages;
+    args.fuse = fuse;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, group_size));
     const int sub = kGroup / group_size;
     if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;

@@ -87,6 +87,11 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
     const int mt = pair / ptiles, p = (pair - mt * ptiles) * 2 + rank;   // this CTA's weight panel
     const int m0 = mt * kUmma2Tok;
     const int NB = a.K / kUmmaBlockK;
+    // this kernel has no fused gate/up epilogue: a layer tiled for one is refused by every CTA before any barrier exists
+    if (__ldg(&a.trailer->flags) & kFormatGateUp) {
+        if (threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(bar_full + 8 * s, 1);
@@ -340,6 +345,7 @@ int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const
     args.G = K / kGroup;
     args.S = 1;
     args.stages = plan.stages;
+    args.fuse = 0;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup));
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;

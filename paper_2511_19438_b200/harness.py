@@ -33,7 +33,7 @@ def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a)).to(device)
 
 
-def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda") -> DeviceLinear:
+def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda", gate_up: bool = False) -> DeviceLinear:
     qw = to_device(L.qweight, device)
     qz = to_device(L.qzeros, device)
     sc = to_device(L.scales, device)
@@ -42,7 +42,7 @@ def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda
     qz_t = torch.empty(B.gptq_repack_bytes(1, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     sc_t = torch.empty(B.gptq_repack_bytes(2, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     perm = torch.empty(L.K, dtype=torch.int32, device=device) if L.act_order else None
-    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0
+    fmt = (B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0) | (B.GPTQ_FORMAT_GATE_UP if gate_up else 0)
     B.check(B.gptq_repack_format(qw, qz, sc, gi, qw_t, qz_t, sc_t, perm, L.N, L.K, L.group_size, L.act_order, fmt),
             "gptq_repack_format")
     torch.cuda.current_stream().synchronize()
@@ -78,3 +78,13 @@ def gemm(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream
     B.check(B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, D.N, D.K, D.group_size,
                         D.act_order, stream), "gptq_gemm")
     return y
+
+
+def gemm_silu_mul(x: torch.Tensor, D: DeviceLinear, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """out[M, N / 2] = silu(gate) * up through gptq_gemm_silu_mul (D repacked with gate_up=True)."""
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, D.N // 2), dtype=torch.float16, device=x.device)
+    B.check(B.gptq_gemm_silu_mul(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, out, M, D.N, D.K, D.group_size,
+                                 D.act_order, stream), "gptq_gemm_silu_mul")
+    return out

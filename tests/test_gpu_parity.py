@@ -439,7 +439,7 @@ def test_variant_dequant_bit_exact(gs, act, zm1):
     w.zero_()
     B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
     assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
-    assert B.gptq_dequant_f32_format(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 2) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_dequant_f32_format(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 4) == B.GPTQ_ERR_LAYOUT
 
 
 @pytest.mark.parametrize("gs,act,zm1", VARIANTS)
@@ -482,8 +482,123 @@ def test_variants_unsupported_entry_points():
     assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 4, N, K, 16, 0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack_format(D.qweight_t, D.qzeros_t, D.scales_t, None, D.qweight_t, D.qzeros_t, D.scales_t, None,
                                 N, K, 64, 0, 4) == B.GPTQ_ERR_LAYOUT
+    w = torch.zeros((K, N), dtype=torch.float32, device="cuda")     # the interleave is no property of a checkpoint
+    assert B.gptq_dequant_f32_format(H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales), None, w,
+                                     N, K, 64, 0, 0, B.GPTQ_FORMAT_GATE_UP) == B.GPTQ_ERR_LAYOUT
     torch.cuda.synchronize()
     assert torch.count_nonzero(y) == 0
+
+
+# ------------------------------------------------------------------------------- fused gate/up epilogue
+def silu_mul_bound(y64: np.ndarray, K: int) -> np.ndarray:
+    """What the stated matmul tolerance allows for out = silu(g) * u when g and u each carry an error of at most
+    t(v) = 1e-2 sqrt(K/4096) + 1e-2 |v|: since -0.1 < silu' < 1.1, |d out| <= 1.1 t(g) |u| + |silu(g)| t(u)
+    + 1.1 t(g) t(u), plus the final fp16 rounding of out."""
+    half = y64.shape[1] // 2
+    g, u = y64[:, :half], y64[:, half:]
+    tg = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(g)
+    tu = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(u)
+    out = oracle.silu_mul_f64(y64)
+    return 1.1 * tg * np.abs(u) + np.abs(g / (1 + np.exp(-g))) * tu + 1.1 * tg * tu + 2.0 ** -11 * np.abs(out) + 1e-7
+
+
+def check_silu_mul(L, x_np, ws):
+    D = H.upload_and_repack(L, gate_up=True)
+    ws.ensure_for(x_np.shape[0], D)
+    out = H.gemm_silu_mul(H.to_device(x_np), D)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size, zeros_minus_one=L.zeros_minus_one)
+    want = oracle.silu_mul_f64(y64)
+    got = out.cpu().numpy().astype(np.float64)
+    assert got.shape == want.shape and np.all(np.isfinite(got))
+    err = np.abs(got - want)
+    bound = silu_mul_bound(y64, L.K)
+    assert np.all(err <= bound), f"{int((err > bound).sum())} violations, worst ratio {(err / bound).max():.2f}"
+    # the bound above is what the contract allows; the kernels (fp32 sums, at most one fp16 rounding of each factor)
+    # should sit far inside it
+    assert np.sqrt(np.mean(err ** 2)) <= 0.2 * np.sqrt(np.mean(bound ** 2))
+    return D
+
+
+@pytest.mark.parametrize("gs,act,zm1", [(128, False, False), (128, True, False), (64, False, True), (32, True, False)])
+@pytest.mark.parametrize("M", [1, 7, 16, 23, 50, 130, 300, 513])
+def test_silu_mul_small_layers(gs, act, zm1, M, ws):
+    """A small layer, so that the K range is split over a cluster on every kernel family (the owner of an output
+    column pair sums both factors over the cluster before the activation)."""
+    K, N = 1024, 512
+    L = wl.make_linear(K, N, seed=wl.seed_for("silu", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    check_silu_mul(L, wl.make_x(M, K, wl.seed_for("silu-x", M)), ws)
+
+
+@pytest.mark.parametrize("M", [1, 4, 16, 40, 2040])
+def test_silu_mul_llama7b_gate_up(M, ws):
+    """The merged gate/up projection of the 7B model (K = 4096, N = 2 x 11008): more panels than SMs, so a CTA owns
+    whole panels and the activation is applied straight from its accumulators."""
+    K, N = wl.SHAPES_7B["gate_up"]
+    L = wl.make_linear(K, N, seed=wl.seed_for("silu-7b"))
+    check_silu_mul(L, wl.make_x(M, K, wl.seed_for("silu-7b-x", M)), ws)
+
+
+def test_silu_mul_layout_round_trip_and_mismatch(ws):
+    """The interleaved tiling dequantises back to the checkpoint's column order bit for bit, and each matmul entry
+    point refuses the tiling it was not built for: nothing is stored and the status word says so once."""
+    K, N, M = 512, 512, 5
+    L = wl.make_linear(K, N, seed=wl.seed_for("silu-layout"), act_order=True)
+    x = H.to_device(wl.make_x(M, K, 3))
+    D_gu = H.upload_and_repack(L, gate_up=True)
+    D = H.upload_and_repack(L)
+    ws.ensure_for(40, D)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    B.check(B.gptq_dequant_f32(D_gu.qweight_t, D_gu.qzeros_t, D_gu.scales_t, D_gu.perm, w, N, K, 128, 1, 1), "dequant")
+    want = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert not torch.equal(D_gu.qweight_t, D.qweight_t)
+    for rows in (M, 40):                                   # mma.sync and tcgen05 kernels
+        xr = H.to_device(wl.make_x(rows, K, 4))
+        y = torch.zeros((rows, N), dtype=torch.float16, device="cuda")
+        H.gemm(xr, D_gu, y)
+        assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+        assert "layout" in B.gptq_status_string(B.GPTQ_ERR_LAYOUT)
+        assert B.gptq_check_status() == B.GPTQ_OK
+        assert torch.count_nonzero(y) == 0
+        out = torch.zeros((rows, N // 2), dtype=torch.float16, device="cuda")
+        H.gemm_silu_mul(xr, D, out)
+        assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+        assert torch.count_nonzero(out) == 0
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    B.check(B.gptq_gemm_noalloc(x, D_gu.qweight_t, D_gu.qzeros_t, D_gu.scales_t, D_gu.perm, y, M, N, K, 128, 1), "noalloc")
+    assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+    assert torch.count_nonzero(y) == 0
+    B.check(B.gptq_set_cta_pairs(1), "pairs on")
+    try:
+        xr = H.to_device(wl.make_x(256, K, 5))
+        y = torch.zeros((256, N), dtype=torch.float16, device="cuda")
+        H.gemm(xr, D_gu, y)
+        assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+        assert torch.count_nonzero(y) == 0
+    finally:
+        B.check(B.gptq_set_cta_pairs(0), "pairs off")
+    full_check(L, wl.make_x(M, K, 3), H.gemm(x, D).cpu().numpy())          # and the context is still usable
+
+
+def test_silu_mul_special_values(ws):
+    """Scales 1, zero points 8, one-hot x rows: y is the integer q - 8 of one weight row, so out must be the fp16
+    rounding of silu(q_gate - 8) * (q_up - 8) computed in double - exact arguments, the activation alone is tested."""
+    K, N = 256, 256
+    r = np.random.default_rng(9)
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    L = wl.make_linear_from_values(q, np.full((K // 128, N), 8, np.uint8), np.ones((K // 128, N), np.float16), 128)
+    for M in (3, 20):
+        x = np.zeros((M, K), np.float16)
+        rows = r.integers(0, K, M)
+        x[np.arange(M), rows] = 1
+        D = H.upload_and_repack(L, gate_up=True)
+        out = H.gemm_silu_mul(H.to_device(x), D).cpu().numpy()
+        assert B.gptq_check_status() == B.GPTQ_OK
+        y64 = q[rows].astype(np.float64) - 8.0
+        want = oracle.silu_mul_f64(y64)
+        assert np.all(np.abs(out.astype(np.float64) - want) <= 2.0 ** -10 * np.abs(want) + 1e-7)
+        assert np.all(out[y64[:, N // 2:] == 0] == 0) and np.all(out[y64[:, :N // 2] == 0] == 0)
 
 
 def test_bounded_wait_reports_timeout():
