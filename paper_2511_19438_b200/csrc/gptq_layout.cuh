@@ -252,9 +252,20 @@ __global__ void gather_x_kernel(const __half *__restrict__ x, const int32_t *__r
 int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, int K, cudaStream_t s)
 {
     const int T = 256;
-    dim3 grid((K + T - 1) / T, (unsigned)min(M, 64));
-    gather_x_kernel<<<grid, T, 0, s>>>(x, perm, x_out, M, K);
-    return record_cuda_error(cudaGetLastError());
+    // launched as a programmatic dependent of the kernel before it: its CTAs become resident while that kernel still
+    // runs, and griddepcontrol.wait holds the copy back until that kernel (which may write x, and may still be reading
+    // the previous contents of x_out) has completed
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((K + T - 1) / T, (unsigned)min(M, 64));
+    cfg.blockDim = dim3(T);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, gather_x_kernel, x, perm, x_out, M, K));
 }
 
 }  // namespace gptq

@@ -33,7 +33,16 @@ namespace gptq {
 
 // warp 0: TMA producer, warp 1: MMA issue + TMEM, then four dequant/epilogue warps per panel of the CTA
 // (two sets of them, taking alternate K groups, when one warp per scheduler cannot keep up with the MMA)
-__host__ __device__ constexpr int umma_threads(int NP, int SETS) { return 64 + 128 * NP * SETS; }
+// MMA-issuing warps: one thread pays 60-110 cycles for every instruction it issues (and more when its scheduler is
+// shared with busy dequant warps).  With 64-token tiles each dequant warp set gets an issuing warp and an accumulator
+// of its own, and the epilogue adds the accumulators (measured 0-6 % faster there; with 32-token tiles the third
+// resident CTA that a single accumulator leaves room for is worth more).
+__host__ __device__ constexpr int umma_issuers(int TOK, int SETS) { return (TOK == 64 && SETS == 2) ? 2 : 1; }
+// warp 0: TMA producer; warps 1 .. ISS: MMA issue; then four dequant warps per panel and set
+__host__ __device__ constexpr int umma_threads(int TOK, int NP, int SETS)
+{
+    return 32 * (1 + umma_issuers(TOK, SETS)) + 128 * NP * SETS;
+}
 constexpr int kUmmaDequantWarps = 4;     // per panel: one warp per 32 TMEM lanes
 constexpr int kUmmaBlockK = 64;
 constexpr int kUmmaWBlockBytes = 4096;   // packed weights of one K64 block of a panel
@@ -159,16 +168,16 @@ __host__ __device__ constexpr int umma_slot_bytes(int TOK, int NP)
 {
     return (umma_blocks_per_slot(TOK) * (TOK * 128 + NP * kUmmaWBlockBytes) + 1023) & ~1023;
 }
-__host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP)
+__host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP, int ISS)
 {
-    // per panel: accumulator (TOK columns) + A ring (32 columns = one K64 block per stage); a power of two >= 32
-    int need = NP * (TOK + NA * 32), c = 32;
+    // per panel: accumulators (TOK columns each) + A ring (32 columns = one K64 block per stage); a power of two >= 32
+    int need = NP * (ISS * TOK + NA * 32), c = 32;
     while (c < need) c <<= 1;
     return c;
 }
 
 template <int TOK, int NA, int NP, int SETS, int SUB>
-__global__ void __launch_bounds__(umma_threads(NP, SETS), (NP > 1 || TOK > 128) ? 1 : TOK <= 32 ? 3 : 2)
+__global__ void __launch_bounds__(umma_threads(TOK, NP, SETS), (NP > 1 || TOK > 128) ? 1 : TOK <= 32 ? 3 : 2)
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -177,13 +186,18 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     constexpr int BPS = umma_blocks_per_slot(TOK);
     constexpr int kXTile = TOK * 128;
     constexpr int kOffW = BPS * kXTile;
-    constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP);
-    constexpr uint32_t kAcol = NP * TOK;                   // accumulators first, then the A rings (panel-major)
+    constexpr int ISS = umma_issuers(TOK, SETS);
+    constexpr int kFirstDq = 1 + ISS;                       // first dequant warp
+    constexpr uint32_t kCols = umma_tmem_cols(TOK, NA, NP, ISS);
+    constexpr uint32_t kAcol = NP * ISS * TOK;             // accumulators first, then the A rings (panel-major)
 
     // A warp set jumps 2 SETS - 1 blocks from one K group to its next.  Its parity wait on an A stage is only
     // unambiguous if that jump is no longer than the A ring: then the wait it passed for the previous block implies
     // that the stage's completion before the awaited one has already happened.
     static_assert(SETS == 1 || NA >= 2 * SETS - 1, "A ring too short for this many dequant warp sets");
+    // With two issuers each dequant set must own its A stages (blocks b and b + NA belong to the same set), so that
+    // an issuer sees every completion of the barriers it waits on.
+    static_assert(umma_issuers(TOK, SETS) == 1 || NA == 2 * SETS, "issuers need A stages of their own");
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     // full[s]: the TMA data of ring slot s has landed; a_full: an A stage has been written; done[b mod 16]: the MMAs
     // of K64 block b have completed (one tcgen05.commit per block tells the producer that the block's ring slot and
@@ -210,7 +224,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         }
         for (int s = 0; s < NP * NA; ++s) mbar_init(bar_afull + 8 * s, kUmmaDequantWarps);
         for (int s = 0; s < kUmmaDoneRing; ++s) mbar_init(bar_done + 8 * s, 1);
-        mbar_init(bar_dfull, 1);
+        mbar_init(bar_dfull, ISS);
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -270,18 +284,24 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 if (++s == NS) s = 0;
             }
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issue (one thread)
+    } else if (warp <= ISS) {
+        // ---------------------------------------------------------------- MMA issue (one thread per issuing warp)
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_f16(128, TOK);
-            // One thread, and every instruction it issues costs it 60-110 cycles (a tcgen05.mma about 60, a commit
+            // Every instruction this thread issues costs it 60-110 cycles (a tcgen05.mma about 60, a commit
             // about 80, a barrier wait about 100 even when the barrier is ready), so the loop is kept to one wait
             // per panel, the four MMAs and one commit per K64 block.  It does not wait for the slot's TMA data
             // itself: the dequant warps did before they wrote the A stage, and their a_full arrival orders it.
-            int s = 0, sa = 0;
-            uint32_t pha = 0;
+            // With one issuer it takes the blocks in order; with two, issuer t takes the blocks of dequant set t
+            // (K groups t, t + SETS, ...) and accumulates them in its own tensor-memory columns.
+            const int t = warp - 1;
+            const int b_begin = ISS == 1 ? 0 : 2 * t;
+            int b = b_begin;
+            int s = (b / BPS) % NS;
             bool ok = true;
-            for (int b = 0; b < NB && ok; ++b) {
+            while (b < NB && ok) {
+                const int sa = b % NA;
+                const uint32_t pha = (uint32_t)(b / NA) & 1u;
                 const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage + (b % BPS) * kXTile);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
@@ -290,21 +310,24 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
-                        umma_f16_ts(tmem_base + j * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
-                                    bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)((b | kk) != 0));
+                        umma_f16_ts(tmem_base + (j * ISS + t) * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
+                                    bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)(b != b_begin || kk != 0));
                 }
                 if (!ok) break;
                 umma_commit(bar_done + 8 * (b & (kUmmaDoneRing - 1)));     // this block's A stage(s) and x tile may be overwritten
-                if ((b % BPS) == BPS - 1 && ++s == NS) s = 0;
-                if (++sa == NA) { sa = 0; pha ^= 1u; }
+                const int step = ISS == 1 ? 1 : ((b & 1) ? 2 * SETS - 1 : 1);   // to this issuer's next block
+                s += (b + step) / BPS - b / BPS;                            // and to that block's ring slot
+                while (s >= NS) s -= NS;
+                b += step;
             }
-            umma_commit(bar_dfull);
+            if (b_begin < NB) umma_commit(bar_dfull);
+            else mbar_arrive(bar_dfull);            // this issuer had no block
         }
     } else {
         // ---------------------------------------------------------------- dequant warps, then epilogue
         const int q = warp & 3;                 // the 32 TMEM lanes this warp may touch
-        const int j = ((warp - 2) >> 2) % NP;   // which of the CTA's panels this warp dequantises
-        const int set = ((warp - 2) >> 2) / NP; // and which K64 blocks: set, set + SETS, ...
+        const int j = ((warp - kFirstDq) >> 2) % NP;   // which of the CTA's panels this warp dequantises
+        const int set = ((warp - kFirstDq) >> 2) / NP; // and which K64 blocks: set, set + SETS, ...
         const int p = p0 + j;
         const int n = 32 * q + lane;            // weight column inside the panel = TMEM lane
         const int u = n >> 4, g = n & 7, h = (n >> 3) & 1;
@@ -412,6 +435,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
         if (ok) tc_fence_after_sync();
         ok = ok && layout_ok;
+        // 32 tokens (from c0) of this lane's column: the sum of the issuers' accumulators (an issuer without blocks,
+        // possible when this CTA has a single K group, left its columns unwritten)
+        auto load_acc = [&](int c0, uint32_t (&r)[32]) {
+            tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + (j * ISS) * TOK + c0, r);
+            tmem_wait_ld();
+            if (ISS > 1 && NB > 2) {
+                uint32_t r2[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + (j * ISS + 1) * TOK + c0, r2);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+            }
+        };
         if (S == 1) {
             // The accumulator holds a column of y per TMEM lane, so a thread's 32 values of a chunk belong to 32
             // different rows of y.  The four warps of a set turn their 32-token x 128-column chunk around through
@@ -427,8 +463,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 if (SETS > 1 && ((c0 >> 5) % SETS) != set) continue;   // the warp sets share the token chunks
                 if (ok) {
                     uint32_t r[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + j * TOK + c0, r);
-                    tmem_wait_ld();
+                    load_acc(c0, r);
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
                         sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
@@ -476,8 +511,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 if (m0 + c0 >= a.M) break;
                 if (SETS > 1 && ((c0 >> 5) % SETS) != set) continue;
                 uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + j * TOK + c0, r);
-                tmem_wait_ld();
+                load_acc(c0, r);
                 // split-K: park the fp32 partial tile [token][column] at the start of the (idle) ring
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
@@ -490,7 +524,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         __syncwarp();
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (warp >= 2 && layout_ok) {
+        if (warp >= kFirstDq && layout_ok) {
             const int p = p0;   // split-K runs with one panel per CTA (NP == 1)
             const int rows = (a.M - m0) < TOK ? (a.M - m0) : TOK;
             // four columns of token row m, starting at tile column cc, summed over the cluster in rank order
@@ -520,14 +554,14 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;   // width is 16, 32 or 64
             if (!a.fuse) {
                 const int w4 = width >> 2;      // four columns (16 bytes) per thread and step
-                for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
+                for (int idx = threadIdx.x - 32 * kFirstDq; idx < rows * w4; idx += 128 * NP * SETS) {
                     const int m = idx / w4, cc = c_lo + 4 * (idx - m * w4);
                     store4(a.y + (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc, sum4(m, cc));
                 }
             } else {
                 // this CTA finishes gate columns [rank width / 2, ...) of the tile and the matching up columns 64 further
                 const int half_w = width >> 1, w4 = half_w >> 2;
-                for (int idx = threadIdx.x - 64; idx < rows * w4; idx += 128 * NP * SETS) {
+                for (int idx = threadIdx.x - 32 * kFirstDq; idx < rows * w4; idx += 128 * NP * SETS) {
                     const int m = idx / w4, cc = rank * half_w + 4 * (idx - m * w4);
                     const float4 gsum = sum4(m, cc), usum = sum4(m, 64 + cc);
                     store4(a.y + (size_t)(m0 + m) * (a.N / 2) + (size_t)p * 64 + cc,
@@ -649,7 +683,7 @@ static int launch_umma_sub(const UmmaArgs &args, const CUtensorMap &w_map, const
     if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)ctas);
-    cfg.blockDim = dim3(umma_threads(NP, SETS));
+    cfg.blockDim = dim3(umma_threads(TOK, NP, SETS));
     cfg.dynamicSmemBytes = (size_t)plan.smem_bytes;
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
