@@ -115,6 +115,9 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     constexpr int kXTile = MT * 1024;                       // one K64 tile of x
     constexpr int kOffW = streamk_x_bytes(MT), kOffS = kOffW + kItemWBytes, kOffZ = kOffS + SUB * kItemSBytes;
 
+    // the layer's format flags are needed late (first item, epilogue): ask for them first, so that the round trip to
+    // HBM hides behind the set-up
+    const uint32_t flags = __ldg(&a.trailer->flags);
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_base;                  // stages x 8 B
     const uint32_t bar_empty = smem_base + 64;            // stages x 8 B
@@ -149,10 +152,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
     const int g = lane >> 2, t4 = lane & 3;
-    // a layer tiled for the fused gate/up epilogue must be used with it, and only with it: otherwise nothing is
-    // stored and the status word says so
-    const bool layout_ok = ((__ldg(&a.trailer->flags) & kFormatGateUp) != 0) == (a.fuse != 0);
-    if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
+    bool layout_ok = true;   // set by the consumer warps; the producer must not wait for the trailer
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------------ producer (one thread)
@@ -189,7 +189,12 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
-        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // weights-side data: no need to wait
+        // weights-side data (no need to wait for earlier kernels); requested at the top of the kernel
+        const uint32_t z_add = flags & kFormatZerosMinusOne;
+        // a layer tiled for the fused gate/up epilogue must be used with it, and only with it: otherwise nothing is
+        // stored and the status word says so
+        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0);
+        if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         pdl_wait();
         const int r = token_row_of_slot(g);
         const uint32_t w_off = kOffW + warp * kUnitBytes + lane * 16;
@@ -266,6 +271,10 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     cluster_wait_acquire();                 // every CTA of the cluster has armed its receive barrier
     if (warp < kConsumerWarps) {
         const int width = kPanel / S;       // S is 2, 4 or 8
+        const int wsh = S == 2 ? 6 : S == 4 ? 5 : 4;   // log2(width): owners and offsets by shifts, not divisions
+        // owner q gets columns [q width, (q + 1) width); with the fused epilogue the first half of its slice are gate
+        // columns [q width / 2, ...) and the second half the matching up columns (64 further in the panel)
+        const int qsh = a.fuse ? wsh - 1 : wsh, cmask = a.fuse ? 63 : 127;
         const uint32_t recv = ring + (uint32_t)a.stages * kStage;   // [sender rank][token row][width] floats
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -273,12 +282,9 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             for (int i = 0; i < 4; ++i) {
                 const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                 if (m < a.M) {
-                    // owner q gets columns [q width, (q + 1) width); with the fused epilogue the first half of its
-                    // slice are gate columns [q width / 2, ...) and the second half the matching up columns
-                    const int c = col + 8 * (i >> 1);
-                    const int half_w = width >> 1, cc = c & 63;
-                    const int q = a.fuse ? cc / half_w : c / width;
-                    const int pos = a.fuse ? (c >> 6) * half_w + (cc - q * half_w) : c - q * width;
+                    const int c = col + 8 * (i >> 1), cc = c & cmask;
+                    const int q = cc >> qsh;
+                    const int pos = ((c - cc) >> (7 - wsh)) + cc - (q << qsh);   // (c - cc) is 0, or 64 for an up column
                     const uint32_t off = (uint32_t)((rank * a.M + m) * width + pos) * 4u;
                     st_async_f32(map_to_cluster_rank(recv + off, (uint32_t)q), acc[mt][i],
                                  map_to_cluster_rank(bar_recv, (uint32_t)q));
@@ -298,13 +304,13 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             if (!a.fuse) {
                 const int c_lo = rank * width;
                 for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
-                    const int m = idx / width, cc = idx - m * width;
+                    const int m = idx >> wsh, cc = idx - (m << wsh);
                     a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(slice_sum(m, cc));
                 }
             } else {
                 const int half_w = width >> 1;
                 for (int idx = threadIdx.x; idx < a.M * half_w; idx += kConsumerThreads) {
-                    const int m = idx / half_w, cc = idx - m * half_w;
+                    const int m = idx >> (wsh - 1), cc = idx - (m << (wsh - 1));
                     a.y[(size_t)m * (a.N / 2) + (size_t)p * 64 + rank * half_w + cc] =
                         __float2half_rn(silu_mul(slice_sum(m, cc), slice_sum(m, half_w + cc)));
                 }

@@ -153,11 +153,7 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     const int t0 = sk_range_begin(T, C, c), t1 = sk_range_begin(T, C, c + 1);
     const int stages = a.stages;
     __shared__ int s_last;
-    // this kernel has no fused gate/up epilogue: a layer tiled for one is refused by every CTA before any barrier exists
-    if (__ldg(&a.trailer->flags) & kFormatGateUp) {
-        if (threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
-        return;
-    }
+    const uint32_t flags = __ldg(&a.trailer->flags);   // needed by the consumers only; asked for first to hide the round trip
 
     if (threadIdx.x == kConsumerThreads) {
         for (int s = 0; s < stages; ++s) {
@@ -207,7 +203,10 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     }
 
     // -------------------------------------------------------------------- consumer warps
-    const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // weights-side data: no need to wait
+    const uint32_t z_add = flags & kFormatZerosMinusOne;   // weights-side data: no need to wait
+    // this kernel has no fused gate/up epilogue: a layer tiled for one is computed but not stored, and reported
+    const bool layout_ok = (flags & kFormatGateUp) == 0;
+    if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
     pdl_wait();
     const int g = lane >> 2, t4 = lane & 3;
     const int r = token_row_of_slot(g);
@@ -255,7 +254,7 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
-                        if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
+                        if (m < a.M && layout_ok) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
                     }
             } else {
                 const int slot = (p == first_panel) ? 0 : 1;
@@ -300,7 +299,7 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
                             for (int u = 0; u < 8; ++u) sum += v[u];
                         }
                         const int m = idx / kPanel, cc_col = idx % kPanel;
-                        a.y[(size_t)m * a.N + (size_t)p * kPanel + cc_col] = __float2half_rn(sum);
+                        if (layout_ok) a.y[(size_t)m * a.N + (size_t)p * kPanel + cc_col] = __float2half_rn(sum);
                     }
                     if (threadIdx.x == 0) a.tickets[p] = 0;   // ready for the next launch
                 }

@@ -181,6 +181,9 @@ __global__ void __launch_bounds__(umma_threads(TOK, NP, SETS), (NP > 1 || TOK > 
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];
+    // the layer's format flags are needed by the dequant warps only: requested first, so that the round trip to HBM
+    // hides behind the set-up
+    const uint32_t flags = __ldg(&a.trailer->flags);
     constexpr int kStage = umma_slot_bytes(TOK, NP);
     // ring slot = BPS K64 blocks: [x tile of each block][W blocks of each panel]
     constexpr int BPS = umma_blocks_per_slot(TOK);
@@ -237,9 +240,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     tc_fence_after_sync();
     const uint32_t tmem_base = lds32(tmem_slot);
     pdl_launch_dependents();
-    // a layer tiled for the fused gate/up epilogue must be used with it, and only with it (else: nothing is stored)
-    const bool layout_ok = ((__ldg(&a.trailer->flags) & kFormatGateUp) != 0) == (a.fuse != 0);
-    if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
+    bool layout_ok = true;   // set by the dequant warps; the producer and the MMA issuers must not wait for the trailer
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (one thread)
@@ -294,31 +295,45 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
             // itself: the dequant warps did before they wrote the A stage, and their a_full arrival orders it.
             // With one issuer it takes the blocks in order; with two, issuer t takes the blocks of dequant set t
             // (K groups t, t + SETS, ...) and accumulates them in its own tensor-memory columns.
-            const int t = warp - 1;
+            const int t = ISS == 1 ? 0 : warp - 1;          // a constant for the single issuer: nothing to compute per MMA
             const int b_begin = ISS == 1 ? 0 : 2 * t;
-            int b = b_begin;
-            int s = (b / BPS) % NS;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(t * TOK);
             bool ok = true;
-            while (b < NB && ok) {
-                const int sa = b % NA;
-                const uint32_t pha = (uint32_t)(b / NA) & 1u;
+            // one block: wait for its A stage(s), four MMAs per panel, one commit (every extra instruction of this
+            // thread shows in the prefill rate, so the bookkeeping below is kept incremental)
+            auto issue_block = [&](int b, int s, int sa, uint32_t pha) {
                 const uint64_t bdesc = umma_desc_k_major_sw128(ring + s * kStage + (b % BPS) * kXTile);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
                     ok = mbar_wait(bar_afull + 8 * (j * NA + sa), pha);
-                    if (!ok) break;
+                    if (!ok) return;
                     tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
-                        umma_f16_ts(tmem_base + (j * ISS + t) * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
+                        umma_f16_ts(d_tmem + j * ISS * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
                                     bdesc + (uint64_t)(kk * 2), idesc, (uint32_t)(b != b_begin || kk != 0));
                 }
-                if (!ok) break;
                 umma_commit(bar_done + 8 * (b & (kUmmaDoneRing - 1)));     // this block's A stage(s) and x tile may be overwritten
-                const int step = ISS == 1 ? 1 : ((b & 1) ? 2 * SETS - 1 : 1);   // to this issuer's next block
-                s += (b + step) / BPS - b / BPS;                            // and to that block's ring slot
-                while (s >= NS) s -= NS;
-                b += step;
+            };
+            if (ISS == 1) {
+                int s = 0, sa = 0;
+                uint32_t pha = 0;
+                for (int b = 0; b < NB && ok; ++b) {
+                    issue_block(b, s, sa, pha);
+                    if ((b % BPS) == BPS - 1 && ++s == NS) s = 0;
+                    if (++sa == NA) { sa = 0; pha ^= 1u; }
+                }
+            } else {
+                // the blocks of dequant set t: K groups t, t + SETS, ...; A stage b mod NA, filled for the (b / NA)-th time
+                int b = b_begin;
+                int s = (b / BPS) % NS;
+                while (b < NB && ok) {
+                    issue_block(b, s, b % NA, (uint32_t)(b / NA) & 1u);
+                    const int step = (b & 1) ? 2 * SETS - 1 : 1;   // to this issuer's next block
+                    s += (b + step) / BPS - b / BPS;                // and to that block's ring slot
+                    while (s >= NS) s -= NS;
+                    b += step;
+                }
             }
             if (b_begin < NB) umma_commit(bar_dfull);
             else mbar_arrive(bar_dfull);            // this issuer had no block
@@ -341,7 +356,6 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // A 128-row item holds SUB quantisation groups (128 / group_size), each with its own scales and zeros.
         const uint8_t *s_gl = a.scales + ((size_t)p * a.G + g0) * (SUB * kItemSBytes) + (16 * u + 2 * g + h) * 2;
         const uint8_t *z_gl = a.qzeros + ((size_t)p * a.G + g0) * (SUB * kItemZBytes) + 8 * u + g;
-        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // stored zero points one too small
         auto load_sz = [&](int gg, uint32_t (&sc)[SUB], uint32_t (&zb)[SUB]) {
             // through L2 only: this kernel may start while its predecessor still runs, and the buffers may have been
             // rewritten since an earlier kernel left lines of them in this SM's L1
@@ -355,6 +369,11 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
 #pragma unroll
         for (int sub = 0; sub < SUB; ++sub) sc_next[sub] = zb_next[sub] = 0;
         if (2 * set < NB) load_sz(set, sc_next, zb_next);
+        // (the format flags are looked at only now, with the first scales and zeros already on their way)
+        const uint32_t z_add = flags & kFormatZerosMinusOne;   // stored zero points one too small
+        // a layer tiled for the fused gate/up epilogue must be used with it, and only with it (else: nothing is stored)
+        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0);
+        if (!layout_ok && threadIdx.x == 32 * kFirstDq) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
         // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1; block b lives in ring refill b / BPS
         int b = 2 * set;

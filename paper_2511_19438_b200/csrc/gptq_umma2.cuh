@@ -87,11 +87,7 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
     const int mt = pair / ptiles, p = (pair - mt * ptiles) * 2 + rank;   // this CTA's weight panel
     const int m0 = mt * kUmma2Tok;
     const int NB = a.K / kUmmaBlockK;
-    // this kernel has no fused gate/up epilogue: a layer tiled for one is refused by every CTA before any barrier exists
-    if (__ldg(&a.trailer->flags) & kFormatGateUp) {
-        if (threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
-        return;
-    }
+    const uint32_t flags = __ldg(&a.trailer->flags);   // needed by the dequant warps only; asked for first to hide the round trip
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(bar_full + 8 * s, 1);
@@ -200,7 +196,10 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         int s = set % NS, sa = b % NA;
         uint32_t ph = (uint32_t)(set / NS) & 1u;
         uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
-        const uint32_t z_add = __ldg(&a.trailer->flags) & kFormatZerosMinusOne;   // stored zero points one too small
+        const uint32_t z_add = flags & kFormatZerosMinusOne;   // stored zero points one too small
+        // this kernel has no fused gate/up epilogue: a layer tiled for one is multiplied but not stored, and reported
+        const bool layout_ok = (flags & kFormatGateUp) == 0;
+        if (!layout_ok && threadIdx.x == 64) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {
             const uint32_t st = ring + s * kStage;
@@ -264,6 +263,7 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         pdl_wait();
         ok = __all_sync(0xffffffffu, ok && mbar_wait(bar_dfull, 0));
         if (ok) tc_fence_after_sync();
+        ok = ok && layout_ok;
         {
             // as in the single-CTA kernel: each set's four warps turn a 32-token chunk around through the idle ring
             // and write whole 128-byte lines of y; every warp takes part in the named barriers
