@@ -132,7 +132,8 @@ int gptq_set_workspace(void *ptr, size_t bytes);
 /* The GPTQ linear layer of Sections 1 and 3 (the product all three of the paper's optimisations serve; Section
  * 4.4's last paragraph fixes what "the same result" means: equal up to summation order).
  * y fp16[M,N] = x fp16[M,K] . dequant(W).  qweight/qzeros/scales are the REPACKED buffers from
- * gptq_repack; with act_order != 0, g_idx is gptq_repack's perm_out (else it may be NULL).
+ * gptq_repack; with act_order != 0, g_idx is gptq_repack's perm_out (16-byte aligned like every other pointer, else
+ * GPTQ_ERR_ALIGN; without act-order it may be NULL).
  * fp32 accumulation, one round-to-nearest-even conversion to fp16.  Any M >= 1.  Up to 16 rows the
  * weights enter the MMA as exact integers q - z and the scale multiplies fp32 group sums; above
  * that each scaled weight is rounded to fp16 once before the MMA.

@@ -371,6 +371,7 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     if (st) return st;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
         return GPTQ_ERR_ALIGN;
+    if (act_order && !aligned16(g_idx)) return GPTQ_ERR_ALIGN;
     st = check_fast_path(N, K, group_size);
     if (st) return st;
 
@@ -476,6 +477,7 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
     if (st) return st;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
         return GPTQ_ERR_ALIGN;
+    if (act_order && !aligned16(g_idx)) return GPTQ_ERR_ALIGN;
     st = check_fast_path(N, K, group_size);
     if (st) return st;
     if (group_size != kGroup) return GPTQ_ERR_UNSUPPORTED;   // the stream-K kernel is built for group size 128 only

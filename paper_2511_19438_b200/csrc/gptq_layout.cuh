@@ -249,8 +249,55 @@ __global__ void gather_x_kernel(const __half *__restrict__ x, const int32_t *__r
     for (int m = blockIdx.y; m < M; m += gridDim.y) x_out[(size_t)m * K + i] = x[(size_t)m * K + src];
 }
 
+// The same for many token rows: a block stages kGatherRows whole rows of x in shared memory with coalesced 16-byte
+// loads, then every thread picks eight permuted elements per row from there and writes them with one 16-byte store.
+// (The element-per-thread kernel above reads 2 bytes per 32-byte sector; from a few dozen rows on that costs more than
+// the copy itself.)
+constexpr int kGatherRows = 4;
+__global__ void __launch_bounds__(256)
+gather_x_rows_kernel(const __half *__restrict__ x, const int32_t *__restrict__ perm, __half *__restrict__ x_out, int M, int K)
+{
+    extern __shared__ uint4 gather_rows[];     // kGatherRows x K halves
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m0 = blockIdx.x * kGatherRows;
+    const int nrows = (M - m0) < kGatherRows ? (M - m0) : kGatherRows;
+    const int chunks = K / 8;                  // 16-byte chunks per row
+    const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)m0 * K);   // the rows are adjacent in memory
+    for (int i = threadIdx.x; i < nrows * chunks; i += blockDim.x) gather_rows[i] = src[i];
+    __syncthreads();
+    const __half *rows = reinterpret_cast<const __half *>(gather_rows);
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        const int4 pa = reinterpret_cast<const int4 *>(perm)[2 * c], pb = reinterpret_cast<const int4 *>(perm)[2 * c + 1];
+        const int idx[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+        for (int r = 0; r < nrows; ++r) {
+            __align__(16) __half v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = rows[(size_t)r * K + idx[e]];
+            *reinterpret_cast<uint4 *>(x_out + (size_t)(m0 + r) * K + 8 * c) = *reinterpret_cast<const uint4 *>(v);
+        }
+    }
+}
+
 int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, int K, cudaStream_t s)
 {
+    const size_t rows_smem = (size_t)kGatherRows * K * sizeof(__half);
+    if (M >= 32 && K % 8 == 0 && rows_smem <= 200 * 1024) {
+        static int configured_smem[64] = {};
+        const int cfg_st = ensure_dynamic_smem((const void *)gather_x_rows_kernel, configured_smem, (int)rows_smem);
+        if (cfg_st) return cfg_st;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)((M + kGatherRows - 1) / kGatherRows));
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = rows_smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return record_cuda_error(cudaLaunchKernelEx(&cfg, gather_x_rows_kernel, x, perm, x_out, M, K));
+    }
     const int T = 256;
     // launched as a programmatic dependent of the kernel before it: its CTAs become resident while that kernel still
     // runs, and griddepcontrol.wait holds the copy back until that kernel (which may write x, and may still be reading

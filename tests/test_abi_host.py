@@ -56,6 +56,7 @@ def test_gemm_validation_order_without_gpu():
     assert call(group_size=0) == B.GPTQ_ERR_SHAPE
     assert call(x=A16 + 8) == B.GPTQ_ERR_ALIGN
     assert call(qw=A16 + 4) == B.GPTQ_ERR_ALIGN
+    assert call(act_order=1, gi=A16 + 4) == B.GPTQ_ERR_ALIGN   # perm_out is read 16 bytes at a time
     assert call(group_size=16) == B.GPTQ_ERR_UNSUPPORTED   # 128, 64 and 32 have a tiled layout
     assert call(group_size=256) == B.GPTQ_ERR_UNSUPPORTED
     assert call(N=4096 + 64) == B.GPTQ_ERR_UNSUPPORTED
