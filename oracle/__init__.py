@@ -38,7 +38,8 @@ def _load():
         lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
         lib.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
-                     "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64"):
+                     "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64",
+                     "oracle_add_bias_residual_f64"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -156,4 +157,15 @@ def silu_mul_f64(y: np.ndarray) -> np.ndarray:
     assert N % 2 == 0
     out = np.empty((M, N // 2), dtype=np.float64)
     _load().oracle_silu_mul_f64(_p(y), ctypes.c_int(M), ctypes.c_int(N // 2), _p(out))
+    return out
+
+
+def add_bias_residual_f64(y: np.ndarray, bias: np.ndarray | None, residual: np.ndarray | None) -> np.ndarray:
+    """out[M, N] = y + bias[n] + residual[m, n] in fp64 (bias fp16 [N], residual fp16 [M, N]; either may be None)."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    M, N = y.shape
+    b = None if bias is None else _f16(bias, (N,))
+    r = None if residual is None else _f16(residual, (M, N))
+    out = np.empty((M, N), dtype=np.float64)
+    _load().oracle_add_bias_residual_f64(_p(y), _p(b), _p(r), ctypes.c_int(M), ctypes.c_int(N), _p(out))
     return out

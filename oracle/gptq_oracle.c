@@ -208,3 +208,21 @@ void oracle_silu_mul_f64(const double *y, int M, int I, double *out)
             out[(size_t)m * I + i] = g / (1.0 + exp(-g)) * u;
         }
 }
+
+/* ---- the additive neighbours of a projection -------------------------------------------------
+ * A linear layer of the served models may carry a bias (one fp16 value per output column), and the o and down
+ * projections of a Llama-class block (Section 4.1) are followed by the residual add h = h + proj(...).  The paper's
+ * kernels stop at the matmul; the library can fuse both additions into the matmul's epilogue, and this is their
+ * definition: out[m][n] = y[m][n] + bias[n] + residual[m][n] in fp64, y the fp64 matmul result [M, N]; bias (fp16
+ * bits, [N]) and residual (fp16 bits, [M, N]) may each be NULL (then it adds nothing). */
+void oracle_add_bias_residual_f64(const double *y, const uint16_t *bias, const uint16_t *residual, int M, int N,
+                                  double *out)
+{
+    for (int m = 0; m < M; m++)
+        for (int n = 0; n < N; n++) {
+            double v = y[(size_t)m * N + n];
+            if (bias) v += (double)oracle_half_to_float(bias[n]);
+            if (residual) v += (double)oracle_half_to_float(residual[(size_t)m * N + n]);
+            out[(size_t)m * N + n] = v;
+        }
+}

@@ -346,3 +346,32 @@ def test_silu_mul_against_the_tanh_form_and_its_symmetry():
     assert np.allclose(out - neg, g * u, rtol=1e-13, atol=1e-13)                           # silu(t) - silu(-t) = t
     # gate columns first, up columns second: swapping the halves is a different function
     assert not np.allclose(out, oracle.silu_mul_f64(np.concatenate([u, g], axis=1)))
+
+
+# ------------------------------------------------------------------------------- bias and residual
+def test_add_bias_residual_small_integers_are_exact_and_oriented():
+    """Small integers are exact in fp16 and fp64, so the sum has one right answer; a non-square case with a bias that
+    counts columns and a residual that counts rows shows which operand goes along which axis."""
+    M, N = 3, 5
+    y = np.arange(M * N, dtype=np.float64).reshape(M, N) * 0.25
+    bias = np.arange(N).astype(np.float16)                                  # bias[n] = n
+    resid = np.repeat(np.arange(M)[:, None] * 100, N, axis=1).astype(np.float16)   # residual[m, n] = 100 m
+    out = oracle.add_bias_residual_f64(y, bias, resid)
+    for m in range(M):
+        for n in range(N):
+            assert out[m, n] == 0.25 * (m * N + n) + n + 100 * m
+    assert np.array_equal(oracle.add_bias_residual_f64(y, None, None), y)
+    assert np.array_equal(oracle.add_bias_residual_f64(y, bias, None) - y, np.tile(np.arange(N, dtype=np.float64), (M, 1)))
+    assert np.array_equal(oracle.add_bias_residual_f64(y, None, resid) - y, resid.astype(np.float64))
+
+
+def test_add_bias_residual_reads_fp16_exactly_and_adds_in_double():
+    """The operands are the fp16 values themselves (0.1 is not representable: its fp16 neighbour is what is added), and
+    the sum keeps what a single-precision sum would lose."""
+    y = np.array([[1e8, -3.0]])
+    bias = np.array([0.1, 65504.0], np.float16)
+    resid = np.array([[1.0, 2.0 ** -24]], np.float16)                       # the smallest fp16 subnormal
+    out = oracle.add_bias_residual_f64(y, bias, resid)
+    assert out[0, 0] == 1e8 + 0.0999755859375 + 1.0                         # fp16(0.1) = 0.0999755859375; exact in fp64
+    assert out[0, 1] == -3.0 + 65504.0 + 2.0 ** -24
+    assert np.float32(1e8) + np.float32(0.0999755859375) == np.float32(1e8)   # fp32 would have dropped the bias
