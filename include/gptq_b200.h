@@ -152,6 +152,17 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
 
+/* (No counterpart in the paper: additions fused into the epilogue of the product of Sections 1 and 3.)
+ * y fp16[M,N] = x . dequant(W) + bias[n] + residual[m][n]: the bias of a projection (fp16 [N]) and the residual add
+ * that follows the o and down projections of a Llama block (fp16 [M,N]), joined to the fp32 sums before the one
+ * rounding to fp16.  Either pointer may be NULL (adds nothing); both NULL is gptq_gemm.  residual may be y itself
+ * (h += proj(x)): each element is read and then written by the same thread.  Both must be 16-byte aligned and are
+ * read after earlier work on the stream has finished.  Other arguments, layouts, accuracy and errors as for
+ * gptq_gemm; a layer tiled with GPTQ_FORMAT_GATE_UP is refused the same way.  The CTA-pair switch does not apply. */
+int gptq_gemm_bias_residual(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                            const int32_t *g_idx, const void *bias, const void *residual, void *y,
+                            int M, int N, int K, int group_size, int act_order, void *stream);
+
 /* (No counterpart in the paper: an epilogue fused into the product of Sections 1 and 3.)
  * out fp16[M, N / 2] = silu(y[:, :N/2]) * y[:, N/2:], silu(g) = g / (1 + exp(-g)), for y = x . dequant(W) of a layer
  * repacked with GPTQ_FORMAT_GATE_UP: the activation of a Llama MLP block applied before the product leaves the chip,

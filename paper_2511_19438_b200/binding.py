@@ -70,6 +70,7 @@ _SIGNATURES = {
     "gptq_set_workspace": (_i, [_vp, _sz]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_silu_mul": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_bias_residual": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_set_cta_pairs": (_i, [_i]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
@@ -191,6 +192,12 @@ def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_st
 def gptq_gemm_silu_mul(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, stream=None) -> int:
     return _lib.gptq_gemm_silu_mul(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(out), M, N,
                                    K, group_size, int(act_order), _stream(stream))
+
+
+def gptq_gemm_bias_residual(x, qweight, qzeros, scales, g_idx, bias, residual, y, M, N, K, group_size, act_order,
+                            stream=None) -> int:
+    return _lib.gptq_gemm_bias_residual(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(bias),
+                                        _ptr(residual), _ptr(y), M, N, K, group_size, int(act_order), _stream(stream))
 
 
 def gptq_gemm_noalloc(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:

@@ -364,7 +364,8 @@ int gptq_set_workspace(void *ptr, size_t bytes)
 
 // y = x W (fuse == 0, y is [M, N]) or silu(gate) * up of y's column halves (fuse == 1, y is [M, N / 2])
 static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
-                         void *y, int M, int N, int K, int group_size, int act_order, int fuse, void *stream)
+                         void *y, int M, int N, int K, int group_size, int act_order, int fuse, const void *bias,
+                         const void *residual, void *stream)
 {
     if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(M, N, K, group_size);
@@ -372,6 +373,7 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
         return GPTQ_ERR_ALIGN;
     if (act_order && !aligned16(g_idx)) return GPTQ_ERR_ALIGN;
+    if (!aligned16(bias) || !aligned16(residual)) return GPTQ_ERR_ALIGN;     // a null pointer passes
     st = check_fast_path(N, K, group_size);
     if (st) return st;
 
@@ -380,6 +382,7 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     if (st) return st;
     cudaStream_t s = (cudaStream_t)stream;
     const __half *xin = (const __half *)x;
+    const bool extras = bias != nullptr || residual != nullptr;
     if (act_order) {
         Workspace ws;
         {
@@ -394,19 +397,21 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     }
     const size_t ldy = fuse ? (size_t)N / 2 : (size_t)N;
     if (M >= kUmmaMinTokens) {
-        if (!fuse && g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
+        if (!fuse && !extras && g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
             const Umma2Plan p2 = plan_umma2(M, N, K);
             return launch_umma2(xin, qweight, qzeros, scales, (__half *)y, M, N, K, p2, s);
         }
         // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
-        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, fuse, s);
+        return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, fuse, (const __half *)bias,
+                           (const __half *)residual, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
         const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sms);
         st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * ldy, rows, N, K,
-                           pl, fuse, s);
+                           pl, fuse, (const __half *)bias,
+                           residual ? (const __half *)residual + (size_t)m0 * N : nullptr, s);
         if (st) return st;
     }
     return GPTQ_OK;
@@ -417,14 +422,21 @@ extern "C" {
 int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
               void *y, int M, int N, int K, int group_size, int act_order, void *stream)
 {
-    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, stream);
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, nullptr, nullptr, stream);
+}
+
+int gptq_gemm_bias_residual(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                            const int32_t *g_idx, const void *bias, const void *residual, void *y, int M, int N, int K,
+                            int group_size, int act_order, void *stream)
+{
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, bias, residual, stream);
 }
 
 int gptq_gemm_silu_mul(const void *x, const void *qweight, const void *qzeros, const void *scales,
                        const int32_t *g_idx, void *out, int M, int N, int K, int group_size, int act_order,
                        void *stream)
 {
-    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, stream);
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, nullptr, nullptr, stream);
 }
 
 int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, const void *scales,

@@ -251,8 +251,8 @@ __global__ void gather_x_kernel(const __half *__restrict__ x, const int32_t *__r
 
 // The same for many token rows: a block stages kGatherRows whole rows of x in shared memory with coalesced 16-byte
 // loads, then every thread picks eight permuted elements per row from there and writes them with one 16-byte store.
-// (The element-per-thread kernel above reads 2 bytes per 32-byte sector; from a few dozen rows on that costs more than
-// the copy itself.)
+// (The element-per-thread kernel above reads 2 bytes per 32-byte sector; with thousands of rows that costs several
+// times the copy itself.)
 constexpr int kGatherRows = 4;
 __global__ void __launch_bounds__(256)
 gather_x_rows_kernel(const __half *__restrict__ x, const int32_t *__restrict__ perm, __half *__restrict__ x_out, int M, int K)
@@ -282,7 +282,9 @@ gather_x_rows_kernel(const __half *__restrict__ x, const int32_t *__restrict__ p
 int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, int K, cudaStream_t s)
 {
     const size_t rows_smem = (size_t)kGatherRows * K * sizeof(__half);
-    if (M >= 32 && K % 8 == 0 && rows_smem <= 200 * 1024) {
+    // measured on the 7B shapes: pays from about a thousand rows on (M = 4096: 17-57 us instead of 48-250), from 512
+    // rows on the long-K layers; below that its few blocks leave most SMs idle and the element-per-thread kernel wins
+    if ((M >= 1024 || (M >= 512 && K >= 8192)) && K % 8 == 0 && rows_smem <= 200 * 1024) {
         static int configured_smem[64] = {};
         const int cfg_st = ensure_dynamic_smem((const void *)gather_x_rows_kernel, configured_smem, (int)rows_smem);
         if (cfg_st) return cfg_st;

@@ -92,6 +92,8 @@ struct SplitKArgs {
     int stages;
     const TiledTrailer *trailer;   // behind the tiled zero points
     int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
+    const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
+    const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
 };
 
 // silu(g) * u in fp32
@@ -223,6 +225,15 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     // accumulator i of tile mt: weight column col + 8*(i>>1), token slot 2*t4 + (i&1)
     const int col = warp * 16 + g;
     const int m_lo = token_row_of_slot(2 * t4), m_hi = token_row_of_slot(2 * t4 + 1);
+    // what the epilogue adds to the fp32 sum of output (m, n) before the one rounding: bias[n] + residual[m][n]
+    // (read after griddepcontrol.wait: an earlier kernel may have produced them; the thread that reads an element of
+    // the residual is the one that writes the same element of y, so the two may be one buffer)
+    auto addend = [&](int m, int n) {
+        float v = 0.f;
+        if (a.bias) v += __half2float(a.bias[n]);
+        if (a.residual) v += __half2float(a.residual[(size_t)m * a.N + n]);
+        return v;
+    };
     if (S == 1) {
         if (warp < kConsumerWarps && layout_ok) {
             if (!a.fuse) {
@@ -232,7 +243,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
-                        if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i]);
+                        if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i] + addend(m, p * kPanel + col + 8 * (i >> 1)));
                     }
             } else {
                 // warps 4-7 hold the up columns of the gate columns of warps 0-3: hand them over through the
@@ -305,7 +316,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 const int c_lo = rank * width;
                 for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
                     const int m = idx >> wsh, cc = idx - (m << wsh);
-                    a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(slice_sum(m, cc));
+                    a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(slice_sum(m, cc) + addend(m, p * kPanel + c_lo + cc));
                 }
             } else {
                 const int half_w = width >> 1;
@@ -393,7 +404,8 @@ static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, co
 }
 
 int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
-                  int M, int N, int K, const SplitKPlan &plan, int fuse, cudaStream_t s)
+                  int M, int N, int K, const SplitKPlan &plan, int fuse, const __half *bias, const __half *residual,
+                  cudaStream_t s)
 {
     SplitKArgs args;
     args.qweight = (const uint8_t *)qweight;
@@ -407,6 +419,8 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.S = plan.S;
     args.stages = plan.stages;
     args.fuse = fuse;
+    args.bias = bias;
+    args.residual = residual;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;

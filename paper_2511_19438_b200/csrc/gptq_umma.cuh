@@ -157,6 +157,8 @@ struct UmmaArgs {
     int stages;             // shared-memory ring depth
     const TiledTrailer *trailer;   // behind the tiled zero points
     int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
+    const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
+    const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
 };
 
 // K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
@@ -483,6 +485,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 if (ok) {
                     uint32_t r[32];
                     load_acc(c0, r);
+                    if (a.bias || a.residual) {
+                        // bias[column] + residual[token][column] join the fp32 sum before the one rounding; the 32 lanes
+                        // of a warp read 32 neighbouring columns of one token row per load
+                        const size_t ncol = (size_t)p * kPanel + n;
+                        const float bv = a.bias ? __half2float(a.bias[ncol]) : 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int m = m0 + c0 + i;
+                            float v = __uint_as_float(r[i]) + bv;
+                            if (a.residual && m < a.M) v += __half2float(a.residual[(size_t)m * a.N + ncol]);
+                            r[i] = __float_as_uint(v);
+                        }
+                    }
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
                         sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
@@ -575,7 +590,21 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 const int w4 = width >> 2;      // four columns (16 bytes) per thread and step
                 for (int idx = threadIdx.x - 32 * kFirstDq; idx < rows * w4; idx += 128 * NP * SETS) {
                     const int m = idx / w4, cc = c_lo + 4 * (idx - m * w4);
-                    store4(a.y + (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc, sum4(m, cc));
+                    const size_t at = (size_t)(m0 + m) * a.N + (size_t)p * kPanel + cc;
+                    float4 v = sum4(m, cc);
+                    if (a.bias) {
+                        const uint2 b = *reinterpret_cast<const uint2 *>(a.bias + (size_t)p * kPanel + cc);
+                        const float2 b0 = __half22float2(*reinterpret_cast<const __half2 *>(&b.x));
+                        const float2 b1 = __half22float2(*reinterpret_cast<const __half2 *>(&b.y));
+                        v.x += b0.x, v.y += b0.y, v.z += b1.x, v.w += b1.y;
+                    }
+                    if (a.residual) {
+                        const uint2 q = *reinterpret_cast<const uint2 *>(a.residual + at);
+                        const float2 q0 = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+                        const float2 q1 = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+                        v.x += q0.x, v.y += q0.y, v.z += q1.x, v.w += q1.y;
+                    }
+                    store4(a.y + at, v);
                 }
             } else {
                 // this CTA finishes gate columns [rank width / 2, ...) of the tile and the matching up columns 64 further
@@ -730,7 +759,8 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
 }
 
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
-                int K, int group_size, const UmmaPlan &plan, int fuse, cudaStream_t s)
+                int K, int group_size, const UmmaPlan &plan, int fuse, const __half *bias, const __half *residual,
+                cudaStream_t s)
 {
     UmmaArgs args;
     args.scales = (const uint8_t *)scales;
@@ -743,6 +773,8 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.S = plan.S;
     args.stages = plan.stages;
     args.fuse = fuse;
+    args.bias = bias;
+    args.residual = residual;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, group_size));
     const int sub = kGroup / group_size;
     if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;

@@ -88,3 +88,14 @@ def gemm_silu_mul(x: torch.Tensor, D: DeviceLinear, out: torch.Tensor | None = N
     B.check(B.gptq_gemm_silu_mul(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, out, M, D.N, D.K, D.group_size,
                                  D.act_order, stream), "gptq_gemm_silu_mul")
     return out
+
+
+def gemm_bias_residual(x: torch.Tensor, D: DeviceLinear, bias: torch.Tensor | None, residual: torch.Tensor | None,
+                       y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """y = x . dequant(W) + bias + residual through gptq_gemm_bias_residual (y may be the residual buffer)."""
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, D.N), dtype=torch.float16, device=x.device)
+    B.check(B.gptq_gemm_bias_residual(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, bias, residual, y, M, D.N, D.K,
+                                      D.group_size, D.act_order, stream), "gptq_gemm_bias_residual")
+    return y

@@ -74,6 +74,9 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_repack_format(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, 4, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_dequant_f32_format(A16, A16, A16, None, A16, 128, 128, 128, 0, 0, B.GPTQ_FORMAT_GATE_UP, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_gemm_silu_mul(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_bias_residual(A16, A16, A16, A16, None, A16, A16, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_bias_residual(A16, A16, A16, A16, None, A16 + 2, None, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_ALIGN
+    assert B.gptq_gemm_bias_residual(A16, A16, A16, A16, None, None, A16 + 8, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_ALIGN
     assert B.gptq_gemm_silu_mul(A16, A16, A16, A16, None, A16, 1, 192, 128, 128, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack_bytes(1, 256, 512, 32, 0) == (512 // 32) * 256 // 2 + 16    # zero points + format trailer
     assert B.gptq_plan_noalloc(4, 128, 512, 64, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED

@@ -489,6 +489,74 @@ def test_variants_unsupported_entry_points():
     assert torch.count_nonzero(y) == 0
 
 
+# ------------------------------------------------------------------------------- bias and residual in the epilogue
+def check_bias_residual(L, M, ws, use_bias, use_resid, in_place=False):
+    K, N = L.K, L.N
+    x_np = wl.make_x(M, K, wl.seed_for("br-x", M, K))
+    r = np.random.default_rng(wl.seed_for("br", M, N))
+    bias_np = (r.normal(0, 2, N)).astype(np.float16) if use_bias else None
+    resid_np = (r.normal(0, 8, (M, N))).astype(np.float16) if use_resid else None
+    D = H.upload_and_repack(L)
+    ws.ensure_for(M, D)
+    bias = H.to_device(bias_np) if use_bias else None
+    resid = H.to_device(resid_np) if use_resid else None
+    y = H.gemm_bias_residual(H.to_device(x_np), D, bias, resid, y=resid if in_place else None)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
+    want = oracle.add_bias_residual_f64(y64, bias_np, resid_np)
+    got = y.cpu().numpy().astype(np.float64)
+    err = np.abs(got - want)
+    # the matmul part within its stated bar, the additions exact in fp32 up to the one final rounding of the sum
+    loose = 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64) + 2.0 ** -11 * np.abs(want)
+    assert np.all(np.isfinite(got)) and np.all(err <= loose), f"{int((err > loose).sum())} violations, max {err.max():.3e}"
+    if M <= 16:   # exact integer MMA inputs, fp32 sums: only the final rounding and the summation order show
+        tight = 1e-4 * math.sqrt(K / 4096) + 2.0 ** -11 * np.abs(want) + 2.0 ** -22 * (np.abs(y64) + np.abs(want))
+        assert np.all(err <= tight), f"{int((err > tight).sum())} violations of the tight bound, max {err.max():.3e}"
+    if not in_place and use_resid:
+        assert np.array_equal(resid.cpu().numpy(), resid_np)            # the residual itself is only read
+
+
+@pytest.mark.parametrize("use_bias,use_resid", [(True, True), (False, True), (True, False)])
+@pytest.mark.parametrize("M", [1, 8, 16, 20, 64, 130, 300])
+def test_bias_residual_small_layer(M, use_bias, use_resid, ws):
+    """K split over a cluster in every kernel family (the owner of a column slice adds bias and residual to the cluster
+    sum), act-order on."""
+    L = wl.make_linear(1024, 384, seed=wl.seed_for("br-small"), act_order=True)
+    check_bias_residual(L, M, ws, use_bias, use_resid)
+
+
+@pytest.mark.parametrize("M", [1, 16, 40, 2040])
+def test_bias_residual_in_place_on_down_projection(M, ws):
+    """h += down(x) on the 7B down projection: y and the residual are one buffer; also a shape whose CTAs own whole
+    panels at the larger M (no cluster exchange)."""
+    K, N = wl.SHAPES_7B["down"]
+    L = wl.make_linear(K, N, seed=wl.seed_for("br-down"))
+    check_bias_residual(L, M, ws, use_bias=False, use_resid=True, in_place=True)
+
+
+def test_bias_residual_wide_layer_without_split(ws):
+    K, N = wl.SHAPES_7B["gate_up"]                       # more panels than SMs: S = 1 in the mma.sync kernel
+    L = wl.make_linear(K, N, seed=wl.seed_for("br-wide"))
+    for M in (2, 16):
+        check_bias_residual(L, M, ws, True, True)
+
+
+def test_bias_residual_null_operands_and_refusals(ws):
+    """Both operands NULL is gptq_gemm bit for bit; misaligned operands and an interleaved layer are refused."""
+    K, N, M = 512, 256, 6
+    L = wl.make_linear(K, N, seed=wl.seed_for("br-null"))
+    D = H.upload_and_repack(L)
+    x = H.to_device(wl.make_x(M, K, 2))
+    assert torch.equal(H.gemm_bias_residual(x, D, None, None), H.gemm(x, D))
+    bias = torch.zeros(N + 8, dtype=torch.float16, device="cuda")
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm_bias_residual(x, D.qweight_t, D.qzeros_t, D.scales_t, None, bias[1:], None, y, M, N, K, 128, 0) == B.GPTQ_ERR_ALIGN
+    D_gu = H.upload_and_repack(L, gate_up=True)
+    H.gemm_bias_residual(x, D_gu, bias[:N], None, y)
+    assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+    assert torch.count_nonzero(y) == 0
+
+
 # ------------------------------------------------------------------------------- fused gate/up epilogue
 def silu_mul_bound(y64: np.ndarray, K: int) -> np.ndarray:
     """What the stated matmul tolerance allows for out = silu(g) * u when g and u each carry an error of at most
