@@ -12,7 +12,8 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgptq_b200.so")
+# GPTQ_B200_LIB names another build of the same library (the timeline tool loads its instrumented build this way)
+LIB_PATH = os.environ.get("GPTQ_B200_LIB") or os.path.join(_HERE, "libgptq_b200.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -78,6 +79,8 @@ _SIGNATURES = {
     "gptq_gemm_host_batch": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_check_status": (_i, [_vp]),
     "gptq_selftest_wait_timeout": (_i, [ctypes.c_uint, _vp]),
+    "gptq_trace_reset": (_i, [_vp]),
+    "gptq_trace_read": (_i, [_vp, _i, _vp]),
     "gptq_plan": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_noalloc": (_i, [_i, _i, _i, _i, _i, _i, ctypes.POINTER(gptq_plan_t)]),
     "gptq_plan_cta_range": (_i, [_i, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]),
@@ -232,6 +235,18 @@ def gptq_check_status(stream=None) -> int:
 
 def gptq_selftest_wait_timeout(limit_us, stream=None) -> int:
     return _lib.gptq_selftest_wait_timeout(int(limit_us), _stream(stream))
+
+
+def gptq_trace_reset(stream=None) -> int:
+    return _lib.gptq_trace_reset(_stream(stream))
+
+
+def gptq_trace_read(max_rows: int = 64, stream=None):
+    """Returns (status or row count, rows) with rows a list of 8-tuples of ints (see the header)."""
+    buf = (ctypes.c_ulonglong * (8 * max_rows))()
+    n = _lib.gptq_trace_read(ctypes.cast(buf, ctypes.c_void_p), max_rows, _stream(stream))
+    rows = [tuple(buf[8 * i + j] for j in range(8)) for i in range(max(n, 0))]
+    return n, rows
 
 
 def plan_kernel_name(plan) -> str:

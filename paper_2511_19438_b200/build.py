@@ -31,16 +31,30 @@ def stale() -> bool:
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
+def _compile(out: str, extra, verbose: bool) -> str:
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = out + f".{os.getpid()}.tmp"
+    cmd = [nvcc] + NVCC_FLAGS + list(extra) + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+    subprocess.check_call(cmd)
+    os.replace(tmp, out)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not stale():
         return LIB
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + f".{os.getpid()}.tmp"
     extra = os.environ.get("GPTQ_NVCC_EXTRA", "").split()      # e.g. -DGPTQ_UMMA_MIN_TOKENS=17
-    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
-    subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    return _compile(LIB, extra, verbose)
+
+
+TIMELINE_LIB = os.path.join(HERE, "libgptq_b200_timeline.so")
+
+
+def build_timeline(force: bool = False) -> str:
+    """The same library with the launch timeline compiled in (-DGPTQ_TIMELINE), as a file of its own."""
+    if not force and os.path.exists(TIMELINE_LIB) and not any(os.path.getmtime(p) > os.path.getmtime(TIMELINE_LIB) for p in _deps()):
+        return TIMELINE_LIB
+    return _compile(TIMELINE_LIB, ["-DGPTQ_TIMELINE"], False)
 
 
 if __name__ == "__main__":

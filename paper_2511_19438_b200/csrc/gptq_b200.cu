@@ -24,6 +24,16 @@ int record_cuda_error(cudaError_t e)
     return GPTQ_ERR_CUDA;
 }
 
+int next_trace_slot()
+{
+#ifdef GPTQ_TIMELINE
+    static std::atomic<int> next{0};
+    return next.fetch_add(1) % kTraceLaunches;
+#else
+    return -1;
+#endif
+}
+
 int ensure_dynamic_smem(const void *kernel, int *configured, int smem_bytes)
 {
     static std::mutex mu;
@@ -622,6 +632,40 @@ int gptq_selftest_wait_timeout(unsigned int limit_us, void *stream)
     if (limit_us < 1 || limit_us > 1000000) return GPTQ_ERR_SHAPE;
     wait_selftest_kernel<<<1, 1, 0, (cudaStream_t)stream>>>((unsigned long long)limit_us * 1000ull);
     return record_cuda_error(cudaGetLastError());
+}
+
+int gptq_trace_reset(void *stream)
+{
+#ifdef GPTQ_TIMELINE
+    static TraceRow blank[kTraceLaunches];
+    for (int i = 0; i < kTraceLaunches; ++i) {
+        blank[i].first_entry = blank[i].first_weight_issue = blank[i].first_wait_done = blank[i].first_data = ~0ull;
+        blank[i].last_wait_done = blank[i].last_exit = blank[i].kernel_id = blank[i].ctas = 0;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyToSymbolAsync(g_trace, blank, sizeof(blank), 0, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    return record_cuda_error(e);
+#else
+    (void)stream;
+    return GPTQ_ERR_UNSUPPORTED;
+#endif
+}
+
+int gptq_trace_read(unsigned long long *rows_out, int max_rows, void *stream)
+{
+#ifdef GPTQ_TIMELINE
+    if (!rows_out || max_rows < 0) return GPTQ_ERR_NULL;
+    const int n = max_rows < kTraceLaunches ? max_rows : kTraceLaunches;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyFromSymbolAsync(rows_out, g_trace, (size_t)n * sizeof(TraceRow), 0, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    return n;
+#else
+    (void)rows_out; (void)max_rows; (void)stream;
+    return GPTQ_ERR_UNSUPPORTED;
+#endif
 }
 
 int gptq_check_status(void *stream)

@@ -162,6 +162,32 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// ---- launch timeline (compiled in with -DGPTQ_TIMELINE only) -----------------------------------
+// Every matmul launch of a timeline build takes the next of kTraceLaunches rows and its CTAs record, with %globaltimer
+// and 64-bit atomic min / max, when the grid's first CTA started, when the first weight copy was issued, when
+// griddepcontrol.wait first and last returned, when the first activation tile had landed and when the last CTA was
+// done.  gptq_trace_reset / gptq_trace_read move the rows; in a normal build the macros expand to nothing.
+constexpr int kTraceLaunches = 64;
+struct TraceRow {
+    unsigned long long first_entry, first_weight_issue, first_wait_done, last_wait_done, first_data, last_exit;
+    unsigned long long kernel_id, ctas;     // 1 = mma.sync kernel, 2 = tcgen05 kernel; grid size
+};
+#ifdef GPTQ_TIMELINE
+__device__ TraceRow g_trace[kTraceLaunches];
+#define GPTQ_TRACE_MIN(slot, field) \
+    do { if ((slot) >= 0) atomicMin(&g_trace[(slot)].field, (unsigned long long)global_timer_ns()); } while (0)
+#define GPTQ_TRACE_MAX(slot, field) \
+    do { if ((slot) >= 0) atomicMax(&g_trace[(slot)].field, (unsigned long long)global_timer_ns()); } while (0)
+#define GPTQ_TRACE_SET(slot, field, v) \
+    do { if ((slot) >= 0) g_trace[(slot)].field = (unsigned long long)(v); } while (0)
+#else
+#define GPTQ_TRACE_MIN(slot, field) do { } while (0)
+#define GPTQ_TRACE_MAX(slot, field) do { } while (0)
+#define GPTQ_TRACE_SET(slot, field, v) do { } while (0)
+#endif
+// the row the next launch takes (host side; -1 in a normal build)
+int next_trace_slot();
+
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __noinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, uint64_t limit_ns)
 {

@@ -94,6 +94,7 @@ struct SplitKArgs {
     int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
     const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
     const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
+    int trace_slot;         // row of the launch timeline, or -1
 };
 
 // silu(g) * u in fp32
@@ -120,6 +121,13 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     // the layer's format flags are needed late (first item, epilogue): ask for them first, so that the round trip to
     // HBM hides behind the set-up
     const uint32_t flags = __ldg(&a.trailer->flags);
+    if (threadIdx.x == 0) {
+        GPTQ_TRACE_MIN(a.trace_slot, first_entry);
+        if (blockIdx.x == 0) {
+            GPTQ_TRACE_SET(a.trace_slot, kernel_id, 1);
+            GPTQ_TRACE_SET(a.trace_slot, ctas, gridDim.x);
+        }
+    }
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar_full = smem_base;                  // stages x 8 B
     const uint32_t bar_empty = smem_base + 64;            // stages x 8 B
@@ -171,8 +179,11 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 bulk_g2s_hint(dst + kOffZ, a.qzeros + (size_t)t * (SUB * kItemZBytes), SUB * kItemZBytes, bar, policy);
             };
             // weights never depend on earlier work in the stream: fill the ring before waiting on it
+            GPTQ_TRACE_MIN(a.trace_slot, first_weight_issue);
             for (int i = 0; i < n_pre; ++i) issue_weights(t0 + i, i);
             pdl_wait();
+            GPTQ_TRACE_MIN(a.trace_slot, first_wait_done);
+            GPTQ_TRACE_MAX(a.trace_slot, last_wait_done);
             int s = 0, round = 0;
             for (int it = 0; it < n_items; ++it) {
                 const uint32_t bar = bar_full + 8 * s;
@@ -211,6 +222,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         for (int it = 0; it < n_items; ++it) {
             const uint32_t st = ring + s * kStage;
             if (ok) ok = mbar_wait(bar_full + 8 * s, phase);   // on failure: stale data, status word set
+            if (it == 0 && threadIdx.x == 0) GPTQ_TRACE_MIN(a.trace_slot, first_data);
 
             ItemSums<MT, SUB> sums;
             consume_item<MT, SUB>(st, w_off, s_off, z_off, x_off0, x_off1, z_add, sums);
@@ -274,6 +286,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 }
             }
         }
+        if (threadIdx.x == 0) GPTQ_TRACE_MAX(a.trace_slot, last_exit);
         return;
     }
 
@@ -327,6 +340,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 }
             }
         }
+        if (threadIdx.x == 0) GPTQ_TRACE_MAX(a.trace_slot, last_exit);
     }
 }
 
@@ -421,6 +435,7 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.fuse = fuse;
     args.bias = bias;
     args.residual = residual;
+    args.trace_slot = next_trace_slot();
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;

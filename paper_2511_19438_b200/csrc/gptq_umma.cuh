@@ -159,6 +159,7 @@ struct UmmaArgs {
     int fuse;               // 1: y[M, N / 2] = silu(gate) * up of a layer tiled with its column halves interleaved
     const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
     const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
+    int trace_slot;         // row of the launch timeline, or -1
 };
 
 // K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
@@ -186,6 +187,13 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     // the layer's format flags are needed by the dequant warps only: requested first, so that the round trip to HBM
     // hides behind the set-up
     const uint32_t flags = __ldg(&a.trailer->flags);
+    if (threadIdx.x == 0) {
+        GPTQ_TRACE_MIN(a.trace_slot, first_entry);
+        if (blockIdx.x == 0) {
+            GPTQ_TRACE_SET(a.trace_slot, kernel_id, 2);
+            GPTQ_TRACE_SET(a.trace_slot, ctas, gridDim.x);
+        }
+    }
     constexpr int kStage = umma_slot_bytes(TOK, NP);
     // ring slot = BPS K64 blocks: [x tile of each block][W blocks of each panel]
     constexpr int BPS = umma_blocks_per_slot(TOK);
@@ -262,11 +270,14 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     tma_load_2d(st + kOffW + j * BPS * kUmmaWBlockBytes, &w_map, 0, (2 * a.G * (p0 + j) + b_first + b) * 64, bar);
             };
             const int n_pre = NR < NS ? NR : NS;
+            GPTQ_TRACE_MIN(a.trace_slot, first_weight_issue);
             for (int i = 0; i < n_pre; ++i) {                // weights do not depend on earlier kernels
                 mbar_expect_tx(bar_full + 8 * i, kWBytes);
                 issue_w(i, i);
             }
             pdl_wait();
+            GPTQ_TRACE_MIN(a.trace_slot, first_wait_done);
+            GPTQ_TRACE_MAX(a.trace_slot, last_wait_done);
             // Every instruction of this thread (a wait, an expect, a copy) costs it about 0.1 us, which bounds
             // the kernel when there are many of them per byte, so a ring slot holds a whole K group where shared
             // memory allows and a refill is one wait, one arrive-and-expect and the copies.  The slot is free
@@ -310,6 +321,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     ok = mbar_wait(bar_afull + 8 * (j * NA + sa), pha);
                     if (!ok) return;
                     tc_fence_after_sync();
+                    if (b == b_begin) GPTQ_TRACE_MIN(a.trace_slot, first_data);   // (nothing in a normal build)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)   // 16 k per MMA: 8 TMEM columns of A, 32 bytes of each x row
                         umma_f16_ts(d_tmem + j * ISS * TOK, tmem_base + kAcol + (j * NA + sa) * 32 + kk * 8,
@@ -625,6 +637,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) GPTQ_TRACE_MAX(a.trace_slot, last_exit);
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kCols);
@@ -775,6 +788,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.fuse = fuse;
     args.bias = bias;
     args.residual = residual;
+    args.trace_slot = next_trace_slot();
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, group_size));
     const int sub = kGroup / group_size;
     if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;
@@ -810,6 +824,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
         ta.tile0 = plan.ctas / plan.S;
         ta.S = plan.tail_S;
         ta.stages = plan.tail_stages;
+        ta.trace_slot = next_trace_slot();
         st = launch(ta, plan.tail_tiles * plan.tail_S);
     }
     return st;

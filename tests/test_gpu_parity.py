@@ -6,6 +6,7 @@ within rtol 1e-2 / atol 1e-2*sqrt(K/4096) of the fp64 oracle (the stated toleran
 within the much tighter bound this implementation should meet (exact integer q - z, fp32
 accumulation, one fp16 rounding: |err| <= 2^-11 |y| + 1e-4 * sqrt(K/4096))."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -771,3 +772,30 @@ def test_config5_decode_step_layer(layer, ws):
             ws.ensure_for(M, D)
             full_check(L, x, H.gemm(H.to_device(x), D).cpu().numpy())
     assert B.gptq_check_status() == B.GPTQ_OK
+
+
+# ------------------------------------------------------------------------------- launch timeline
+def test_trace_entry_points_are_inert_in_the_normal_build():
+    assert B.gptq_trace_reset() == B.GPTQ_ERR_UNSUPPORTED
+    n, rows = B.gptq_trace_read(4)
+    assert n == B.GPTQ_ERR_UNSUPPORTED and rows == []
+
+
+def test_timeline_tool_shows_weight_prefetch_overlapping_the_previous_launch():
+    """The instrumented build (a library file of its own, run in a child process) traces a chain of decode launches:
+    every launch after the first must have issued its first weight copy before the launch ahead of it was done, and
+    its griddepcontrol.wait must not return before that."""
+    import re
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-m", "paper_2511_19438_b200.timeline", "--m", "1", "--rounds", "2"],
+                         cwd=root, capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    rows = [l for l in out.stdout.splitlines() if re.match(r"\s*\d+\s+\w+\s+(mma\.sync|tcgen05)", l)]
+    assert len(rows) == 8, out.stdout
+    for line in rows[1:]:
+        left, mid, _ = line.split("|")
+        started, weights, wait_first = (float(v) for v in mid.split()[:3])
+        assert weights < 0.0, f"no prefetch overlap: {line}"
+        assert started < weights and wait_first > 0.0, line
