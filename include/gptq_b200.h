@@ -152,6 +152,12 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
 
+/* act_order argument of the matmul entry points: 0 = groups are consecutive rows; 1 = act-order, the call first
+ * gathers x into the sorted row order with g_idx (= gptq_repack's perm_out); GPTQ_ACT_ORDER_PRESORTED = act-order, but
+ * x already is in the sorted row order (its producer wrote it that way, see gptq_gemm_silu_mul_scatter): no gather,
+ * no workspace, g_idx is ignored and may be NULL.  gptq_gemm_noalloc takes 0 and 1 only. */
+#define GPTQ_ACT_ORDER_PRESORTED 2
+
 /* (No counterpart in the paper: additions fused into the epilogue of the product of Sections 1 and 3.)
  * y fp16[M,N] = x . dequant(W) + bias[n] + residual[m][n]: the bias of a projection (fp16 [N]) and the residual add
  * that follows the o and down projections of a Llama block (fp16 [M,N]), joined to the fp32 sums before the one
@@ -174,6 +180,18 @@ int gptq_gemm_bias_residual(const void *x, const void *qweight, const void *qzer
 int gptq_gemm_silu_mul(const void *x, const void *qweight, const void *qzeros, const void *scales,
                        const int32_t *g_idx, void *out, int M, int N, int K, int group_size, int act_order,
                        void *stream);
+
+/* (No counterpart in the paper.)  gptq_gemm_silu_mul whose output column i is stored at column out_index[i] of `out`
+ * (int32 [N / 2], device, 16-byte aligned, a permutation of 0 .. N/2 - 1): with out_index = the inverse of the sort
+ * permutation of an act-order layer that consumes `out` (gptq_invert_perm of that layer's perm_out), `out` is written in
+ * that layer's sorted row order and its matmul can run with GPTQ_ACT_ORDER_PRESORTED - the separate gather launch of
+ * act-order and its round trip through memory disappear.  Meant for decode-sized M: the stores are 2 bytes each. */
+int gptq_gemm_silu_mul_scatter(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                               const int32_t *g_idx, const int32_t *out_index, void *out, int M, int N, int K,
+                               int group_size, int act_order, void *stream);
+/* inverse[perm[i]] = i for i < K (perm a permutation of 0 .. K-1, e.g. gptq_repack's perm_out; entries out of range are
+ * skipped). */
+int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream);
 
 /* Process-wide switch: with enable != 0, gptq_gemm runs problems with M >= 256 and an even number
  * of 128-column panels on CTA pairs (tcgen05.mma.cta_group::2: two SMs share one 256 x 256 x 16 MMA and

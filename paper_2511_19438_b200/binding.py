@@ -24,6 +24,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 GPTQ_FORMAT_ZEROS_MINUS_ONE = 1
 GPTQ_FORMAT_GATE_UP = 2
+GPTQ_ACT_ORDER_PRESORTED = 2
 GPTQ_OK = 0
 GPTQ_ERR_NULL = -1
 GPTQ_ERR_SHAPE = -2
@@ -72,6 +73,8 @@ _SIGNATURES = {
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_silu_mul": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_bias_residual": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_silu_mul_scatter": (_i, [_vp] * 7 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_invert_perm": (_i, [_vp, _vp, _i, _vp]),
     "gptq_set_cta_pairs": (_i, [_i]),
     "gptq_gemm_host": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
@@ -195,6 +198,16 @@ def gptq_gemm_host(x_host, qweight, qzeros, scales, g_idx, y_host, x_stage, y_st
 def gptq_gemm_silu_mul(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, stream=None) -> int:
     return _lib.gptq_gemm_silu_mul(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(out), M, N,
                                    K, group_size, int(act_order), _stream(stream))
+
+
+def gptq_gemm_silu_mul_scatter(x, qweight, qzeros, scales, g_idx, out_index, out, M, N, K, group_size, act_order,
+                               stream=None) -> int:
+    return _lib.gptq_gemm_silu_mul_scatter(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(out_index),
+                                           _ptr(out), M, N, K, group_size, int(act_order), _stream(stream))
+
+
+def gptq_invert_perm(perm, inverse, K, stream=None) -> int:
+    return _lib.gptq_invert_perm(_ptr(perm), _ptr(inverse), K, _stream(stream))
 
 
 def gptq_gemm_bias_residual(x, qweight, qzeros, scales, g_idx, bias, residual, y, M, N, K, group_size, act_order,

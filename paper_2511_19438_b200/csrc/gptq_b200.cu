@@ -120,7 +120,7 @@ static StreamKGemmPlan make_streamk_plan(int M, int N, int K, int act_order, int
 // gptq_gemm keeps its split-K partials on chip; its only scratch is the gathered x of act-order layers.
 static size_t gemm_workspace_need(int M, int K, int act_order)
 {
-    return act_order ? (((size_t)M * K * sizeof(__half) + 255) & ~(size_t)255) : 0;
+    return act_order == 1 ? (((size_t)M * K * sizeof(__half) + 255) & ~(size_t)255) : 0;   // 2: x arrives sorted
 }
 
 // Copy streams and events of gptq_gemm_host_batch (per device, created on first use; no device memory).
@@ -375,15 +375,16 @@ int gptq_set_workspace(void *ptr, size_t bytes)
 // y = x W (fuse == 0, y is [M, N]) or silu(gate) * up of y's column halves (fuse == 1, y is [M, N / 2])
 static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
                          void *y, int M, int N, int K, int group_size, int act_order, int fuse, const void *bias,
-                         const void *residual, void *stream)
+                         const void *residual, const int32_t *out_index, void *stream)
 {
-    if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
+    if (act_order < 0 || act_order > GPTQ_ACT_ORDER_PRESORTED) return GPTQ_ERR_LAYOUT;
+    if (!x || !qweight || !qzeros || !scales || !y || (act_order == 1 && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(M, N, K, group_size);
     if (st) return st;
     if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y))
         return GPTQ_ERR_ALIGN;
-    if (act_order && !aligned16(g_idx)) return GPTQ_ERR_ALIGN;
-    if (!aligned16(bias) || !aligned16(residual)) return GPTQ_ERR_ALIGN;     // a null pointer passes
+    if (act_order == 1 && !aligned16(g_idx)) return GPTQ_ERR_ALIGN;
+    if (!aligned16(bias) || !aligned16(residual) || !aligned16(out_index)) return GPTQ_ERR_ALIGN;     // a null pointer passes
     st = check_fast_path(N, K, group_size);
     if (st) return st;
 
@@ -393,7 +394,7 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     cudaStream_t s = (cudaStream_t)stream;
     const __half *xin = (const __half *)x;
     const bool extras = bias != nullptr || residual != nullptr;
-    if (act_order) {
+    if (act_order == 1) {
         Workspace ws;
         {
             std::lock_guard<std::mutex> lock(g_mutex);
@@ -414,14 +415,14 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
         // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
         return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, fuse, (const __half *)bias,
-                           (const __half *)residual, s);
+                           (const __half *)residual, out_index, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
         const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sms);
         st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * ldy, rows, N, K,
                            pl, fuse, (const __half *)bias,
-                           residual ? (const __half *)residual + (size_t)m0 * N : nullptr, s);
+                           residual ? (const __half *)residual + (size_t)m0 * N : nullptr, out_index, s);
         if (st) return st;
     }
     return GPTQ_OK;
@@ -432,21 +433,38 @@ extern "C" {
 int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
               void *y, int M, int N, int K, int group_size, int act_order, void *stream)
 {
-    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, nullptr, nullptr, stream);
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, nullptr, nullptr, nullptr, stream);
 }
 
 int gptq_gemm_bias_residual(const void *x, const void *qweight, const void *qzeros, const void *scales,
                             const int32_t *g_idx, const void *bias, const void *residual, void *y, int M, int N, int K,
                             int group_size, int act_order, void *stream)
 {
-    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, bias, residual, stream);
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, bias, residual, nullptr, stream);
 }
 
 int gptq_gemm_silu_mul(const void *x, const void *qweight, const void *qzeros, const void *scales,
                        const int32_t *g_idx, void *out, int M, int N, int K, int group_size, int act_order,
                        void *stream)
 {
-    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, nullptr, nullptr, stream);
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, nullptr, nullptr, nullptr,
+                         stream);
+}
+
+int gptq_gemm_silu_mul_scatter(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                               const int32_t *g_idx, const int32_t *out_index, void *out, int M, int N, int K,
+                               int group_size, int act_order, void *stream)
+{
+    if (!out_index) return GPTQ_ERR_NULL;
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, nullptr, nullptr, out_index,
+                         stream);
+}
+
+int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream)
+{
+    if (!perm || !inverse) return GPTQ_ERR_NULL;
+    if (K < 1) return GPTQ_ERR_SHAPE;
+    return launch_invert_perm(perm, inverse, K, (cudaStream_t)stream);
 }
 
 int gptq_gemm_host(const void *x_host, const void *qweight, const void *qzeros, const void *scales,
@@ -494,6 +512,7 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
                       const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
                       void *stream)
 {
+    if (act_order < 0 || act_order > 1) return GPTQ_ERR_LAYOUT;   // the pre-sorted mode belongs to gptq_gemm only
     if (!x || !qweight || !qzeros || !scales || !y || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(M, N, K, group_size);
     if (st) return st;
@@ -544,7 +563,7 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
         const gptq_host_problem_t &q = problems[i];
         int st = GPTQ_OK;
         if (!q.x_host || !q.y_host || !q.x_stage || !q.y_stage || !q.qweight || !q.qzeros || !q.scales ||
-            (q.act_order && !q.g_idx))
+            (q.act_order == 1 && !q.g_idx))
             st = GPTQ_ERR_NULL;
         if (!st) st = check_shape(q.M, q.N, q.K, q.group_size);
         if (!st && (!aligned16(q.x_stage) || !aligned16(q.y_stage) || !aligned16(q.qweight) || !aligned16(q.qzeros) ||

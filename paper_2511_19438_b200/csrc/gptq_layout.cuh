@@ -317,4 +317,19 @@ int launch_gather_x(const __half *x, const int32_t *perm, __half *x_out, int M, 
     return record_cuda_error(cudaLaunchKernelEx(&cfg, gather_x_kernel, x, perm, x_out, M, K));
 }
 
+// inverse[perm[i]] = i: where an element that sits at original position c goes in the sorted order
+__global__ void invert_perm_kernel(const int32_t *__restrict__ perm, int32_t *__restrict__ inverse, int K)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= K) return;
+    const int c = perm[i];
+    if (c >= 0 && c < K) inverse[c] = i;
+}
+
+int launch_invert_perm(const int32_t *perm, int32_t *inverse, int K, cudaStream_t s)
+{
+    invert_perm_kernel<<<(K + 255) / 256, 256, 0, s>>>(perm, inverse, K);
+    return record_cuda_error(cudaGetLastError());
+}
+
 }  // namespace gptq

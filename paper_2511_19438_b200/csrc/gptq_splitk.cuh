@@ -95,6 +95,7 @@ struct SplitKArgs {
     const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
     const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
     int trace_slot;         // row of the launch timeline, or -1
+    const int32_t *out_index; // with fuse: output column i is stored at column out_index[i] (nullptr: at i)
 };
 
 // silu(g) * u in fp32
@@ -272,7 +273,6 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 }
                 named_bar_sync(1, kConsumerThreads);
                 if (warp < 4) {
-                    __half *yp = a.y + (size_t)p * 64 + col;
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -280,7 +280,9 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                             const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                             if (m < a.M) {
                                 const float up = lds_f32(hand + (uint32_t)(m * 64 + col + 8 * (i >> 1)) * 4u);
-                                yp[(size_t)m * (a.N / 2) + 8 * (i >> 1)] = __float2half_rn(silu_mul(acc[mt][i], up));
+                                const int oc = p * 64 + col + 8 * (i >> 1);
+                                a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
+                                    __float2half_rn(silu_mul(acc[mt][i], up));
                             }
                         }
                 }
@@ -335,7 +337,8 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 const int half_w = width >> 1;
                 for (int idx = threadIdx.x; idx < a.M * half_w; idx += kConsumerThreads) {
                     const int m = idx >> (wsh - 1), cc = idx - (m << (wsh - 1));
-                    a.y[(size_t)m * (a.N / 2) + (size_t)p * 64 + rank * half_w + cc] =
+                    const int oc = p * 64 + rank * half_w + cc;
+                    a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
                         __float2half_rn(silu_mul(slice_sum(m, cc), slice_sum(m, half_w + cc)));
                 }
             }
@@ -425,7 +428,7 @@ static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, co
 
 int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
                   int M, int N, int K, const SplitKPlan &plan, int fuse, const __half *bias, const __half *residual,
-                  cudaStream_t s)
+                  const int32_t *out_index, cudaStream_t s)
 {
     SplitKArgs args;
     args.qweight = (const uint8_t *)qweight;
@@ -442,6 +445,7 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.bias = bias;
     args.residual = residual;
     args.trace_slot = next_trace_slot();
+    args.out_index = out_index;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;

@@ -160,6 +160,7 @@ struct UmmaArgs {
     const __half *bias;     // fp16 [N] added to every row of y, or nullptr (not with fuse)
     const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
     int trace_slot;         // row of the launch timeline, or -1
+    const int32_t *out_index; // with fuse: output column i is stored at column out_index[i] (nullptr: at i)
 };
 
 // K64 blocks per ring slot of the single-CTA kernel: a whole K group (two blocks: fewer, larger copies for the
@@ -544,8 +545,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                                 const __half2 o = __floats2half2_rn(silu_mul(gf.x, uf.x), silu_mul(gf.y, uf.y));
                                 ow[e] = *reinterpret_cast<const uint32_t *>(&o);
                             }
-                            *reinterpret_cast<uint4 *>(a.y + (size_t)m * (a.N / 2) + (size_t)p * 64 + c8 * 8) =
-                                make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                            __half *orow = a.y + (size_t)m * (a.N / 2);
+                            const int oc = p * 64 + c8 * 8;
+                            if (a.out_index == nullptr) {
+                                *reinterpret_cast<uint4 *>(orow + oc) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                            } else {
+                                // scattered columns: eight destinations (two 16-byte index loads), eight 2-byte stores
+                                const int4 ia = *reinterpret_cast<const int4 *>(a.out_index + oc);
+                                const int4 ib = *reinterpret_cast<const int4 *>(a.out_index + oc + 4);
+                                const int dst[8] = {ia.x, ia.y, ia.z, ia.w, ib.x, ib.y, ib.z, ib.w};
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    orow[dst[e]] = __ushort_as_half((unsigned short)(ow[e >> 1] >> (16 * (e & 1))));
+                            }
                         }
                     }
                 }
@@ -624,9 +636,19 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 for (int idx = threadIdx.x - 32 * kFirstDq; idx < rows * w4; idx += 128 * NP * SETS) {
                     const int m = idx / w4, cc = rank * half_w + 4 * (idx - m * w4);
                     const float4 gsum = sum4(m, cc), usum = sum4(m, 64 + cc);
-                    store4(a.y + (size_t)(m0 + m) * (a.N / 2) + (size_t)p * 64 + cc,
-                           make_float4(silu_mul(gsum.x, usum.x), silu_mul(gsum.y, usum.y), silu_mul(gsum.z, usum.z),
-                                       silu_mul(gsum.w, usum.w)));
+                    const float4 ov = make_float4(silu_mul(gsum.x, usum.x), silu_mul(gsum.y, usum.y), silu_mul(gsum.z, usum.z),
+                                                  silu_mul(gsum.w, usum.w));
+                    __half *orow = a.y + (size_t)(m0 + m) * (a.N / 2);
+                    const int oc = p * 64 + cc;
+                    if (a.out_index == nullptr) {
+                        store4(orow + oc, ov);
+                    } else {
+                        const int4 ia = *reinterpret_cast<const int4 *>(a.out_index + oc);
+                        orow[ia.x] = __float2half_rn(ov.x);
+                        orow[ia.y] = __float2half_rn(ov.y);
+                        orow[ia.z] = __float2half_rn(ov.z);
+                        orow[ia.w] = __float2half_rn(ov.w);
+                    }
                 }
             }
         }
@@ -773,7 +795,7 @@ static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const
 
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
                 int K, int group_size, const UmmaPlan &plan, int fuse, const __half *bias, const __half *residual,
-                cudaStream_t s)
+                const int32_t *out_index, cudaStream_t s)
 {
     UmmaArgs args;
     args.scales = (const uint8_t *)scales;
@@ -789,6 +811,7 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     args.bias = bias;
     args.residual = residual;
     args.trace_slot = next_trace_slot();
+    args.out_index = out_index;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, group_size));
     const int sub = kGroup / group_size;
     if (plan.stages < 1 || plan.stages * umma_blocks_per_slot(plan.tok) >= kUmmaDoneRing) return GPTQ_ERR_UNSUPPORTED;

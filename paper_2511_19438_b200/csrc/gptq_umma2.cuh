@@ -349,6 +349,7 @@ int launch_umma2(const __half *x, const void *qweight, const void *qzeros, const
     args.bias = nullptr;
     args.residual = nullptr;
     args.trace_slot = -1;
+    args.out_index = nullptr;
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup));
     CUtensorMap w_map, x_map;
     const uint64_t w_rows = (uint64_t)K * N / 2 / 64;

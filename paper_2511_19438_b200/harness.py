@@ -99,3 +99,31 @@ def gemm_bias_residual(x: torch.Tensor, D: DeviceLinear, bias: torch.Tensor | No
     B.check(B.gptq_gemm_bias_residual(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, bias, residual, y, M, D.N, D.K,
                                       D.group_size, D.act_order, stream), "gptq_gemm_bias_residual")
     return y
+
+
+def invert_perm(perm: torch.Tensor) -> torch.Tensor:
+    """inverse[perm[i]] = i through gptq_invert_perm."""
+    inv = torch.empty_like(perm)
+    B.check(B.gptq_invert_perm(perm, inv, perm.numel()), "gptq_invert_perm")
+    return inv
+
+
+def gemm_silu_mul_scatter(x: torch.Tensor, D: DeviceLinear, out_index: torch.Tensor, out: torch.Tensor | None = None,
+                          stream=None) -> torch.Tensor:
+    """gemm_silu_mul whose output column i lands at column out_index[i]."""
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, D.N // 2), dtype=torch.float16, device=x.device)
+    B.check(B.gptq_gemm_silu_mul_scatter(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, out_index, out, M, D.N, D.K,
+                                         D.group_size, D.act_order, stream), "gptq_gemm_silu_mul_scatter")
+    return out
+
+
+def gemm_presorted(x_sorted: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """gptq_gemm of an act-order layer whose input already is in the layer's sorted row order (no gather)."""
+    M = x_sorted.shape[0]
+    if y is None:
+        y = torch.empty((M, D.N), dtype=torch.float16, device=x_sorted.device)
+    B.check(B.gptq_gemm(x_sorted, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, D.N, D.K, D.group_size,
+                        B.GPTQ_ACT_ORDER_PRESORTED, stream), "gptq_gemm (pre-sorted)")
+    return y

@@ -774,6 +774,56 @@ def test_config5_decode_step_layer(layer, ws):
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
+# ------------------------------------------------------------------------------- act-order without the gather
+@pytest.mark.parametrize("M", [1, 6, 16, 24, 70, 300])
+def test_mlp_block_with_act_order_down_and_no_gather(M, ws):
+    """gate_up -> silu(gate) * up -> down, with an act-order down projection.  Path A: fused activation, then gptq_gemm
+    gathers its input.  Path B: the fused epilogue scatters its output straight into down's sorted row order and down
+    runs pre-sorted.  Both feed the same kernels the same numbers in the same order, so they agree bit for bit; and the
+    result matches the oracle applied to the fp16 activations the GPU produced."""
+    H_, I_ = 512, 1024                                    # hidden size, intermediate size
+    Lg = wl.make_linear(H_, 2 * I_, seed=wl.seed_for("mlp-gu"))
+    Ld = wl.make_linear(I_, H_, seed=wl.seed_for("mlp-down"), act_order=True)
+    Dg, Dd = H.upload_and_repack(Lg, gate_up=True), H.upload_and_repack(Ld)
+    ws.ensure_for(M, Dd)
+    x_np = wl.make_x(M, H_, wl.seed_for("mlp-x", M))
+    x = H.to_device(x_np)
+    inv = H.invert_perm(Dd.perm)
+    perm_np = Dd.perm.cpu().numpy()
+    assert np.array_equal(inv.cpu().numpy()[perm_np], np.arange(I_))             # inverse[perm[i]] = i
+    act = H.gemm_silu_mul(x, Dg)                                                   # [M, I] in checkpoint column order
+    y_a = H.gemm(act, Dd)
+    act_sorted = H.gemm_silu_mul_scatter(x, Dg, inv)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    assert torch.equal(act_sorted, act[:, Dd.perm.long()])                         # column i went to inverse[i]
+    y_b = H.gemm_presorted(act_sorted, Dd)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    assert torch.equal(y_a, y_b)
+    act_np = act.cpu().numpy()
+    want = oracle.gemm_f64(act_np, Ld.qweight, Ld.qzeros, Ld.scales, Ld.g_idx, 128)
+    # the stated bar is for unit-variance activations; these rows (products of two projections) have an rms of 2-4,
+    # and every error term of the matmul is proportional to it
+    rms = np.maximum(1.0, np.sqrt(np.mean(act_np.astype(np.float64) ** 2, axis=1, keepdims=True)))
+    err = np.abs(y_b.cpu().numpy().astype(np.float64) - want)
+    bar = 1e-2 * math.sqrt(I_ / 4096) * rms + 1e-2 * np.abs(want)
+    assert np.all(err <= bar), f"{int((err > bar).sum())} violations, worst ratio {(err / bar).max():.2f}"
+
+
+def test_presorted_mode_argument_checks():
+    K, N, M = 512, 256, 3
+    L = wl.make_linear(K, N, seed=wl.seed_for("presorted"), act_order=True)
+    D = H.upload_and_repack(L)
+    x = H.to_device(wl.make_x(M, K, 1))
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, N, K, 128, 3) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, N, K, 128, 1) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, N, K, 128, 2) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_workspace_bytes(M, N, K, 128, B.GPTQ_ACT_ORDER_PRESORTED) == 0
+    assert B.gptq_gemm_silu_mul_scatter(x, D.qweight_t, D.qzeros_t, D.scales_t, None, None, y, M, N, K, 128, 0) == B.GPTQ_ERR_NULL
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(y) == 0
+
+
 # ------------------------------------------------------------------------------- launch timeline
 def test_trace_entry_points_are_inert_in_the_normal_build():
     assert B.gptq_trace_reset() == B.GPTQ_ERR_UNSUPPORTED
