@@ -96,6 +96,11 @@ struct SplitKArgs {
     const __half *residual; // fp16 [M, N] added to y, or nullptr (not with fuse); may be y itself
     int trace_slot;         // row of the launch timeline, or -1
     const int32_t *out_index; // with fuse: output column i is stored at column out_index[i] (nullptr: at i)
+    // split-K column slices: the panel is one run of 128 columns, or with fuse two runs of 64 (gate, up); within a run
+    // owner q finishes columns [lo(q), lo(q + 1)), lo(q) = q * run / S (byte q of slice_lo, q < 8; lo(S) = run);
+    // slice_max = the widest slice
+    unsigned long long slice_lo;
+    int slice_max;
 };
 
 // silu(g) * u in fp32
@@ -151,7 +156,11 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         fence_barrier_init();
         fence_proxy_async();
         // split-K: S slices of a.M x (128 / S) floats will arrive in this CTA's receive buffer
-        if (S > 1) mbar_arrive_expect_tx(bar_recv, (uint32_t)(a.M * kPanel * 4));
+        if (S > 1) {
+            const int run = a.fuse ? 64 : kPanel;
+            const int mine = (rank + 1 < S ? (int)((a.slice_lo >> (8 * (rank + 1))) & 255) : run) - (int)((a.slice_lo >> (8 * rank)) & 255);
+            mbar_arrive_expect_tx(bar_recv, (uint32_t)(S * a.M * (a.fuse ? 2 : 1) * mine * 4));
+        }
     }
     __syncthreads();
     if (S > 1) cluster_arrive_release();   // "my receive barrier is armed"; waited for before the first send
@@ -296,50 +305,53 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     __syncwarp();
     cluster_wait_acquire();                 // every CTA of the cluster has armed its receive barrier
     if (warp < kConsumerWarps) {
-        const int width = kPanel / S;       // S is 2, 4 or 8
-        const int wsh = S == 2 ? 6 : S == 4 ? 5 : 4;   // log2(width): owners and offsets by shifts, not divisions
-        // owner q gets columns [q width, (q + 1) width); with the fused epilogue the first half of its slice are gate
-        // columns [q width / 2, ...) and the second half the matching up columns (64 further in the panel)
-        const int qsh = a.fuse ? wsh - 1 : wsh, cmask = a.fuse ? 63 : 127;
-        const uint32_t recv = ring + (uint32_t)a.stages * kStage;   // [sender rank][token row][width] floats
+        // One run of 128 columns, or with the fused epilogue two runs of 64 (gate | up).  Within a run owner q finishes
+        // columns [lo(q), lo(q + 1)); S is any value from 2 to 8, so the slices may differ by one column.
+        // Receive buffer of an owner: [sender rank][token row][run][slice_max] floats.
+        const int hsh = a.fuse ? 6 : 7, hmask = (1 << hsh) - 1;            // log2(run), column within the run
+        const int runs = a.fuse ? 2 : 1;
+        const int hwmax = a.slice_max, wstride = runs * hwmax;
+        const uint32_t recv = ring + (uint32_t)a.stages * kStage;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
                 if (m < a.M) {
-                    const int c = col + 8 * (i >> 1), cc = c & cmask;
-                    const int q = cc >> qsh;
-                    const int pos = ((c - cc) >> (7 - wsh)) + cc - (q << qsh);   // (c - cc) is 0, or 64 for an up column
-                    const uint32_t off = (uint32_t)((rank * a.M + m) * width + pos) * 4u;
+                    const int c = col + 8 * (i >> 1), cc = c & hmask;
+                    const int q = ((cc + 1) * S - 1) >> hsh;                 // the q with lo(q) <= cc < lo(q + 1)
+                    const int pos = (c >> hsh) * hwmax + cc - (int)((a.slice_lo >> (8 * q)) & 255);
+                    const uint32_t off = (uint32_t)((rank * a.M + m) * wstride + pos) * 4u;
                     st_async_f32(map_to_cluster_rank(recv + off, (uint32_t)q), acc[mt][i],
                                  map_to_cluster_rank(bar_recv, (uint32_t)q));
                 }
             }
         if (mbar_wait_cluster(bar_recv, 0) && layout_ok) {
-            auto slice_sum = [&](int m, int cc) {   // rank order
+            auto slice_sum = [&](int m, int j) {   // rank order
                 float v[8];
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    v[q] = q < S ? lds_f32(recv + (uint32_t)((q * a.M + m) * width + cc) * 4u) : 0.f;
+                    v[q] = q < S ? lds_f32(recv + (uint32_t)((q * a.M + m) * wstride + j) * 4u) : 0.f;
                 float sum = 0.f;
 #pragma unroll
                 for (int q = 0; q < 8; ++q) sum += v[q];
                 return sum;
             };
-            if (!a.fuse) {
-                const int c_lo = rank * width;
-                for (int idx = threadIdx.x; idx < a.M * width; idx += kConsumerThreads) {
-                    const int m = idx >> wsh, cc = idx - (m << wsh);
-                    a.y[(size_t)m * a.N + (size_t)p * kPanel + c_lo + cc] = __float2half_rn(slice_sum(m, cc) + addend(m, p * kPanel + c_lo + cc));
-                }
-            } else {
-                const int half_w = width >> 1;
-                for (int idx = threadIdx.x; idx < a.M * half_w; idx += kConsumerThreads) {
-                    const int m = idx >> (wsh - 1), cc = idx - (m << (wsh - 1));
-                    const int oc = p * 64 + rank * half_w + cc;
-                    a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
-                        __float2half_rn(silu_mul(slice_sum(m, cc), slice_sum(m, half_w + cc)));
+            const int lo = (int)((a.slice_lo >> (8 * rank)) & 255);
+            const int hw = (rank + 1 < S ? (int)((a.slice_lo >> (8 * (rank + 1))) & 255) : (1 << hsh)) - lo;   // at most 64 columns per run
+            // threads as [rows per pass][jw columns], jw the power of two that holds the slice (8 .. 64)
+            const int jsh = hw <= 8 ? 3 : hw <= 16 ? 4 : hw <= 32 ? 5 : 6;
+            const int j = threadIdx.x & ((1 << jsh) - 1);
+            if (j < hw) {
+                for (int m = threadIdx.x >> jsh; m < a.M; m += kConsumerThreads >> jsh) {
+                    if (!a.fuse) {
+                        const int n = p * kPanel + lo + j;
+                        a.y[(size_t)m * a.N + n] = __float2half_rn(slice_sum(m, j) + addend(m, n));
+                    } else {
+                        const int oc = p * 64 + lo + j;
+                        a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
+                            __float2half_rn(silu_mul(slice_sum(m, j), slice_sum(m, hwmax + j)));
+                    }
                 }
             }
         }
@@ -364,16 +376,27 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int group_size, int sm_count)
     const int G = K / kGroup, panels = N / kPanel;
     pl.sub = kGroup / group_size;
     const int stage = streamk_stage_bytes(MT, pl.sub);
-    const int cps_max = splitk_ctas_per_sm(MT);
+    // The 8-row, group-128 instantiation needs 56 registers, so four of its CTAs fit an SM, and for it cluster sizes 3
+    // and 6 are candidates too (5 and 7 measured badly: clusters of that size often find no room): the 7B gate_up
+    // (172 panels) takes 13.8 us with 3 x 172 CTAs against 14.9 with 2 x 172, the 13B qkv 12.6 us with S = 4 against 13.9
+    // with S = 2.  The other instantiations keep powers of two and three CTAs per SM.
+    const bool wide = (MT == 1 && pl.sub == 1);
+    const int cps_max = wide ? 4 : splitk_ctas_per_sm(MT);
+    static const int kSizesWide[] = {1, 2, 3, 4, 6, 8}, kSizes[] = {1, 2, 4, 8};
+    const int *sizes = wide ? kSizesWide : kSizes;
+    const int n_sizes = wide ? 6 : 4;
     int best_S = 1;
     long long best_t = -1;
     for (int pass = 0; pass < 2 && best_t < 0; ++pass) {
-        for (int S = 1; S <= 8; S *= 2) {
+        for (int si = 0; si < n_sizes; ++si) {
+            const int S = sizes[si];
             if (S > G || (pass == 1 && S > 1)) break;          // nothing fits at once: several waves, no split
             const long long ctas = (long long)panels * S, ipc = (G + S - 1) / S;
             const long long on_busiest_sm = (ctas + sm_count - 1) / sm_count;
             if (pass == 0 && on_busiest_sm > cps_max) continue;
-            const long long serial = ipc * 45, shared = on_busiest_sm * ipc * 30;
+            // per item and SM: about 0.33 us with two resident CTAs, 0.28 with three or four (measured, hundredths of a us)
+            const long long per_item = !wide ? 30 : on_busiest_sm >= 3 ? 28 : 33;
+            const long long serial = ipc * 45, shared = on_busiest_sm * ipc * per_item;
             const long long t = (serial > shared ? serial : shared) + (S > 1 ? 100 : 0);
             if (best_t < 0 || t < best_t) { best_t = t; best_S = S; }
         }
@@ -384,7 +407,7 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int group_size, int sm_count)
     if (per_sm > cps_max) per_sm = cps_max;
     const int smem_cap = (227 * 1024) / per_sm - 1024;                 // per_sm CTAs fit ...
     const int smem_floor = (227 * 1024) / (per_sm + 1) + 512;          // ... per_sm + 1 do not
-    const int recv_bytes = MT * 4096;   // receive buffer of the split-K exchange, after the ring
+    const int recv_bytes = MT * 4480;   // receive buffer of the split-K exchange, after the ring: rows x (S slices: at most 140) floats
     int stages = (smem_cap - 2 * kRingOffset - recv_bytes) / stage;
     if (stages > 8) stages = 8;
     if (stages > items_per_cta) stages = items_per_cta;
@@ -446,6 +469,12 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     args.residual = residual;
     args.trace_slot = next_trace_slot();
     args.out_index = out_index;
+    {
+        const int run = fuse ? 64 : kPanel;
+        args.slice_lo = 0;
+        for (int q = 0; q < 8; ++q) args.slice_lo |= (unsigned long long)(q < plan.S ? q * run / plan.S : run) << (8 * q);
+        args.slice_max = (run + plan.S - 1) / plan.S;
+    }
     args.trailer = reinterpret_cast<const TiledTrailer *>((const uint8_t *)qzeros + tiled_zero_bytes(N, K, kGroup / plan.sub));
     // x as a 2-D tensor [M rows, K halves]; a box is one K64 tile of all token rows of the CTA tile
     CUtensorMap x_map;

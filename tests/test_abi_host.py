@@ -156,13 +156,14 @@ def test_cluster_plan_is_consistent(K, N, M, sms):
         return
     assert M <= 16
     assert pl.kernel == 1
-    assert pl.cluster_size in (1, 2, 4, 8) and pl.cluster_size <= G
+    wide = pl.m_tile == 8                     # 8 token rows, group 128: 56 registers, four CTAs fit an SM, S = 3 and 6 allowed
+    assert pl.cluster_size in ((1, 2, 3, 4, 6, 8) if wide else (1, 2, 4, 8)) and pl.cluster_size <= G
     assert pl.ctas == panels * pl.cluster_size
     assert pl.split_panels == (panels if pl.cluster_size > 1 else 0)
     assert pl.m_tile in (8, 16, 32, 64) and pl.m_tile >= min(M, 64)
     assert pl.m_chunks == (M + 63) // 64
     assert 1 <= pl.stages <= 8
-    per_sm = min(-(-pl.ctas // sms), 3 if pl.m_tile <= 16 else 1)
+    per_sm = min(-(-pl.ctas // sms), 4 if wide else 3 if pl.m_tile <= 16 else 1)
     assert per_sm * (pl.smem_bytes + 1024) <= 227 * 1024          # that many CTAs fit on an SM ...
     assert (per_sm + 1) * (pl.smem_bytes + 1024) > 227 * 1024     # ... and no more (even spreading)
     # the ring doubles as the fp32 partial tile of the cluster reduction

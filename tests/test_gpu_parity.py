@@ -774,6 +774,25 @@ def test_config5_decode_step_layer(layer, ws):
     assert B.gptq_check_status() == B.GPTQ_OK
 
 
+# ------------------------------------------------------------------------------- cluster sizes 3 and 6
+@pytest.mark.parametrize("K,N,S", [(768, 256, 6), (3072, 2432, 6), (768, 12672, 3)])
+@pytest.mark.parametrize("M", [1, 5, 8])
+def test_split_k_over_clusters_of_three_and_six(K, N, S, M, ws):
+    """Column slices of unequal width (128 / 3, 128 / 6) in the exchange: plain, with bias and residual, fused
+    activation, act-order on."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    st, pl = B.gptq_plan(M, N, K, 128, 1, sms)
+    if sms == 148:
+        assert pl.cluster_size == S, "the planner no longer picks this cluster size here: choose another shape"
+    L = wl.make_linear(K, N, seed=wl.seed_for("s36", K, N), act_order=True)
+    x_np = wl.make_x(M, K, wl.seed_for("s36-x", M))
+    y, D = run_gemm(L, x_np, ws)
+    y64 = oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert_close(y, y64, K, M)
+    check_bias_residual(L, M, ws, True, True)
+    check_silu_mul(L, x_np, ws)
+
+
 # ------------------------------------------------------------------------------- act-order without the gather
 @pytest.mark.parametrize("M", [1, 6, 16, 24, 70, 300])
 def test_mlp_block_with_act_order_down_and_no_gather(M, ws):
