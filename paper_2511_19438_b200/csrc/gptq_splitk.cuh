@@ -115,8 +115,16 @@ struct SplitKPlan {
     int smem_bytes;
 };
 
+// The 8-row, group-128 instantiation compiles to 56 registers, which plan_splitk counts on for four resident CTAs; the
+// timeline build's extra code would push it over, so there the bound is stated (a stated bound of 4 in the normal build
+// made the compiler choose 52 registers and a 1-2 % slower schedule).
+#ifdef GPTQ_TIMELINE
+constexpr int kSplitKWideCtas = 4;
+#else
+constexpr int kSplitKWideCtas = 3;
+#endif
 template <int MT, int SUB>
-__global__ void __launch_bounds__(kStreamKThreads, 3)
+__global__ void __launch_bounds__(kStreamKThreads, (MT == 1 && SUB == 1) ? kSplitKWideCtas : 3)
 splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 {
     extern __shared__ uint8_t smem_raw[];

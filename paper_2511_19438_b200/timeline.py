@@ -1,6 +1,6 @@
 """Launch timeline of a chain of decode matmuls: do consecutive launches overlap?
 
-    python -m paper_2511_19438_b200.timeline [--shapes 7b|13b] [--m 1] [--rounds 3] [--act-order]
+    python -m paper_2511_19438_b200.timeline [--shapes 7b|13b] [--only gate_up,down] [--m 1] [--rounds 3] [--act-order]
 
 Builds the library with the launch timeline compiled in (as libgptq_b200_timeline.so, next to the normal build),
 captures the layer's matmuls - each on distinct weights, so that every launch streams from HBM - in a CUDA graph,
@@ -20,6 +20,7 @@ def main():
     ap.add_argument("--m", type=int, default=1)
     ap.add_argument("--rounds", type=int, default=3, help="times the layer's matmuls are chained (distinct weights each)")
     ap.add_argument("--act-order", action="store_true")
+    ap.add_argument("--only", default="", help="comma-separated shape names: chain only these (e.g. gate_up)")
     args = ap.parse_args()
 
     from . import build as libbuild
@@ -28,6 +29,9 @@ def main():
     from . import binding as B, harness as H, workloads as wl
 
     shapes = wl.SHAPES_7B if args.shapes == "7b" else wl.SHAPES_13B
+    if args.only:
+        shapes = {k: v for k, v in shapes.items() if k in args.only.split(",")}
+        assert shapes, "no such shape"
     M = args.m
     ws = H.WorkspaceHolder()
     chain = []
