@@ -270,11 +270,12 @@ int gptq_selftest_wait_timeout(unsigned int limit_us, void *stream);
 /* ---- launch timeline (no counterpart in the paper: a tracing aid) ------------------------ */
 
 /* A library built with -DGPTQ_TIMELINE (GPTQ_NVCC_EXTRA=-DGPTQ_TIMELINE for the Python build) gives every matmul launch
- * the next of 64 rows (round robin) in which its CTAs record %globaltimer times: first CTA started, first weight
+ * the next of 64 rows (round robin) in which its CTAs record %globaltimer times: first and last CTA started, first weight
  * copy issued, griddepcontrol.wait first / last returned, first activation tile landed, last CTA done - what shows
  * whether consecutive launches overlap.  gptq_trace_reset clears the rows (synchronises `stream`); gptq_trace_read
  * synchronises `stream`, copies up to max_rows rows of eight 64-bit values {first_entry, first_weight_issue,
- * first_wait_done, last_wait_done, first_data, last_exit, kernel (1 mma.sync, 2 tcgen05), CTAs} in nanoseconds to host
+ * first_wait_done, last_wait_done, first_data, last_exit, kernel (1 mma.sync, 2 tcgen05) << 32 | CTAs, last_entry} (times in
+ * nanoseconds) to host
  * memory and returns the number of rows.  A row nobody wrote keeps ~0 in its "first" fields.  In a normal build both
  * return GPTQ_ERR_UNSUPPORTED and the kernels carry no tracing code.  `python -m paper_2511_19438_b200.timeline` prints
  * the table for a chain of decode launches. */

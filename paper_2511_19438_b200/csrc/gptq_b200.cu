@@ -659,7 +659,7 @@ int gptq_trace_reset(void *stream)
     static TraceRow blank[kTraceLaunches];
     for (int i = 0; i < kTraceLaunches; ++i) {
         blank[i].first_entry = blank[i].first_weight_issue = blank[i].first_wait_done = blank[i].first_data = ~0ull;
-        blank[i].last_wait_done = blank[i].last_exit = blank[i].kernel_id = blank[i].ctas = 0;
+        blank[i].last_wait_done = blank[i].last_exit = blank[i].kernel_and_ctas = blank[i].last_entry = 0;
     }
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = cudaMemcpyToSymbolAsync(g_trace, blank, sizeof(blank), 0, cudaMemcpyHostToDevice, s);

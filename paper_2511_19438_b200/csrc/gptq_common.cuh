@@ -164,13 +164,14 @@ __device__ __forceinline__ uint64_t global_timer_ns()
 }
 // ---- launch timeline (compiled in with -DGPTQ_TIMELINE only) -----------------------------------
 // Every matmul launch of a timeline build takes the next of kTraceLaunches rows and its CTAs record, with %globaltimer
-// and 64-bit atomic min / max, when the grid's first CTA started, when the first weight copy was issued, when
+// and 64-bit atomic min / max, when the grid's first and last CTA started, when the first weight copy was issued, when
 // griddepcontrol.wait first and last returned, when the first activation tile had landed and when the last CTA was
 // done.  gptq_trace_reset / gptq_trace_read move the rows; in a normal build the macros expand to nothing.
 constexpr int kTraceLaunches = 64;
 struct TraceRow {
     unsigned long long first_entry, first_weight_issue, first_wait_done, last_wait_done, first_data, last_exit;
-    unsigned long long kernel_id, ctas;     // 1 = mma.sync kernel, 2 = tcgen05 kernel; grid size
+    unsigned long long kernel_and_ctas;     // (1 = mma.sync kernel, 2 = tcgen05 kernel) << 32 | grid size
+    unsigned long long last_entry;          // when the grid's last CTA started
 };
 #ifdef GPTQ_TIMELINE
 __device__ TraceRow g_trace[kTraceLaunches];

@@ -137,9 +137,9 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
     const uint32_t flags = __ldg(&a.trailer->flags);
     if (threadIdx.x == 0) {
         GPTQ_TRACE_MIN(a.trace_slot, first_entry);
+        GPTQ_TRACE_MAX(a.trace_slot, last_entry);
         if (blockIdx.x == 0) {
-            GPTQ_TRACE_SET(a.trace_slot, kernel_id, 1);
-            GPTQ_TRACE_SET(a.trace_slot, ctas, gridDim.x);
+            GPTQ_TRACE_SET(a.trace_slot, kernel_and_ctas, (1ull << 32) | gridDim.x);
         }
     }
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;

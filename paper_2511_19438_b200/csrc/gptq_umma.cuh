@@ -190,9 +190,9 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     const uint32_t flags = __ldg(&a.trailer->flags);
     if (threadIdx.x == 0) {
         GPTQ_TRACE_MIN(a.trace_slot, first_entry);
+        GPTQ_TRACE_MAX(a.trace_slot, last_entry);
         if (blockIdx.x == 0) {
-            GPTQ_TRACE_SET(a.trace_slot, kernel_id, 2);
-            GPTQ_TRACE_SET(a.trace_slot, ctas, gridDim.x);
+            GPTQ_TRACE_SET(a.trace_slot, kernel_and_ctas, (2ull << 32) | gridDim.x);
         }
     }
     constexpr int kStage = umma_slot_bytes(TOK, NP);

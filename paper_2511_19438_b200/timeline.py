@@ -5,7 +5,7 @@
 Builds the library with the launch timeline compiled in (as libgptq_b200_timeline.so, next to the normal build),
 captures the layer's matmuls - each on distinct weights, so that every launch streams from HBM - in a CUDA graph,
 replays it and prints, per launch, %globaltimer times relative to the moment the previous launch's last CTA was
-done: first CTA started, first weight copy issued, griddepcontrol.wait first / last returned, first activation tile
+done: first and last CTA started, first weight copy issued, griddepcontrol.wait first / last returned, first activation tile
 landed, last CTA done.  A negative "started" or "weights" column is the overlap that programmatic dependent launch buys.
 """
 from __future__ import annotations
@@ -70,16 +70,17 @@ def main():
     launches = [r for r in launches if r[6] != 0]
     print(f"M = {M}, {len(chain)} matmuls ({'act-order: a gather launch precedes each, not traced' if args.act_order else 'no act-order'}); "
           f"{len(launches)} traced launches; microseconds relative to the previous launch's last CTA being done")
-    print(f"{'launch':>6} {'shape':>8} {'kernel':>8} {'CTAs':>5} | {'started':>8} {'weights':>8} {'wait first':>10} {'wait last':>9} "
+    print(f"{'launch':>6} {'shape':>8} {'kernel':>8} {'CTAs':>5} | {'started':>8} {'last CTA':>8} {'weights':>8} {'wait first':>10} {'wait last':>9} "
           f"{'x landed':>8} {'done':>7} | {'own duration':>12}")
     prev_exit = None
     names = [c[0] for c in chain]
     for i, r in enumerate(launches):
-        entry, wissue, wait0, wait1, data, last, kid, ctas = r
+        entry, wissue, wait0, wait1, data, last, kc, last_entry = r
+        kid, ctas = kc >> 32, kc & 0xffffffff
         ref = prev_exit if prev_exit is not None else entry
         f = lambda v: f"{(v - ref) / 1e3:8.2f}" if v not in (0, 2 ** 64 - 1) else "       -"
         name = names[i] if len(launches) == len(chain) else "?"
-        print(f"{i:6d} {name:>8} {'mma.sync' if kid == 1 else 'tcgen05':>8} {ctas:5d} | {f(entry)} {f(wissue)} {f(wait0):>10} {f(wait1):>9} "
+        print(f"{i:6d} {name:>8} {'mma.sync' if kid == 1 else 'tcgen05':>8} {ctas:5d} | {f(entry)} {f(last_entry)} {f(wissue)} {f(wait0):>10} {f(wait1):>9} "
               f"{f(data)} {f(last):>7} | {(last - entry) / 1e3:12.2f}")
         prev_exit = last
 

@@ -865,6 +865,6 @@ def test_timeline_tool_shows_weight_prefetch_overlapping_the_previous_launch():
     assert len(rows) == 8, out.stdout
     for line in rows[1:]:
         left, mid, _ = line.split("|")
-        started, weights, wait_first = (float(v) for v in mid.split()[:3])
+        started, last_cta, weights, wait_first = (float(v) for v in mid.split()[:4])
         assert weights < 0.0, f"no prefetch overlap: {line}"
-        assert started < weights and wait_first > 0.0, line
+        assert started < weights and started <= last_cta and wait_first > 0.0, line
