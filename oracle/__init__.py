@@ -37,9 +37,12 @@ def _load():
         lib.oracle_half_to_float.restype = ctypes.c_float
         lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
         lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_bfloat16_to_float.restype = ctypes.c_float
+        lib.oracle_bfloat16_to_float.argtypes = [ctypes.c_uint16]
         for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
                      "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64",
-                     "oracle_add_bias_residual_f64"):
+                     "oracle_add_bias_residual_f64", "oracle_dequant_f32_bf16", "oracle_gemm_f64_bf16",
+                     "oracle_gemm_f64_bf16_at"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -168,4 +171,78 @@ def add_bias_residual_f64(y: np.ndarray, bias: np.ndarray | None, residual: np.n
     r = None if residual is None else _f16(residual, (M, N))
     out = np.empty((M, N), dtype=np.float64)
     _load().oracle_add_bias_residual_f64(_p(y), _p(b), _p(r), ctypes.c_int(M), ctypes.c_int(N), _p(out))
+    return out
+
+
+# ---- bfloat16 activations and scales: numpy has no such type, so they travel as uint16 bit patterns ----------------
+
+def _bf16_bits(a, shape=None):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    if shape is not None:
+        assert a.shape == shape, (a.shape, shape)
+    return a
+
+
+def bfloat16_to_float(bits: int) -> float:
+    return float(_load().oracle_bfloat16_to_float(ctypes.c_uint16(bits)))
+
+
+def dequant_f32_bf16(qweight, qzeros, scales_bits, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp32[K, N] dequantised weights for bfloat16 scales given as uint16 bit patterns [G, N]."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales_bits = _bf16_bits(scales_bits, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    out = np.empty((K, N), dtype=np.float32)
+    _load().oracle_dequant_f32_bf16(_p(qweight), _p(qzeros), _p(scales_bits), _p(g), ctypes.c_int(K), ctypes.c_int(N),
+                                    ctypes.c_int(group_size), ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
+    return out
+
+
+def gemm_f64_bf16(x_bits, qweight, qzeros, scales_bits, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp64[M, N] = x . dequant(W) for bfloat16 x [M, K] and scales [G, N], both as uint16 bit patterns."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    x_bits = _bf16_bits(x_bits)
+    M = x_bits.shape[0]
+    assert x_bits.shape == (M, K)
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales_bits = _bf16_bits(scales_bits, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    out = np.empty((M, N), dtype=np.float64)
+    _load().oracle_gemm_f64_bf16(_p(x_bits), _p(qweight), _p(qzeros), _p(scales_bits), _p(g), ctypes.c_int(M),
+                                 ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size),
+                                 ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
+    return out
+
+
+def gemm_f64_bf16_at(x_bits, qweight, qzeros, scales_bits, g_idx, group_size: int, rows, cols,
+                     zeros_minus_one: bool = False) -> np.ndarray:
+    """The same sum as :func:`gemm_f64_bf16` for chosen (row, col) outputs only."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 8
+    G = K // group_size
+    x_bits = _bf16_bits(x_bits)
+    M = x_bits.shape[0]
+    assert x_bits.shape == (M, K)
+    qzeros = _i32(qzeros, (G, N // 8))
+    scales_bits = _bf16_bits(scales_bits, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    rows = _i32(rows)
+    cols = _i32(cols)
+    assert rows.shape == cols.shape and rows.ndim == 1
+    assert rows.min(initial=0) >= 0 and rows.max(initial=0) < M
+    assert cols.min(initial=0) >= 0 and cols.max(initial=0) < N
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _load().oracle_gemm_f64_bf16_at(_p(x_bits), _p(qweight), _p(qzeros), _p(scales_bits), _p(g), ctypes.c_int(M),
+                                    ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size),
+                                    ctypes.c_int(1 if zeros_minus_one else 0),
+                                    _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
     return out

@@ -226,3 +226,74 @@ void oracle_add_bias_residual_f64(const double *y, const uint16_t *bias, const u
             out[(size_t)m * N + n] = v;
         }
 }
+
+/* ---- format variant: bfloat16 activations and scales ------------------------------------------
+ * The paper's models run in fp16 (Section 4.1); the same checkpoints are also served with bfloat16
+ * activations and scales, and the method is unchanged: only the two 16-bit number formats differ.
+ * bfloat16 is the upper half of an IEEE-754 binary32 (1 sign, 8 exponent, 7 fraction bits), so its
+ * value is the binary32 whose upper 16 bits it is and whose lower 16 bits are zero.  The product
+ * float(q - z) * s stays exact in fp32 (4 bits times an 8-bit significand).
+ * zeros_plus = 0: the stored nibble is the zero point; 1: it is the zero point minus one. */
+float oracle_bfloat16_to_float(uint16_t b)
+{
+    uint32_t bits = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+static inline float dequant_one_bf16(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                                     const int32_t *g_idx, int N, int group_size, int zeros_plus, int k, int n)
+{
+    int g = group_of(g_idx, k, group_size);
+    int q = (int)nibble(qweight[(size_t)(k >> 3) * N + n], k & 7);
+    int z = (int)nibble(qzeros[(size_t)g * (N / 8) + (n >> 3)], n & 7) + zeros_plus;
+    float s = oracle_bfloat16_to_float(scales[(size_t)g * N + n]);
+    return (float)(q - z) * s;
+}
+
+void oracle_dequant_f32_bf16(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                             const int32_t *g_idx, int K, int N, int group_size, int zeros_plus, float *w_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            w_out[(size_t)k * N + n] = dequant_one_bf16(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+}
+
+/* y[m][n] in fp64, k ascending; x and scales are bfloat16 bits. */
+void oracle_gemm_f64_bf16(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                          const uint16_t *scales, const int32_t *g_idx,
+                          int M, int N, int K, int group_size, int zeros_plus, double *y_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; n++) {
+        for (int m = 0; m < M; m++) {
+            double acc = 0.0;
+            for (int k = 0; k < K; k++) {
+                float w = dequant_one_bf16(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+                acc += (double)oracle_bfloat16_to_float(x[(size_t)m * K + k]) * (double)w;
+            }
+            y_out[(size_t)m * N + n] = acc;
+        }
+    }
+}
+
+/* The same sum on chosen outputs only: y_out[i] = y[rows[i]][cols[i]]. */
+void oracle_gemm_f64_bf16_at(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                             const uint16_t *scales, const int32_t *g_idx,
+                             int M, int N, int K, int group_size, int zeros_plus,
+                             const int32_t *rows, const int32_t *cols, int count, double *y_out)
+{
+    (void)M;
+    #pragma omp parallel for schedule(static)
+    for (int i = 0; i < count; i++) {
+        int m = rows[i], n = cols[i];
+        double acc = 0.0;
+        for (int k = 0; k < K; k++) {
+            float w = dequant_one_bf16(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+            acc += (double)oracle_bfloat16_to_float(x[(size_t)m * K + k]) * (double)w;
+        }
+        y_out[i] = acc;
+    }
+}

@@ -143,6 +143,25 @@ def make_x(M: int, K: int, seed: int) -> np.ndarray:
     return _rng(seed).standard_normal((M, K), dtype=np.float32).astype(np.float16)
 
 
+def bf16_bits(a: np.ndarray) -> np.ndarray:
+    """Finite float values -> the bit patterns (uint16) of the nearest bfloat16, ties to even.  Inputs for the
+    bfloat16 variant travel in this form because numpy has no bfloat16 type."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = u + 0x7FFF + ((u >> 16) & 1)
+    return (u >> 16).astype(np.uint16)
+
+
+def make_x_bf16(M: int, K: int, seed: int) -> np.ndarray:
+    """Standard-normal activations as bfloat16 bit patterns [M, K]."""
+    return bf16_bits(_rng(seed).standard_normal((M, K), dtype=np.float32))
+
+
+def make_scales_bf16(G: int, N: int, seed: int) -> np.ndarray:
+    """The scale recipe of :func:`make_scales`, rounded to bfloat16 instead of fp16 (bit patterns [G, N])."""
+    r = _rng(seed)
+    return bf16_bits(SCALE_FLOOR + np.abs(r.standard_normal((G, N), dtype=np.float32) * SCALE_SIGMA))
+
+
 def algorithmic_bytes(M: int, K: int, N: int, group_size: int = GROUP_SIZE,
                       act_order: bool = False) -> int:
     """Bytes the matmul must move: packed weights, scales, packed zeros,

@@ -375,3 +375,120 @@ def test_add_bias_residual_reads_fp16_exactly_and_adds_in_double():
     assert out[0, 0] == 1e8 + 0.0999755859375 + 1.0                         # fp16(0.1) = 0.0999755859375; exact in fp64
     assert out[0, 1] == -3.0 + 65504.0 + 2.0 ** -24
     assert np.float32(1e8) + np.float32(0.0999755859375) == np.float32(1e8)   # fp32 would have dropped the bias
+
+
+# --------------------------------------------------------------------------- bfloat16 activations and scales
+def torch_bf16_bits_to_f64(bits):
+    """bfloat16 bit patterns -> float64 through torch's own bfloat16 type (a library routine, not the oracle's shift)."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16)
+    return t.to(torch.float64).numpy()
+
+
+def test_bfloat16_to_float_all_bit_patterns_against_torch():
+    bits = np.arange(65536, dtype=np.uint16)
+    want = torch_bf16_bits_to_f64(bits).astype(np.float32)
+    got = np.array([oracle.bfloat16_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+    # literal values from the format: 1 sign, 8 exponent (bias 127), 7 fraction bits
+    assert oracle.bfloat16_to_float(0x3FC0) == 1.5
+    assert oracle.bfloat16_to_float(0x4049) == 3.140625
+    assert oracle.bfloat16_to_float(0xC2F7) == -123.5
+    assert oracle.bfloat16_to_float(0x3080) == 2.0 ** -30        # far below the smallest fp16 subnormal
+    assert oracle.bfloat16_to_float(0x0001) == 2.0 ** -133       # the smallest subnormal
+
+
+def test_bf16_generator_rounds_to_nearest_even_like_torch():
+    import torch
+    a = np.concatenate([np.random.default_rng(5).standard_normal(4096).astype(np.float32) * 3,
+                        np.array([1.00390625, 1.01171875, 1.0, -0.0, 3.0e38, 1e-40, 0.002, 65504.0], dtype=np.float32)])
+    want = torch.from_numpy(a).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(wl.bf16_bits(a), want)
+    assert wl.bf16_bits(np.array([1.00390625], np.float32))[0] == 0x3F80     # tie: down to the even 1.0
+    assert wl.bf16_bits(np.array([1.01171875], np.float32))[0] == 0x3F82     # tie: up to the even 1.015625
+
+
+def test_bf16_dequant_hand_values(tiny):
+    """The hand-packed layer with bfloat16 scales typed as bit patterns, among them values fp16 cannot hold
+    (2^-30, 2^100) and one with all seven fraction bits set: every weight is (q - z) s exactly."""
+    q, z, gs = tiny["q"], tiny["z"], tiny["gs"]
+    s_bits = np.array([[0x3F80, 0x3F00, 0x3080, 0x7180, 0x3FFF, 0xBE80, 0x4000, 0x3E00],
+                       [0x3F00, 0x3F80, 0x4040, 0x3080, 0x3C00, 0x3FC0, 0xC000, 0x3D80]], dtype=np.uint16)
+    s = [[1.0, 0.5, 2.0 ** -30, 2.0 ** 100, 1.9921875, -0.25, 2.0, 0.125],
+         [0.5, 1.0, 3.0, 2.0 ** -30, 2.0 ** -7, 1.5, -2.0, 0.0625]]
+    w = oracle.dequant_f32_bf16(tiny["qweight"], tiny["qzeros"], s_bits, None, gs)
+    for k in range(16):
+        for n in range(8):
+            assert float(w[k, n]) == float(np.float32((int(q[k, n]) - int(z[k // gs, n])) * s[k // gs][n])), (k, n)
+    assert w[0, 0] == -1.0                    # (0 - 1) * 1
+    assert w[7, 4] == (int(q[7, 4]) - int(z[0, 4])) * 1.9921875
+    # the older zero convention: every weight one scale smaller
+    w1 = oracle.dequant_f32_bf16(tiny["qweight"], tiny["qzeros"], s_bits, None, gs, zeros_minus_one=True)
+    for k in range(16):
+        for n in range(8):
+            assert float(w1[k, n]) == float(np.float32((int(q[k, n]) - int(z[k // gs, n]) - 1) * s[k // gs][n])), (k, n)
+    # act-order: row k uses the scales and zeros of group g_idx[k]
+    wa = oracle.dequant_f32_bf16(tiny["qweight"], tiny["qzeros"], s_bits, tiny["g_idx"], gs)
+    for k in range(16):
+        g = int(tiny["g_idx"][k])
+        for n in range(8):
+            assert float(wa[k, n]) == float(np.float32((int(q[k, n]) - int(z[g, n])) * s[g][n])), (k, n)
+
+
+@pytest.mark.parametrize("act_order", [False, True])
+def test_bf16_gemm_matches_rational_brute_force(tiny, act_order):
+    """Exact rational arithmetic over the hand tables, with bfloat16 x and scales typed as bit patterns whose values
+    are written out beside them (so a wrong bit-field reading, or a detour through fp16, fails)."""
+    s_bits = np.array([[0x3F80, 0x3F00, 0x3080, 0x3FFF, 0x3E00, 0xBE80, 0x4000, 0x3E00],
+                       [0x3F00, 0x3F80, 0x4040, 0x3080, 0x3C00, 0x3FC0, 0xC000, 0x3D80]], dtype=np.uint16)
+    s = np.array([[1.0, 0.5, 2.0 ** -30, 1.9921875, 0.125, -0.25, 2.0, 0.125],
+                  [0.5, 1.0, 3.0, 2.0 ** -30, 2.0 ** -7, 1.5, -2.0, 0.0625]])
+    x_vals = np.array([[1.0] * 16,
+                       [0.5, -2.0, 3.0, 2.0 ** -20, 1.5, -0.0078125, 96.0, 1.0078125,
+                        -1.0, 0.25, 7.0, -3.0, 2.0 ** 20, 0.0, 1.25, -0.75]])
+    x_bits = wl.bf16_bits(x_vals)
+    assert np.array_equal(torch_bf16_bits_to_f64(x_bits), x_vals)          # all exactly representable
+    g_idx = tiny["g_idx"] if act_order else None
+    groups = [int(g) for g in tiny["g_idx"]] if act_order else [k // tiny["gs"] for k in range(16)]
+    want = brute_force_y(x_vals, tiny["q"], tiny["z"], s, groups)
+    got = oracle.gemm_f64_bf16(x_bits, tiny["qweight"], tiny["qzeros"], s_bits, g_idx, tiny["gs"])
+    for m in range(2):
+        for n in range(8):
+            assert abs(Fraction(float(got[m, n])) - want[m][n]) <= abs(want[m][n]) * Fraction(1, 2 ** 48), (m, n)
+    if not act_order:
+        assert got[0, 0] == 22.0          # as in the fp16 case: column 0 has scales 1 and 0.5
+
+
+@pytest.mark.parametrize("K,N,act,gs", [(4096, 4096, False, 128), (5120, 1024, True, 128), (512, 256, True, 32)])
+def test_bf16_gemm_against_library_fp64_matmul(K, N, act, gs):
+    """numpy's fp64 matmul over a vectorised unpack, with torch turning the bfloat16 bits into numbers."""
+    L = wl.make_linear(K, N, seed=wl.seed_for("pin-bf16", K, N, act), group_size=gs, act_order=act)
+    s_bits = wl.make_scales_bf16(K // gs, N, wl.seed_for("pin-bf16-s", K, N))
+    x_bits = wl.make_x_bf16(3, K, wl.seed_for("pin-bf16-x", K))
+    q, z = numpy_unpack(L.qweight, L.qzeros)
+    grp = L.g_idx if act else np.arange(K) // gs
+    s64 = torch_bf16_bits_to_f64(s_bits)
+    w = (q - z[grp]).astype(np.float64) * s64[grp]
+    want = torch_bf16_bits_to_f64(x_bits) @ w
+    got = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, gs)
+    assert np.allclose(got, want, rtol=1e-11, atol=1e-10)
+    assert np.array_equal(oracle.dequant_f32_bf16(L.qweight, L.qzeros, s_bits, L.g_idx, gs).astype(np.float64), w)
+    # the older zero convention: y_v1 = y - sum_g s[g, n] * sum_{k in g} x[m, k]
+    got1 = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, gs, zeros_minus_one=True)
+    xs = np.zeros((3, K // gs))
+    np.add.at(xs.T, grp, torch_bf16_bits_to_f64(x_bits).T)
+    assert np.allclose(got1, want - xs @ s64, rtol=0, atol=1e-9 * np.abs(want).max())
+
+
+def test_bf16_sampled_outputs_equal_full_product():
+    L = wl.make_linear(256, 64, seed=71, act_order=True)
+    s_bits = wl.make_scales_bf16(2, 64, 72)
+    x_bits = wl.make_x_bf16(6, 256, 73)
+    for zm in (False, True):
+        full = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, 128, zeros_minus_one=zm)
+        rows = np.array([0, 5, 3, 3, 1], dtype=np.int32)
+        cols = np.array([0, 63, 17, 18, 40], dtype=np.int32)
+        at = oracle.gemm_f64_bf16_at(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, 128, rows, cols, zeros_minus_one=zm)
+        assert np.array_equal(at, full[rows, cols])
