@@ -89,6 +89,13 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
  * each 128-column panel holds 64 gate columns and the 64 matching up columns; gptq_gemm_silu_mul needs that order and
  * gptq_gemm refuses it.  gptq_dequant_f32(repacked = 1) undoes it: its output is in checkpoint column order. */
 #define GPTQ_FORMAT_GATE_UP 2
+/* (No counterpart in the paper, whose models run in fp16 - Section 4.1.)  GPTQ_FORMAT_BF16: the scales are bfloat16
+ * (1 sign, 8 exponent, 7 fraction bits: the upper half of an fp32) instead of fp16, as in checkpoints served in
+ * bfloat16.  The repack moves the 16-bit words unchanged and records the flag; gptq_dequant_f32 then reads the scales
+ * as bfloat16 (the fp32 product float(q - z) * s is still exact), and the layer is multiplied with gptq_gemm_bf16, not
+ * gptq_gemm.  May be combined with GPTQ_FORMAT_ZEROS_MINUS_ONE; the fused epilogues (and so GPTQ_FORMAT_GATE_UP),
+ * gptq_gemm_host, gptq_gemm_host_batch and gptq_gemm_noalloc exist for fp16 layers only. */
+#define GPTQ_FORMAT_BF16 4
 /* gptq_dequant_f32 with a format for canonical inputs (repacked = 0; GPTQ_FORMAT_GATE_UP is refused there with
  * GPTQ_ERR_LAYOUT); with repacked = 1 the trailer decides and `format` must be 0 or equal to what the layer was
  * repacked with.  Unknown flag bits: GPTQ_ERR_LAYOUT. */
@@ -151,6 +158,20 @@ int gptq_set_workspace(void *ptr, size_t bytes);
 int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void *scales,
               const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
               void *stream);
+
+/* (No counterpart in the paper: the product of Sections 1 and 3 in the other 16-bit float format.)
+ * y bf16[M,N] = x bf16[M,K] . dequant(W)[K,N] for a layer repacked with GPTQ_FORMAT_BF16: x, y and the scales are
+ * bfloat16, everything else (arguments, layouts, act_order values, workspace, stream semantics, error codes, kernels
+ * chosen by M) as for gptq_gemm.  Up to 16 token rows the exact integers q - z are multiplied with x on the tensor
+ * cores (mma.sync, bf16 operands, fp32 sums) and the scale joins the fp32 group sums; above, each weight is rounded
+ * once to bfloat16 after scaling (relative error up to 2^-8) and multiplied by tcgen05.mma with bf16 operands; y is rounded
+ * once from the fp32 sum.  A layer of the other format (fp16 layer here, bfloat16 layer in gptq_gemm or any other
+ * matmul entry point) is refused: nothing is stored and gptq_check_status returns GPTQ_ERR_LAYOUT.
+ * Accuracy: the bar of gptq_gemm, |y - y_exact| <= 1e-2 sqrt(K/4096) + 1e-2 |y_exact|, holds with the same caveat; the
+ * output rounding alone is up to 2^-8 |y|. */
+int gptq_gemm_bf16(const void *x, const void *qweight, const void *qzeros, const void *scales,
+                   const int32_t *g_idx, void *y, int M, int N, int K, int group_size, int act_order,
+                   void *stream);
 
 /* act_order argument of the matmul entry points: 0 = groups are consecutive rows; 1 = act-order, the call first
  * gathers x into the sorted row order with g_idx (= gptq_repack's perm_out); GPTQ_ACT_ORDER_PRESORTED = act-order, but

@@ -24,6 +24,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 GPTQ_FORMAT_ZEROS_MINUS_ONE = 1
 GPTQ_FORMAT_GATE_UP = 2
+GPTQ_FORMAT_BF16 = 4
 GPTQ_ACT_ORDER_PRESORTED = 2
 GPTQ_OK = 0
 GPTQ_ERR_NULL = -1
@@ -71,6 +72,7 @@ _SIGNATURES = {
     "gptq_workspace_bytes": (_sz, [_i, _i, _i, _i, _i]),
     "gptq_set_workspace": (_i, [_vp, _sz]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_gemm_bf16": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_silu_mul": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_bias_residual": (_i, [_vp] * 8 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_silu_mul_scatter": (_i, [_vp] * 7 + [_i, _i, _i, _i, _i, _vp]),
@@ -182,6 +184,11 @@ def gptq_set_workspace(ptr, nbytes) -> int:
 def gptq_gemm(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
     return _lib.gptq_gemm(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N, K,
                           group_size, int(act_order), _stream(stream))
+
+
+def gptq_gemm_bf16(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
+    return _lib.gptq_gemm_bf16(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N, K,
+                               group_size, act_order, _stream(stream))
 
 
 def gptq_set_cta_pairs(enable) -> int:

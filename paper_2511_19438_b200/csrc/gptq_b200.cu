@@ -199,7 +199,7 @@ int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void 
                             float *w_out, int N, int K, int group_size, int act_order, int repacked, int format,
                             void *stream)
 {
-    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP)) return GPTQ_ERR_LAYOUT;
+    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP | GPTQ_FORMAT_BF16)) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !w_out || (act_order && !g_idx)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
     if (st) return st;
@@ -238,7 +238,7 @@ int gptq_repack_format(const int32_t *qweight, const int32_t *qzeros, const void
                        void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
                        int group_size, int act_order, int format, void *stream)
 {
-    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP)) return GPTQ_ERR_LAYOUT;
+    if (format & ~(GPTQ_FORMAT_ZEROS_MINUS_ONE | GPTQ_FORMAT_GATE_UP | GPTQ_FORMAT_BF16)) return GPTQ_ERR_LAYOUT;
     if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out) return GPTQ_ERR_NULL;
     if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
@@ -375,7 +375,7 @@ int gptq_set_workspace(void *ptr, size_t bytes)
 // y = x W (fuse == 0, y is [M, N]) or silu(gate) * up of y's column halves (fuse == 1, y is [M, N / 2])
 static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
                          void *y, int M, int N, int K, int group_size, int act_order, int fuse, const void *bias,
-                         const void *residual, const int32_t *out_index, void *stream)
+                         const void *residual, const int32_t *out_index, void *stream, int bf16 = 0)
 {
     if (act_order < 0 || act_order > GPTQ_ACT_ORDER_PRESORTED) return GPTQ_ERR_LAYOUT;
     if (!x || !qweight || !qzeros || !scales || !y || (act_order == 1 && !g_idx)) return GPTQ_ERR_NULL;
@@ -394,6 +394,7 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     cudaStream_t s = (cudaStream_t)stream;
     const __half *xin = (const __half *)x;
     const bool extras = bias != nullptr || residual != nullptr;
+    if (bf16 && (fuse || extras)) return GPTQ_ERR_UNSUPPORTED;     // the fused epilogues exist for fp16 only
     if (act_order == 1) {
         Workspace ws;
         {
@@ -408,21 +409,21 @@ static int gemm_dispatch(const void *x, const void *qweight, const void *qzeros,
     }
     const size_t ldy = fuse ? (size_t)N / 2 : (size_t)N;
     if (M >= kUmmaMinTokens) {
-        if (!fuse && !extras && g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
+        if (!fuse && !extras && !bf16 && g_use_cta_pairs.load() && umma2_applicable(M, N) && group_size == kGroup) {
             const Umma2Plan p2 = plan_umma2(M, N, K);
             return launch_umma2(xin, qweight, qzeros, scales, (__half *)y, M, N, K, p2, s);
         }
         // tcgen05 kernel: 32- to 256-token tiles
         const UmmaPlan pl = plan_umma(M, N, K, sms);
         return launch_umma(xin, qweight, qzeros, scales, (__half *)y, M, N, K, group_size, pl, fuse, (const __half *)bias,
-                           (const __half *)residual, out_index, s);
+                           (const __half *)residual, out_index, bf16, s);
     }
     for (int m0 = 0; m0 < M; m0 += kStreamKMaxRows) {
         const int rows = (M - m0) < kStreamKMaxRows ? (M - m0) : kStreamKMaxRows;
         const SplitKPlan pl = plan_splitk(rows, N, K, group_size, sms);
         st = launch_splitk(xin + (size_t)m0 * K, qweight, qzeros, scales, (__half *)y + (size_t)m0 * ldy, rows, N, K,
                            pl, fuse, (const __half *)bias,
-                           residual ? (const __half *)residual + (size_t)m0 * N : nullptr, out_index, s);
+                           residual ? (const __half *)residual + (size_t)m0 * N : nullptr, out_index, bf16, s);
         if (st) return st;
     }
     return GPTQ_OK;
@@ -434,6 +435,13 @@ int gptq_gemm(const void *x, const void *qweight, const void *qzeros, const void
               void *y, int M, int N, int K, int group_size, int act_order, void *stream)
 {
     return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, nullptr, nullptr, nullptr, stream);
+}
+
+int gptq_gemm_bf16(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                   void *y, int M, int N, int K, int group_size, int act_order, void *stream)
+{
+    return gemm_dispatch(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, 0, nullptr, nullptr, nullptr, stream,
+                         1);
 }
 
 int gptq_gemm_bias_residual(const void *x, const void *qweight, const void *qzeros, const void *scales,

@@ -1,6 +1,7 @@
 // Shared definitions of the gptq_b200 CUDA library: the tiled weight layout, PTX wrappers
 // and the device status word.  sm_100a only.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -47,6 +48,8 @@ constexpr int kTrailerBytes = 16;
 constexpr uint32_t kTrailerMagic = 0x51545047u;   // "GPTQ"
 constexpr uint32_t kFormatZerosMinusOne = 1u;     // == GPTQ_FORMAT_ZEROS_MINUS_ONE
 constexpr uint32_t kFormatGateUp = 2u;            // == GPTQ_FORMAT_GATE_UP: column halves interleaved per panel
+constexpr uint32_t kFormatBf16 = 4u;              // == GPTQ_FORMAT_BF16: the scales are bfloat16 (so are x and y of the matmul)
+constexpr uint32_t kFormatMask = 7u;
 // With kFormatGateUp a layer's columns are [gate | up] (N / 2 each) and tiled panel p holds gate columns
 // 64 p .. 64 p + 63 in its first half and the matching up columns in its second, so that one CTA sees both.
 __host__ __device__ inline int gate_up_source_column(int nt, int N)      // tiled column -> checkpoint column
@@ -256,6 +259,84 @@ __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b)
     uint32_t d;
     asm("mul.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
+}
+__device__ __forceinline__ uint32_t bsub2_u32(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("sub.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t bmul2_u32(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// The four 16-bit pairs of exact integers q - z held by one packed word (rows e = 0,1 / 2,3 / 4,5 / 6,7 of its column),
+// in the 16-bit float format of the matmul.  fp16 (10 fraction bits): the low nibble of a byte becomes 1024 + q and the
+// high nibble, left in place, 1024 + 16 q with a second magic exponent (64 + q), so one shift serves four pairs; zlo and
+// zhi are the matching constants 1024 + z and 64 + z.  bfloat16 has 7 fraction bits, a nibble in bits 4..7 would run
+// into the exponent, so every pair is shifted down first and becomes 128 + q; zlo = 128 + z serves all four.
+template <bool BF>
+__device__ __forceinline__ void nibble_pairs_minus_zero(uint32_t w, uint32_t zlo, uint32_t zhi, uint32_t (&o)[4])
+{
+    constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u;
+    if constexpr (BF) {
+        constexpr uint32_t MAGIC = 0x43004300u;
+        o[0] = bsub2_u32(lop3_and_or(w, LO, MAGIC), zlo);
+        o[1] = bsub2_u32(lop3_and_or(w >> 4, LO, MAGIC), zlo);
+        o[2] = bsub2_u32(lop3_and_or(w >> 8, LO, MAGIC), zlo);
+        o[3] = bsub2_u32(lop3_and_or(w >> 12, LO, MAGIC), zlo);
+    } else {
+        constexpr uint32_t MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
+        o[0] = hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo);
+        o[1] = hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi);
+        w >>= 8;
+        o[2] = hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo);
+        o[3] = hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi);
+    }
+}
+// the constants for zero point z (0..16): both halves of a pair hold the same column
+template <bool BF>
+__device__ __forceinline__ void zero_constants(uint32_t z, uint32_t &zlo, uint32_t &zhi)
+{
+    if constexpr (BF) {
+        zlo = (z * 0x00010001u) | 0x43004300u;      // 128 + z
+        zhi = zlo;
+    } else {
+        zlo = (z * 0x00010001u) | 0x64006400u;      // 1024 + z
+        zhi = (z * 0x00100010u) | 0x54005400u;      // 64 + z
+    }
+}
+// a pair of 16-bit floats of the matmul's format -> two floats
+template <bool BF>
+__device__ __forceinline__ float2 pair_to_float2(uint32_t v)
+{
+    if constexpr (BF) return make_float2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+    else return __half22float2(*reinterpret_cast<const __half2 *>(&v));
+}
+// one float -> the 16 bits of the matmul's output format, round to nearest even
+template <bool BF>
+__device__ __forceinline__ unsigned short float_to_out16(float v)
+{
+    if constexpr (BF) return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+    else return __half_as_ushort(__float2half_rn(v));
+}
+// stores one element of y (declared as fp16 storage; with BF the 16 bits are a bfloat16)
+template <bool BF>
+__device__ __forceinline__ void store_out16(__half *p, float v)
+{
+    if constexpr (BF) *reinterpret_cast<unsigned short *>(p) = float_to_out16<true>(v);
+    else *p = __float2half_rn(v);
+}
+// D(16x8, f32) = A(16x16, bf16, row) * B(16x8, bf16, col) + C
+__device__ __forceinline__ void mma_m16n8k16_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                  uint32_t b0, uint32_t b1)
+{
+    asm(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // D(16x8, f32) = A(16x16, f16, row) * B(16x8, f16, col) + C
 __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,

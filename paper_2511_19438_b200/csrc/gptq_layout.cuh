@@ -47,9 +47,14 @@ int launch_unpack_u8(const int32_t *qweight, const int32_t *qzeros, uint8_t *q_o
 
 // ------------------------------------------------------------------------------ dequant fp32
 // One thread per (k, n).  float(q - z) * float(s): a single fp32 multiply whose result is exact.
+// A scale is 16 bits of fp16 or, with the bfloat16 format flag, of bfloat16 (the upper half of an fp32).
+__device__ __forceinline__ float scale_to_float(const __half *p, bool bf16)
+{
+    return bf16 ? __uint_as_float((uint32_t)__half_as_ushort(*p) << 16) : __half2float(*p);
+}
 __global__ void dequant_canonical_kernel(const int32_t *__restrict__ qweight, const int32_t *__restrict__ qzeros,
                                          const __half *__restrict__ scales, const int32_t *__restrict__ g_idx,
-                                         float *__restrict__ w_out, int N, int K, int group_size, int z_add)
+                                         float *__restrict__ w_out, int N, int K, int group_size, int z_add, int bf16)
 {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)K * N) return;
@@ -57,7 +62,7 @@ __global__ void dequant_canonical_kernel(const int32_t *__restrict__ qweight, co
     int g = g_idx ? g_idx[k] : k / group_size;
     int q = (int)(((uint32_t)qweight[(size_t)(k >> 3) * N + n] >> (4 * (k & 7))) & 15u);
     int z = (int)(((uint32_t)qzeros[(size_t)g * (N / 8) + (n >> 3)] >> (4 * (n & 7))) & 15u) + z_add;
-    w_out[idx] = __fmul_rn((float)(q - z), __half2float(scales[(size_t)g * N + n]));
+    w_out[idx] = __fmul_rn((float)(q - z), scale_to_float(scales + (size_t)g * N + n, bf16 != 0));
 }
 
 // Tiled layout: thread per (sorted row i, column n); the row goes back to its original index.
@@ -78,7 +83,7 @@ __global__ void dequant_tiled_kernel(const uint8_t *__restrict__ qweight, const 
     int q = (int)((word >> (4 * slot)) & 15u);
     uint8_t zb = qzeros[repacked_zero_byte(grp, nt, groups, &hi)];
     int z = (hi ? (zb >> 4) : (zb & 15)) + (int)(tr->flags & kFormatZerosMinusOne);
-    float s = __half2float(scales[repacked_scale_index(grp, nt, groups)]);
+    float s = scale_to_float(scales + repacked_scale_index(grp, nt, groups), (tr->flags & kFormatBf16) != 0);
     int k = perm ? perm[i] : i;
     w_out[(size_t)k * N + n] = __fmul_rn((float)(q - z), s);
 }
@@ -97,7 +102,8 @@ int launch_dequant_f32(const void *qweight, const void *qzeros, const void *scal
     else
         dequant_canonical_kernel<<<blocks, T, 0, s>>>((const int32_t *)qweight, (const int32_t *)qzeros,
                                                       (const __half *)scales, act_order ? g_idx : nullptr, w_out,
-                                                      N, K, group_size, (format & (int)kFormatZerosMinusOne) ? 1 : 0);
+                                                      N, K, group_size, (format & (int)kFormatZerosMinusOne) ? 1 : 0,
+                                                      (format & (int)kFormatBf16) ? 1 : 0);
     return record_cuda_error(cudaGetLastError());
 }
 

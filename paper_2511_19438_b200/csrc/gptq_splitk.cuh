@@ -123,7 +123,7 @@ constexpr int kSplitKWideCtas = 4;
 #else
 constexpr int kSplitKWideCtas = 3;
 #endif
-template <int MT, int SUB>
+template <int MT, int SUB, bool BF = false>
 __global__ void __launch_bounds__(kStreamKThreads, (MT == 1 && SUB == 1) ? kSplitKWideCtas : 3)
 splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 {
@@ -224,7 +224,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
         const uint32_t z_add = flags & kFormatZerosMinusOne;
         // a layer tiled for the fused gate/up epilogue must be used with it, and only with it: otherwise nothing is
         // stored and the status word says so
-        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0);
+        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0) && ((flags & kFormatBf16) != 0) == BF;
         if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         pdl_wait();
         const int r = token_row_of_slot(g);
@@ -243,12 +243,12 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
             if (it == 0 && threadIdx.x == 0) GPTQ_TRACE_MIN(a.trace_slot, first_data);
 
             ItemSums<MT, SUB> sums;
-            consume_item<MT, SUB>(st, w_off, s_off, z_off, x_off0, x_off1, z_add, sums);
+            consume_item<MT, SUB, BF>(st, w_off, s_off, z_off, x_off0, x_off1, z_add, sums);
             // release the stage, then fold the group sums into the running sums with the groups' scales
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
             if (++s == stages) { s = 0; phase ^= 1u; }
-            fold_item<MT, SUB>(acc, sums);
+            fold_item<MT, SUB, BF>(acc, sums);
         }
     }
 
@@ -273,7 +273,7 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = mt * 8 + ((i & 1) ? m_hi : m_lo);
-                        if (m < a.M) yp[(size_t)m * a.N + 8 * (i >> 1)] = __float2half_rn(acc[mt][i] + addend(m, p * kPanel + col + 8 * (i >> 1)));
+                        if (m < a.M) store_out16<BF>(yp + (size_t)m * a.N + 8 * (i >> 1), acc[mt][i] + addend(m, p * kPanel + col + 8 * (i >> 1)));
                     }
             } else {
                 // warps 4-7 hold the up columns of the gate columns of warps 0-3: hand them over through the
@@ -298,8 +298,8 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                             if (m < a.M) {
                                 const float up = lds_f32(hand + (uint32_t)(m * 64 + col + 8 * (i >> 1)) * 4u);
                                 const int oc = p * 64 + col + 8 * (i >> 1);
-                                a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
-                                    __float2half_rn(silu_mul(acc[mt][i], up));
+                                store_out16<BF>(a.y + (size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc),
+                                                silu_mul(acc[mt][i], up));
                             }
                         }
                 }
@@ -354,11 +354,11 @@ splitk_kernel(const SplitKArgs a, const __grid_constant__ CUtensorMap x_map)
                 for (int m = threadIdx.x >> jsh; m < a.M; m += kConsumerThreads >> jsh) {
                     if (!a.fuse) {
                         const int n = p * kPanel + lo + j;
-                        a.y[(size_t)m * a.N + n] = __float2half_rn(slice_sum(m, j) + addend(m, n));
+                        store_out16<BF>(a.y + (size_t)m * a.N + n, slice_sum(m, j) + addend(m, n));
                     } else {
                         const int oc = p * 64 + lo + j;
-                        a.y[(size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc)] =
-                            __float2half_rn(silu_mul(slice_sum(m, j), slice_sum(m, hwmax + j)));
+                        store_out16<BF>(a.y + (size_t)m * (a.N / 2) + (a.out_index ? a.out_index[oc] : oc),
+                                        silu_mul(slice_sum(m, j), slice_sum(m, hwmax + j)));
                     }
                 }
             }
@@ -428,11 +428,11 @@ SplitKPlan plan_splitk(int m_rows, int N, int K, int group_size, int sm_count)
     return pl;
 }
 
-template <int MT, int SUB>
+template <int MT, int SUB, bool BF>
 static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, const SplitKPlan &plan, cudaStream_t s)
 {
     static int configured_smem[64] = {};
-    const int cfg_st = ensure_dynamic_smem((const void *)splitk_kernel<MT, SUB>, configured_smem, plan.smem_bytes);
+    const int cfg_st = ensure_dynamic_smem((const void *)splitk_kernel<MT, SUB, BF>, configured_smem, plan.smem_bytes);
     if (cfg_st) return cfg_st;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)plan.ctas);
@@ -454,12 +454,12 @@ static int launch_splitk_mt(const SplitKArgs &args, const CUtensorMap &x_map, co
     attr[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
     cfg.attrs = attr;
     cfg.numAttrs = 3;
-    return record_cuda_error(cudaLaunchKernelEx(&cfg, splitk_kernel<MT, SUB>, args, x_map));
+    return record_cuda_error(cudaLaunchKernelEx(&cfg, splitk_kernel<MT, SUB, BF>, args, x_map));
 }
 
 int launch_splitk(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y,
                   int M, int N, int K, const SplitKPlan &plan, int fuse, const __half *bias, const __half *residual,
-                  const int32_t *out_index, cudaStream_t s)
+                  const int32_t *out_index, int bf16, cudaStream_t s)
 {
     SplitKArgs args;
     args.qweight = (const uint8_t *)qweight;
@@ -489,13 +489,20 @@ int launch_splitk(const __half *x, const void *qweight, const void *qzeros, cons
     int st = make_tensor_map_2d(&x_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, x, (uint64_t)K, (uint64_t)M,
                                 (uint64_t)K * sizeof(__half), 64, (uint32_t)plan.m_tile, CU_TENSOR_MAP_SWIZZLE_128B);
     if (st) return st;
-    switch (plan.m_tile * 10 + plan.sub) {
-    case 81: return launch_splitk_mt<1, 1>(args, x_map, plan, s);
-    case 82: return launch_splitk_mt<1, 2>(args, x_map, plan, s);
-    case 84: return launch_splitk_mt<1, 4>(args, x_map, plan, s);
-    case 161: return launch_splitk_mt<2, 1>(args, x_map, plan, s);
-    case 162: return launch_splitk_mt<2, 2>(args, x_map, plan, s);
-    case 164: return launch_splitk_mt<2, 4>(args, x_map, plan, s);
+    // (the tensor map only moves 16-bit words and zero-fills rows beyond M: the same for fp16 and bfloat16)
+    switch ((bf16 ? 1000 : 0) + plan.m_tile * 10 + plan.sub) {
+    case 81: return launch_splitk_mt<1, 1, false>(args, x_map, plan, s);
+    case 82: return launch_splitk_mt<1, 2, false>(args, x_map, plan, s);
+    case 84: return launch_splitk_mt<1, 4, false>(args, x_map, plan, s);
+    case 161: return launch_splitk_mt<2, 1, false>(args, x_map, plan, s);
+    case 162: return launch_splitk_mt<2, 2, false>(args, x_map, plan, s);
+    case 164: return launch_splitk_mt<2, 4, false>(args, x_map, plan, s);
+    case 1081: return launch_splitk_mt<1, 1, true>(args, x_map, plan, s);
+    case 1082: return launch_splitk_mt<1, 2, true>(args, x_map, plan, s);
+    case 1084: return launch_splitk_mt<1, 4, true>(args, x_map, plan, s);
+    case 1161: return launch_splitk_mt<2, 1, true>(args, x_map, plan, s);
+    case 1162: return launch_splitk_mt<2, 2, true>(args, x_map, plan, s);
+    case 1164: return launch_splitk_mt<2, 4, true>(args, x_map, plan, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }

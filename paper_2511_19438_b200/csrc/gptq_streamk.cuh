@@ -55,7 +55,8 @@ struct ItemSums {
     float g[SUB][MT][4];
     uint32_t sc[SUB];
 };
-template <int MT, int SUB>
+// BF: x and the scales are bfloat16 instead of fp16 (the exact integers q - z are built as bfloat16 too).
+template <int MT, int SUB, bool BF = false>
 __device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32_t s_off, uint32_t z_off,
                                              uint32_t x_off0, uint32_t x_off1, uint32_t z_add, ItemSums<MT, SUB> &out)
 {
@@ -81,10 +82,27 @@ __device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32
                 out.sc[sub] = lds32(st + s_off + sub * kItemSBytes);
                 const uint32_t zb = lds8(st + z_off + sub * kItemZBytes);
                 const uint32_t zA = (zb & 15u) + z_add, zB = (zb >> 4) + z_add;   // up to 16: still exact below
-                zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
-                zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+                if constexpr (BF) {
+                    zero_constants<true>(zA, zloA, zhiA);
+                    zero_constants<true>(zB, zloB, zhiB);
+                } else {
+                    zloA = (zA * 0x00010001u) | MAGIC_LO, zhiA = (zA * 0x00100010u) | MAGIC_HI;
+                    zloB = (zB * 0x00010001u) | MAGIC_LO, zhiB = (zB * 0x00100010u) | MAGIC_HI;
+                }
             }
             uint32_t wA = j ? wq.y : wq.x, wB = j ? wq.w : wq.z;
+            if constexpr (BF) {
+                uint32_t pA[4], pB[4];    // pairs of rows (0,1) (2,3) (4,5) (6,7) of columns g and g + 8
+                nibble_pairs_minus_zero<true>(wA, zloA, zhiA, pA);
+                nibble_pairs_minus_zero<true>(wB, zloB, zhiB, pB);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const uint4 xb = lds128(st + blk * kXTile + mt * 1024 + (j ? x_off1 : x_off0));
+                    mma_m16n8k16_bf16(out.g[sub][mt], pA[0], pB[0], pA[1], pB[1], xb.x, xb.y);
+                    mma_m16n8k16_bf16(out.g[sub][mt], pA[2], pB[2], pA[3], pB[3], xb.z, xb.w);
+                }
+                continue;
+            }
             const uint32_t a0 = hsub2_u32(lop3_and_or(wA, LO, MAGIC_LO), zloA);
             const uint32_t a2 = hsub2_u32(lop3_and_or(wA, HI, MAGIC_HI), zhiA);
             const uint32_t a1 = hsub2_u32(lop3_and_or(wB, LO, MAGIC_LO), zloB);
@@ -105,12 +123,12 @@ __device__ __forceinline__ void consume_item(uint32_t st, uint32_t w_off, uint32
     }
 }
 // folds the item's group sums into the running sums with each group's scales
-template <int MT, int SUB>
+template <int MT, int SUB, bool BF = false>
 __device__ __forceinline__ void fold_item(float (&acc)[MT][4], const ItemSums<MT, SUB> &it)
 {
 #pragma unroll
     for (int sub = 0; sub < SUB; ++sub) {
-        const float2 sf = __half22float2(*reinterpret_cast<const __half2 *>(&it.sc[sub]));
+        const float2 sf = pair_to_float2<BF>(it.sc[sub]);
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
             acc[mt][0] = fmaf(sf.x, it.g[sub][mt][0], acc[mt][0]);
@@ -205,7 +223,7 @@ streamk_kernel(const StreamKArgs a, const __grid_constant__ CUtensorMap x_map)
     // -------------------------------------------------------------------- consumer warps
     const uint32_t z_add = flags & kFormatZerosMinusOne;   // weights-side data: no need to wait
     // this kernel has no fused gate/up epilogue: a layer tiled for one is computed but not stored, and reported
-    const bool layout_ok = (flags & kFormatGateUp) == 0;
+    const bool layout_ok = (flags & (kFormatGateUp | kFormatBf16)) == 0;   // fp16, plain column order only
     if (!layout_ok && threadIdx.x == 0) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
     pdl_wait();
     const int g = lane >> 2, t4 = lane & 3;

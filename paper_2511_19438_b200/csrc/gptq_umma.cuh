@@ -132,9 +132,17 @@ __host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N)
     return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// the same with bfloat16 A and B: operand format fields (bits 7..9 and 10..12) 1 instead of 0
+constexpr uint32_t kUmmaIdescBf16 = (1u << 7) | (1u << 10);
+
 __device__ __forceinline__ void sts_f16(uint32_t addr, __half v)
 {
     asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(v)) : "memory");
+}
+
+__device__ __forceinline__ void sts_b16(uint32_t addr, unsigned short v)
+{
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
 }
 
 __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr)
@@ -180,7 +188,7 @@ __host__ __device__ constexpr int umma_tmem_cols(int TOK, int NA, int NP, int IS
     return c;
 }
 
-template <int TOK, int NA, int NP, int SETS, int SUB>
+template <int TOK, int NA, int NP, int SETS, int SUB, bool BF = false>
 __global__ void __launch_bounds__(umma_threads(TOK, NP, SETS), (NP > 1 || TOK > 128) ? 1 : TOK <= 32 ? 3 : 2)
 umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map)
 {
@@ -302,7 +310,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
     } else if (warp <= ISS) {
         // ---------------------------------------------------------------- MMA issue (one thread per issuing warp)
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_f16(128, TOK);
+            constexpr uint32_t idesc = umma_idesc_f16(128, TOK) | (BF ? kUmmaIdescBf16 : 0u);
             // Every instruction this thread issues costs it 60-110 cycles (a tcgen05.mma about 60, a commit
             // about 80, a barrier wait about 100 even when the barrier is ready), so the loop is kept to one wait
             // per panel, the four MMAs and one commit per K64 block.  It does not wait for the slot's TMA data
@@ -387,7 +395,7 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
         // (the format flags are looked at only now, with the first scales and zeros already on their way)
         const uint32_t z_add = flags & kFormatZerosMinusOne;   // stored zero points one too small
         // a layer tiled for the fused gate/up epilogue must be used with it, and only with it (else: nothing is stored)
-        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0);
+        layout_ok = ((flags & kFormatGateUp) != 0) == (a.fuse != 0) && ((flags & kFormatBf16) != 0) == BF;
         if (!layout_ok && threadIdx.x == 32 * kFirstDq) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, MAGIC_LO = 0x64006400u, MAGIC_HI = 0x54005400u;
         // set k takes groups k, k + SETS, ...: K64 blocks 2 gg and 2 gg + 1; block b lives in ring refill b / BPS
@@ -413,8 +421,12 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 for (int sub = 0; sub < SUB; ++sub) {
                     s2[sub] = sc_next[sub] * 0x00010001u;
                     const uint32_t z = (h ? (zb_next[sub] >> 4) : (zb_next[sub] & 15u)) + z_add;   // up to 16: still exact
-                    zlo[sub] = (z * 0x00010001u) | MAGIC_LO;
-                    zhi[sub] = (z * 0x00100010u) | MAGIC_HI;
+                    if constexpr (BF) {
+                        zero_constants<true>(z, zlo[sub], zhi[sub]);
+                    } else {
+                        zlo[sub] = (z * 0x00010001u) | MAGIC_LO;
+                        zhi[sub] = (z * 0x00100010u) | MAGIC_HI;
+                    }
                 }
                 if (b + 2 * SETS < NB) load_sz((b >> 1) + SETS, sc_next, zb_next);   // this set's next item
             }
@@ -441,6 +453,14 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 for (int t4 = 0; t4 < 4; ++t4) {
                     uint32_t w = jj ? wv[t4].y : wv[t4].x;       // rows 32 jj + 8 t4 + (0..7), TMEM columns 16 jj + 4 t4 + (0..3)
                     uint32_t *o = r + 16 * jj + 4 * t4;
+                    if constexpr (BF) {
+                        // bfloat16: exact q - z, then one rounding in the product with the scale
+                        uint32_t d[4];
+                        nibble_pairs_minus_zero<true>(w, zlo_b[jj], zhi_b[jj], d);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = bmul2_u32(d[e], s2_b[jj]);
+                        continue;
+                    }
                     o[0] = hmul2_u32(hsub2_u32(lop3_and_or(w, LO, MAGIC_LO), zlo_b[jj]), s2_b[jj]);
                     o[1] = hmul2_u32(hsub2_u32(lop3_and_or(w, HI, MAGIC_HI), zhi_b[jj]), s2_b[jj]);
                     w >>= 8;
@@ -513,7 +533,8 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                     }
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
+                        if constexpr (BF) sts_b16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), float_to_out16<true>(__uint_as_float(r[i])));
+                        else sts_f16(stg + (uint32_t)(i * (kPanel * 2) + n * 2), __float2half_rn(__uint_as_float(r[i])));
                 }
                 named_bar_sync(bar_id, 128);
                 if (ok && !a.fuse) {
@@ -603,10 +624,15 @@ umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const _
                 return sum;
             };
             auto store4 = [&](__half *dst, float4 v) {
-                const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
                 uint2 out;
-                out.x = *reinterpret_cast<const uint32_t *>(&lo);
-                out.y = *reinterpret_cast<const uint32_t *>(&hi);
+                if constexpr (BF) {
+                    out.x = (uint32_t)float_to_out16<true>(v.x) | ((uint32_t)float_to_out16<true>(v.y) << 16);
+                    out.y = (uint32_t)float_to_out16<true>(v.z) | ((uint32_t)float_to_out16<true>(v.w) << 16);
+                } else {
+                    const __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
+                    out.x = *reinterpret_cast<const uint32_t *>(&lo);
+                    out.y = *reinterpret_cast<const uint32_t *>(&hi);
+                }
                 *reinterpret_cast<uint2 *>(dst) = out;
             };
             const int c_lo = rank * kPanel / S, width = (rank + 1) * kPanel / S - c_lo;   // width is 16, 32 or 64
@@ -756,11 +782,11 @@ inline UmmaPlan plan_umma(int M, int N, int K, int sm_count)
     return pl;
 }
 
-template <int TOK, int NP, int SETS, int SUB>
+template <int TOK, int NP, int SETS, int SUB, bool BF>
 static int launch_umma_sub(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
                            const UmmaPlan &plan, int ctas, cudaStream_t s)
 {
-    auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS, SUB>;
+    auto kernel = umma_kernel<TOK, umma_a_stages(TOK, NP), NP, SETS, SUB, BF>;
     static int configured_smem[64] = {};
     const int cfg_st = ensure_dynamic_smem((const void *)kernel, configured_smem, plan.smem_bytes);
     if (cfg_st) return cfg_st;
@@ -783,19 +809,22 @@ static int launch_umma_sub(const UmmaArgs &args, const CUtensorMap &w_map, const
 
 template <int TOK, int NP, int SETS>
 static int launch_umma_tok(const UmmaArgs &args, const CUtensorMap &w_map, const CUtensorMap &x_map,
-                           const UmmaPlan &plan, int ctas, int sub, cudaStream_t s)
+                           const UmmaPlan &plan, int ctas, int sub, int bf16, cudaStream_t s)
 {
-    switch (sub) {
-    case 1: return launch_umma_sub<TOK, NP, SETS, 1>(args, w_map, x_map, plan, ctas, s);
-    case 2: return launch_umma_sub<TOK, NP, SETS, 2>(args, w_map, x_map, plan, ctas, s);
-    case 4: return launch_umma_sub<TOK, NP, SETS, 4>(args, w_map, x_map, plan, ctas, s);
+    switch (sub + (bf16 ? 10 : 0)) {
+    case 1: return launch_umma_sub<TOK, NP, SETS, 1, false>(args, w_map, x_map, plan, ctas, s);
+    case 2: return launch_umma_sub<TOK, NP, SETS, 2, false>(args, w_map, x_map, plan, ctas, s);
+    case 4: return launch_umma_sub<TOK, NP, SETS, 4, false>(args, w_map, x_map, plan, ctas, s);
+    case 11: return launch_umma_sub<TOK, NP, SETS, 1, true>(args, w_map, x_map, plan, ctas, s);
+    case 12: return launch_umma_sub<TOK, NP, SETS, 2, true>(args, w_map, x_map, plan, ctas, s);
+    case 14: return launch_umma_sub<TOK, NP, SETS, 4, true>(args, w_map, x_map, plan, ctas, s);
     default: return GPTQ_ERR_UNSUPPORTED;
     }
 }
 
 int launch_umma(const __half *x, const void *qweight, const void *qzeros, const void *scales, __half *y, int M, int N,
                 int K, int group_size, const UmmaPlan &plan, int fuse, const __half *bias, const __half *residual,
-                const int32_t *out_index, cudaStream_t s)
+                const int32_t *out_index, int bf16, cudaStream_t s)
 {
     UmmaArgs args;
     args.scales = (const uint8_t *)scales;
@@ -828,10 +857,10 @@ int launch_umma(const __half *x, const void *qweight, const void *qzeros, const 
     if (st) return st;
     auto launch = [&](const UmmaArgs &la, int ctas) {
         switch (plan.tok) {
-        case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
-        case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
-        case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
-        case 256: return launch_umma_tok<256, 1, 2>(la, w_map, x_map, plan, ctas, sub, s);
+        case 32: return launch_umma_tok<32, 1, 2>(la, w_map, x_map, plan, ctas, sub, bf16, s);
+        case 64: return launch_umma_tok<64, 1, 2>(la, w_map, x_map, plan, ctas, sub, bf16, s);
+        case 128: return launch_umma_tok<128, 1, 2>(la, w_map, x_map, plan, ctas, sub, bf16, s);
+        case 256: return launch_umma_tok<256, 1, 2>(la, w_map, x_map, plan, ctas, sub, bf16, s);
         default: return (int)GPTQ_ERR_UNSUPPORTED;
         }
     };

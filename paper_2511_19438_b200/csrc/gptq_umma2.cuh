@@ -198,7 +198,7 @@ umma2_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap w_map, const 
         uint32_t s2 = 0, zlo = MAGIC_LO, zhi = MAGIC_HI;
         const uint32_t z_add = flags & kFormatZerosMinusOne;   // stored zero points one too small
         // this kernel has no fused gate/up epilogue: a layer tiled for one is multiplied but not stored, and reported
-        const bool layout_ok = (flags & kFormatGateUp) == 0;
+        const bool layout_ok = (flags & (kFormatGateUp | kFormatBf16)) == 0;   // fp16, plain column order only
         if (!layout_ok && threadIdx.x == 64) atomicMax(&g_device_status, (int)kStatusLayoutMismatch);
         bool ok = true;
         for (; b < NB && ok; b += ((b & 1) ? 2 * SETS - 1 : 1)) {

@@ -33,16 +33,24 @@ def to_device(a: np.ndarray, device="cuda") -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a)).to(device)
 
 
-def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda", gate_up: bool = False) -> DeviceLinear:
+def upload_and_repack(L: QuantLinear, keep_canonical: bool = False, device="cuda", gate_up: bool = False,
+                      scales_bf16_bits: np.ndarray | None = None) -> DeviceLinear:
+    """``scales_bf16_bits`` (uint16 [G, N]) replaces the layer's fp16 scales by bfloat16 ones and marks the tiled
+    layer as a bfloat16 layer (to be used with :func:`gemm_bf16`)."""
     qw = to_device(L.qweight, device)
     qz = to_device(L.qzeros, device)
-    sc = to_device(L.scales, device)
+    if scales_bf16_bits is not None:
+        assert scales_bf16_bits.dtype == np.uint16 and scales_bf16_bits.shape == (L.K // L.group_size, L.N)
+        sc = to_device(scales_bf16_bits.view(np.int16), device).view(torch.bfloat16)
+    else:
+        sc = to_device(L.scales, device)
     gi = to_device(L.g_idx, device) if L.act_order else None
     qw_t = torch.empty(B.gptq_repack_bytes(0, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     qz_t = torch.empty(B.gptq_repack_bytes(1, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     sc_t = torch.empty(B.gptq_repack_bytes(2, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
     perm = torch.empty(L.K, dtype=torch.int32, device=device) if L.act_order else None
     fmt = (B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0) | (B.GPTQ_FORMAT_GATE_UP if gate_up else 0)
+    fmt |= B.GPTQ_FORMAT_BF16 if scales_bf16_bits is not None else 0
     B.check(B.gptq_repack_format(qw, qz, sc, gi, qw_t, qz_t, sc_t, perm, L.N, L.K, L.group_size, L.act_order, fmt),
             "gptq_repack_format")
     torch.cuda.current_stream().synchronize()
@@ -77,6 +85,27 @@ def gemm(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream
         y = torch.empty((M, D.N), dtype=torch.float16, device=x.device)
     B.check(B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, D.N, D.K, D.group_size,
                         D.act_order, stream), "gptq_gemm")
+    return y
+
+
+def bf16_from_bits(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bit patterns -> a bfloat16 tensor on the device (no conversion: the same 16 bits)."""
+    return to_device(np.ascontiguousarray(bits).view(np.int16), device).view(torch.bfloat16)
+
+
+def bits_of_bf16(t: torch.Tensor) -> np.ndarray:
+    """A bfloat16 tensor -> its bit patterns as a numpy uint16 array."""
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def gemm_bf16(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """y = x . dequant(W) through gptq_gemm_bf16 (x bfloat16 [M, K] on the device, D repacked with bfloat16 scales)."""
+    assert x.dtype == torch.bfloat16
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, D.N), dtype=torch.bfloat16, device=x.device)
+    B.check(B.gptq_gemm_bf16(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, D.N, D.K, D.group_size,
+                             D.act_order, stream), "gptq_gemm_bf16")
     return y
 
 

@@ -71,9 +71,15 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_repack(A16, A16, A16, None, A16 + 16, None, A16, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_repack(A16, A16, A16, None, A16, A16 + 16, A16 + 32, None, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_repack(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 16, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
-    assert B.gptq_repack_format(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, 4, stream=0) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_repack_format(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, 8, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_dequant_f32_format(A16, A16, A16, None, A16, 128, 128, 128, 0, 0, B.GPTQ_FORMAT_GATE_UP, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_gemm_silu_mul(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    # the bfloat16 matmul validates like gptq_gemm
+    assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, A16, 1, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_bf16(A16 + 2, A16, A16, A16, None, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_ALIGN
+    assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, A16, 1, 128, 128, 16, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, A16, 0, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_SHAPE
     assert B.gptq_gemm_silu_mul_scatter(A16, A16, A16, A16, None, A16 + 4, A16, 1, 256, 128, 128, 0, stream=0) == B.GPTQ_ERR_ALIGN
     assert B.gptq_invert_perm(None, A16, 8, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_invert_perm(A16, A16, 0, stream=0) == B.GPTQ_ERR_SHAPE

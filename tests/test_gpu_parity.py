@@ -440,7 +440,7 @@ def test_variant_dequant_bit_exact(gs, act, zm1):
     w.zero_()
     B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
     assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
-    assert B.gptq_dequant_f32_format(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 4) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_dequant_f32_format(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 8) == B.GPTQ_ERR_LAYOUT
 
 
 @pytest.mark.parametrize("gs,act,zm1", VARIANTS)
@@ -482,7 +482,7 @@ def test_variants_unsupported_entry_points():
     assert B.gptq_gemm_noalloc(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 4, N, K, 64, 0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_gemm(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 4, N, K, 16, 0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack_format(D.qweight_t, D.qzeros_t, D.scales_t, None, D.qweight_t, D.qzeros_t, D.scales_t, None,
-                                N, K, 64, 0, 4) == B.GPTQ_ERR_LAYOUT
+                                N, K, 64, 0, 8) == B.GPTQ_ERR_LAYOUT
     w = torch.zeros((K, N), dtype=torch.float32, device="cuda")     # the interleave is no property of a checkpoint
     assert B.gptq_dequant_f32_format(H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales), None, w,
                                      N, K, 64, 0, 0, B.GPTQ_FORMAT_GATE_UP) == B.GPTQ_ERR_LAYOUT
@@ -868,3 +868,171 @@ def test_timeline_tool_shows_weight_prefetch_overlapping_the_previous_launch():
         started, last_cta, weights, wait_first = (float(v) for v in mid.split()[:4])
         assert weights < 0.0, f"no prefetch overlap: {line}"
         assert started < weights and started <= last_cta and wait_first > 0.0, line
+
+
+# ------------------------------------------------------------------------------- bfloat16 activations and scales
+def torch_bf16_round(a64: np.ndarray) -> np.ndarray:
+    """float64 values -> the nearest bfloat16 (ties to even) as float64, through torch's conversion."""
+    return torch.from_numpy(np.ascontiguousarray(a64, dtype=np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def assert_close_bf16(y_bits: np.ndarray, y64: np.ndarray, K: int, M: int):
+    """bfloat16 has an 8-bit significand: rounding to nearest moves a value by at most 2^-8 of itself (half an ulp
+    just above a power of two).  Up to 16 token rows the kernel multiplies exact integers q - z, applies the scale in
+    fp32 and rounds once: the fp16 path's own bound with that half ulp.  Above, every scaled weight is also rounded once
+    to bfloat16 - three significand bits fewer than fp16 - so the absolute term of the stated fp16 tolerance is taken
+    eight times wider, and the rms error must stay below 2^-8 of y's rms (expected for these inputs: about 1.7e-3)."""
+    y = torch.from_numpy(y_bits.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    err = np.abs(y - y64)
+    assert np.all(np.isfinite(y))
+    if M <= 16:
+        bound = 1e-4 * math.sqrt(K / 4096) + 2.0 ** -8 * np.abs(y64)
+    else:
+        bound = 8e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(y64)
+        assert math.sqrt(np.mean(err ** 2)) <= 2.0 ** -8 * math.sqrt(np.mean(y64 ** 2))
+    assert np.all(err <= bound), f"{int((err > bound).sum())} violations, max err {err.max():.3e}"
+
+
+def run_gemm_bf16(L, s_bits, x_bits, ws):
+    D = H.upload_and_repack(L, scales_bf16_bits=s_bits)
+    ws.ensure_for(x_bits.shape[0], D)
+    y = H.gemm_bf16(H.bf16_from_bits(x_bits), D)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    return H.bits_of_bf16(y), D
+
+
+@pytest.mark.parametrize("gs,act,zm1", [(128, False, False), (128, True, True), (64, False, True), (32, True, False)])
+def test_bf16_dequant_bit_exact(gs, act, zm1):
+    K, N = 512, 256
+    L = wl.make_linear(K, N, seed=wl.seed_for("bf16-dq", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    s_bits = wl.make_scales_bf16(K // gs, N, wl.seed_for("bf16-dq-s", gs))
+    want = oracle.dequant_f32_bf16(L.qweight, L.qzeros, s_bits, L.g_idx, gs, zeros_minus_one=zm1)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    gi = H.to_device(L.g_idx) if act else None
+    fmt = (B.GPTQ_FORMAT_ZEROS_MINUS_ONE if zm1 else 0) | B.GPTQ_FORMAT_BF16
+    B.check(B.gptq_dequant_f32_format(H.to_device(L.qweight), H.to_device(L.qzeros), H.bf16_from_bits(s_bits), gi, w,
+                                      N, K, gs, act, 0, fmt), "dequant canonical")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    D = H.upload_and_repack(L, scales_bf16_bits=s_bits)
+    w.zero_()
+    B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("gs,act,zm1", [(128, False, False), (128, True, True), (64, True, False), (32, False, True)])
+@pytest.mark.parametrize("M", [1, 5, 8, 13, 16, 17, 40, 100, 200, 600])
+def test_bf16_gemm_small_full_compare(gs, act, zm1, M, ws):
+    """Every kernel family in bfloat16 (mma.sync with 8- and 16-row tiles, tcgen05 with 32- to 256-token tiles), split-K
+    clusters included (K = 1024 on few panels)."""
+    K, N = 1024, 384
+    L = wl.make_linear(K, N, seed=wl.seed_for("bf16", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    s_bits = wl.make_scales_bf16(K // gs, N, wl.seed_for("bf16-s", gs))
+    x_bits = wl.make_x_bf16(M, K, wl.seed_for("bf16-x", M))
+    y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+    assert_close_bf16(y, oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, gs, zeros_minus_one=zm1), K, M)
+
+
+@pytest.mark.parametrize("K,N,S", [(768, 256, 6), (768, 12672, 3), (4096, 4096, 8)])
+@pytest.mark.parametrize("M", [1, 8])
+def test_bf16_split_k_cluster_sizes(K, N, S, M, ws):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    st, pl = B.gptq_plan(M, N, K, 128, 0, sms)
+    if sms == 148:
+        assert pl.cluster_size == S, "the planner no longer picks this cluster size here: choose another shape"
+    L = wl.make_linear(K, N, seed=wl.seed_for("bf16-s36", K, N))
+    s_bits = wl.make_scales_bf16(K // 128, N, wl.seed_for("bf16-s36-s", K))
+    x_bits = wl.make_x_bf16(M, K, wl.seed_for("bf16-s36-x", M))
+    y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+    assert_close_bf16(y, oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, None, 128), K, M)
+
+
+@pytest.mark.parametrize("M", [4, 64])
+def test_bf16_integer_case_is_exact(M, ws):
+    """Scales 1, small-integer x: every product and partial sum is an integer, so wherever |y| <= 256 (exact in
+    bfloat16) the result must be the integer itself on both kernel families."""
+    K, N = 512, 256
+    r = np.random.default_rng(77)
+    q = r.integers(0, 16, (K, N), dtype=np.uint8)
+    z = r.integers(0, 16, (K // 128, N), dtype=np.uint8)
+    L = wl.make_linear_from_values(q, z, np.ones((K // 128, N), np.float16), 128)
+    s_bits = np.full((K // 128, N), 0x3F80, dtype=np.uint16)
+    x_vals = r.integers(-1, 2, (M, K)).astype(np.float32)
+    x_bits = wl.bf16_bits(x_vals)
+    y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+    want = x_vals.astype(np.float64) @ (q.astype(np.float64) - z[np.arange(K) // 128].astype(np.float64))
+    assert np.array_equal(oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, None, 128), want)
+    got = torch.from_numpy(y.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    small = np.abs(want) <= 256
+    assert small.mean() > 0.5
+    assert np.array_equal(got[small], want[small])
+    assert np.array_equal(got[~small], torch_bf16_round(want[~small]))    # and rounded once elsewhere
+
+
+@pytest.mark.parametrize("pad_to", [7, 40])
+def test_bf16_one_hot_rows_return_rounded_weights(pad_to, ws):
+    K, N = 512, 256
+    L = wl.make_linear(K, N, seed=103, act_order=True)
+    s_bits = wl.make_scales_bf16(K // 128, N, 104)
+    ks = [0, 1, 9, 127, 128, 300, 511]
+    x = np.zeros((pad_to, K), dtype=np.float32)
+    for i, k in enumerate(ks):
+        x[i, k] = 1.0
+    y, _ = run_gemm_bf16(L, s_bits, wl.bf16_bits(x), ws)
+    w = oracle.dequant_f32_bf16(L.qweight, L.qzeros, s_bits, L.g_idx, 128)
+    got = torch.from_numpy(y.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(got[:len(ks)], torch_bf16_round(w[ks].astype(np.float64)))
+    assert not got[len(ks):].any()
+
+
+def test_bf16_and_fp16_layers_are_not_interchangeable(ws):
+    """A layer's 16-bit format is recorded by the repack; the matmul of the other format stores nothing and reports a
+    layout mismatch through the status word.  The fp16-only entry points refuse a bfloat16 layer the same way."""
+    K, N, M = 512, 256, 4
+    L = wl.make_linear(K, N, seed=105)
+    s_bits = wl.make_scales_bf16(K // 128, N, 106)
+    D16, Db = H.upload_and_repack(L), H.upload_and_repack(L, scales_bf16_bits=s_bits)
+    x = torch.zeros((M, K), dtype=torch.float16, device="cuda")
+    for m_rows in (M, 40):
+        xx = torch.ones((m_rows, K), dtype=torch.float16, device="cuda")
+        y = torch.zeros((m_rows, N), dtype=torch.float16, device="cuda")
+        assert B.gptq_gemm_bf16(xx, D16.qweight_t, D16.qzeros_t, D16.scales_t, None, y, m_rows, N, K, 128, 0) == B.GPTQ_OK
+        assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+        assert torch.count_nonzero(y) == 0
+        assert B.gptq_gemm(xx, Db.qweight_t, Db.qzeros_t, Db.scales_t, None, y, m_rows, N, K, 128, 0) == B.GPTQ_OK
+        assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+        assert torch.count_nonzero(y) == 0
+    y = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm_noalloc(x, Db.qweight_t, Db.qzeros_t, Db.scales_t, None, y, M, N, K, 128, 0) == B.GPTQ_OK
+    assert B.gptq_check_status() == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_check_status() == B.GPTQ_OK              # reading the status clears it
+    assert torch.count_nonzero(y) == 0
+
+
+def test_bf16_config_shapes(ws):
+    """Llama-2-7B shapes in bfloat16: config 1 (4096 x 4096, M = 1) element by element, the widest layer at M = 8 and a
+    prefill batch on sampled outputs."""
+    K, N = 4096, 4096
+    L = wl.make_linear(K, N, seed=wl.seed_for("bf16-config1"))
+    s_bits = wl.make_scales_bf16(K // 128, N, wl.seed_for("bf16-config1-s"))
+    x_bits = wl.make_x_bf16(1, K, wl.seed_for("bf16-config1-x"))
+    y, D = run_gemm_bf16(L, s_bits, x_bits, ws)
+    assert_close_bf16(y, oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, None, 128), K, 1)
+    r = np.random.default_rng(9)
+    for M in (24, 1024):
+        x_bits = wl.make_x_bf16(M, K, wl.seed_for("bf16-config-x", M))
+        y = H.bits_of_bf16(H.gemm_bf16(H.bf16_from_bits(x_bits), D))
+        assert B.gptq_check_status() == B.GPTQ_OK
+        rows = r.integers(0, M, 3000).astype(np.int32)
+        cols = r.integers(0, N, 3000).astype(np.int32)
+        rows[:4], cols[:4] = [0, 0, M - 1, M - 1], [0, N - 1, 0, N - 1]
+        want = oracle.gemm_f64_bf16_at(x_bits, L.qweight, L.qzeros, s_bits, None, 128, rows, cols)
+        assert_close_bf16(y[rows, cols], want, K, M)
+    K, N, M = 4096, 22016, 8
+    L = wl.make_linear(K, N, seed=wl.seed_for("bf16-gate-up"))
+    s_bits = wl.make_scales_bf16(K // 128, N, wl.seed_for("bf16-gate-up-s"))
+    x_bits = wl.make_x_bf16(M, K, wl.seed_for("bf16-gate-up-x"))
+    y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+    rows = r.integers(0, M, 4000).astype(np.int32)
+    cols = r.integers(0, N, 4000).astype(np.int32)
+    rows[:4], cols[:4] = [0, 0, M - 1, M - 1], [0, N - 1, 0, N - 1]
+    assert_close_bf16(y[rows, cols], oracle.gemm_f64_bf16_at(x_bits, L.qweight, L.qzeros, s_bits, None, 128, rows, cols), K, M)
