@@ -171,6 +171,11 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------ workload
+def bf16_scales(L, layer, name):
+    """The bfloat16 scales of the bfloat16 variant of a bench layer (bit patterns [G, N])."""
+    return wl.make_scales_bf16(L.K // L.group_size, L.N, wl.seed_for("bench-bf16-scales", layer, name))
+
+
 def build_problems(spec, layers, H, torch, device):
     """Uploads `layers` distinct seeded copies of every shape (repacked through the C ABI) and the
     activations; returns {M: [(D, x, y, name), ...]} in launch order (layer-major)."""
@@ -180,18 +185,21 @@ def build_problems(spec, layers, H, torch, device):
     for layer in range(layers):
         for name, (K, N) in spec["shapes"].items():
             L = wl.make_linear(K, N, seed=wl.seed_for("bench", layer, name), act_order=spec["act_order"])
-            D = H.upload_and_repack(L)
+            bf16 = spec.get("bf16", False)
+            D = H.upload_and_repack(L, scales_bf16_bits=bf16_scales(L, layer, name) if bf16 else None)
             if layer == 0:
                 host[name] = L
             for M in Ms:
-                if layer == 0:
+                if layer == 0 and bf16:
+                    x = H.bf16_from_bits(wl.make_x_bf16(M, K, wl.seed_for("bench-x", name, M)), device)
+                elif layer == 0:
                     x = H.to_device(wl.make_x(M, K, wl.seed_for("bench-x", name, M)), device)
                 else:   # activations are tiny next to the weights: reuse layer 0's
                     x = per_m[M][list(spec["shapes"]).index(name)][1]
                 if spec["kind"] == "prefill" and layer > 0:
                     y = per_m[M][list(spec["shapes"]).index(name)][2]
                 else:
-                    y = torch.empty((M, N), dtype=torch.float16, device=device)
+                    y = torch.empty((M, N), dtype=torch.bfloat16 if bf16 else torch.float16, device=device)
                 per_m[M].append((D, x, y, name))
     return per_m, host
 
@@ -241,10 +249,12 @@ def oracle_sample(spec, budget_s):
     layer = {n: wl.make_linear(K, N, seed=wl.seed_for("bench", 0, n), act_order=spec["act_order"])
              for n, (K, N) in shapes.items()}
     Lp = layer[small]
-    xp = wl.make_x(Ms[0], Lp.K, wl.seed_for("bench-x", small, Ms[0]))
-    oracle.gemm_f64(xp, Lp.qweight, Lp.qzeros, Lp.scales, Lp.g_idx, Lp.group_size)   # first touch
+    bf16 = spec.get("bf16", False)
+    make_x = wl.make_x_bf16 if bf16 else wl.make_x
+    xp = make_x(Ms[0], Lp.K, wl.seed_for("bench-x", small, Ms[0]))
+    run_oracle_once([(Lp, xp, Ms[0], small)], spec)   # first touch
     t0 = time.perf_counter()
-    oracle.gemm_f64(xp, Lp.qweight, Lp.qzeros, Lp.scales, Lp.g_idx, Lp.group_size)
+    run_oracle_once([(Lp, xp, Ms[0], small)], spec)
     rate = Ms[0] * Lp.K * Lp.N / (time.perf_counter() - t0)
     pick = ladder[0]
     for names, ms in ladder:
@@ -252,19 +262,23 @@ def oracle_sample(spec, budget_s):
         if macs / rate <= budget_s:
             pick = (names, ms)
     names, ms = pick
-    items = [(layer[n], wl.make_x(M, layer[n].K, wl.seed_for("bench-x", n, M)), M) for n in names for M in ms]
+    items = [(layer[n], make_x(M, layer[n].K, wl.seed_for("bench-x", n, M)), M, n) for n in names for M in ms]
     text = f"layer 0 of the workload, shapes {names}, M in {list(ms)}, full outputs"
     return items, text
 
 
 def run_oracle_once(items, spec):
     import oracle
+    scales = {n: bf16_scales(L, 0, n) for (L, x, M, n) in items} if spec.get("bf16", False) else None
     t0 = time.perf_counter()
-    for (L, x, M) in items:
-        oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
+    for (L, x, M, n) in items:
+        if scales is not None:
+            oracle.gemm_f64_bf16(x, L.qweight, L.qzeros, scales[n], L.g_idx, L.group_size)
+        else:
+            oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
     dt = time.perf_counter() - t0
-    nbytes = sum(wl.algorithmic_bytes(M, L.K, L.N, act_order=L.act_order) for (L, x, M) in items)
-    flops = sum(wl.matmul_flops(M, L.K, L.N) for (L, x, M) in items)
+    nbytes = sum(wl.algorithmic_bytes(M, L.K, L.N, act_order=L.act_order) for (L, x, M, n) in items)
+    flops = sum(wl.matmul_flops(M, L.K, L.N) for (L, x, M, n) in items)
     return dt, nbytes, flops
 
 
@@ -347,9 +361,12 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
     ws.ensure(need)
     bytes_m, flops_m = step_bytes_flops(spec, layers)
 
+    bf16 = spec.get("bf16", False)
+    gemm = H.gemm_bf16 if bf16 else H.gemm
+
     def run_m(M):
         for (D, x, y, _n) in per_m[M]:
-            H.gemm(x, D, y)
+            gemm(x, D, y)
 
     # eager warm-up (configures the kernels), then one CUDA graph per M
     stream = torch.cuda.Stream(device)
@@ -410,7 +427,7 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
     for M in Ms:
         for (D, x, y, name) in per_m[M][:len(spec["shapes"])]:
             xh = x.cpu().pin_memory()
-            yh = torch.empty((M, D.N), dtype=torch.float16).pin_memory()
+            yh = torch.empty((M, D.N), dtype=torch.bfloat16 if bf16 else torch.float16).pin_memory()
             host_io[(M, name)] = (xh, yh)
     for M in Ms:
         for (D, x, y, name) in per_m[M]:
@@ -426,7 +443,7 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
     step_problems = B.make_host_problems(step_items)
 
     def e2e_step():
-        st, bad = B.gptq_gemm_host_batch(step_problems)
+        st, bad = (B.gptq_gemm_host_batch_bf16 if bf16 else B.gptq_gemm_host_batch)(step_problems)
         B.check(st, f"gptq_gemm_host_batch (problem {bad})")
         stream.synchronize()   # the step's results are on the host
 
@@ -450,7 +467,7 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
 
     sms = torch.cuda.get_device_properties(device).multi_processor_count
     launches_step = sum(launches_per_gemm(spec, M, nm, sms) for M in Ms for (_D, _x, _y, nm) in per_m[M])
-    kernels = {M: kernel_of(spec, M, sms) for M in Ms}
+    kernels = {M: kernel_of(spec, M, sms) + (" bf16" if bf16 else "") for M in Ms}
     out = dict(total_ms=total_ms, e2e_ms=e2e_ms, e2e_steps=e2e_steps, seg_ms=seg_ms, clocks=clocks, bytes_m=bytes_m,
                flops_m=flops_m, h2d=h2d, d2h=d2h, launches_step=launches_step, kernels=kernels,
                matmuls={M: len(per_m[M]) for M in Ms}, Ms=Ms)
@@ -470,18 +487,24 @@ def per_shape_m1(spec, env, reps=20):
     for name, (K, N) in spec["shapes"].items():
         copies = max(2, math.ceil(600e6 / (K * N // 2)))
         L = wl.make_linear(K, N, seed=wl.seed_for("per-shape", name), act_order=spec["act_order"])
-        Ds = [H.upload_and_repack(L, device=device) for _ in range(copies)]
-        x = H.to_device(wl.make_x(1, K, wl.seed_for("per-shape-x", name)), device)
-        y = torch.empty((1, N), dtype=torch.float16, device=device)
+        bf16 = spec.get("bf16", False)
+        gemm = H.gemm_bf16 if bf16 else H.gemm
+        Ds = [H.upload_and_repack(L, device=device, scales_bf16_bits=bf16_scales(L, 0, name) if bf16 else None)
+              for _ in range(copies)]
+        if bf16:
+            x = H.bf16_from_bits(wl.make_x_bf16(1, K, wl.seed_for("per-shape-x", name)), device)
+        else:
+            x = H.to_device(wl.make_x(1, K, wl.seed_for("per-shape-x", name)), device)
+        y = torch.empty((1, N), dtype=torch.bfloat16 if bf16 else torch.float16, device=device)
         ws.ensure_for(1, Ds[0])
         with torch.cuda.stream(stream):
             for D in Ds:
-                H.gemm(x, D, y, stream=stream)
+                gemm(x, D, y, stream=stream)
             stream.synchronize()
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
                 for D in Ds:
-                    H.gemm(x, D, y, stream=stream)
+                    gemm(x, D, y, stream=stream)
             for _ in range(3):
                 g.replay()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -557,16 +580,18 @@ def report_line(name, spec, layers, steps, warmup, r, world):
     line = {
         "metric": metric, "value": round(value, 2), "unit": unit, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": round(total_ms / steps, 5), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if spec.get("bf16", False) else "f16", "data": "synthetic",
         "config": {"workload": name, "describes": spec["describes"], "layers": layers,
                    "matmuls_per_step": sum(n_matmuls[M] for M in Ms), "group_size": 128,
                    "act_order": spec["act_order"], "parallelism": f"{world} independent replica(s)",
                    "l2": f"inputs larger than L2: each M pass streams {round(bytes_m[Ms[0]] / 1e6)} MB of distinct weights",
-                   "timing": "CUDA events around CUDA-graph replays of the gptq_gemm calls, one graph per M"},
+                   "timing": "CUDA events around CUDA-graph replays of the " + ("gptq_gemm_bf16" if spec.get("bf16", False) else "gptq_gemm") +
+                             " calls, one graph per M"},
         "clocks": clocks,
         "e2e": {"value": round(e2e_value, 2), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
-                "api": "one gptq_gemm_host_batch call per step (x from pinned host memory, y back to it, per matmul)"},
+                "api": ("one gptq_gemm_host_batch_bf16" if spec.get("bf16", False) else "one gptq_gemm_host_batch") +
+                       " call per step (x from pinned host memory, y back to it, per matmul)"},
         "gpu_launches": launches_step * steps,
         "per_M": per_m_report,
         "roofline": roofline,
@@ -591,6 +616,8 @@ def main():
     ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
     ap.add_argument("--cta-pairs", action="store_true", help="prefill on CTA pairs (tcgen05 cta_group::2), off by default")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dtype", default="f16", choices=["f16", "bf16"],
+                    help="bf16: the same workload with bfloat16 activations and scales (gptq_gemm_bf16)")
     ap.add_argument("--prefill-steps", type=int, default=10,
                     help="decode7b only: steps of the prefill7b workload measured after it and reported as `prefill` (0 = skip)")
     ap.add_argument("--ref-budget", type=float, default=150.0,
@@ -604,6 +631,8 @@ def main():
     spec = dict(WORKLOADS[args.workload])
     if args.ms:
         spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
+    if args.dtype == "bf16":
+        spec["bf16"] = True
     layers = args.layers or spec["layers"]
     if args.impl == "reference":
         run_reference(args, spec)
@@ -640,7 +669,7 @@ def main():
     # prefill workload after the decode one, and reports it as a sub-object of the same line.
     prefill = None
     if args.workload == "decode7b" and not args.ms and args.prefill_steps > 0:
-        pspec = dict(WORKLOADS["prefill7b"])
+        pspec = dict(WORKLOADS["prefill7b"], bf16=spec.get("bf16", False))
         prefill = measure_workload("prefill7b", pspec, pspec["layers"], args.prefill_steps, 3, min(args.prefill_steps, 5), env)
     shapes_m1 = None
     if args.workload == "decode7b" and not args.ms and world == 1:

@@ -94,7 +94,8 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
  * bfloat16.  The repack moves the 16-bit words unchanged and records the flag; gptq_dequant_f32 then reads the scales
  * as bfloat16 (the fp32 product float(q - z) * s is still exact), and the layer is multiplied with gptq_gemm_bf16, not
  * gptq_gemm.  May be combined with GPTQ_FORMAT_ZEROS_MINUS_ONE; the fused epilogues (and so GPTQ_FORMAT_GATE_UP),
- * gptq_gemm_host, gptq_gemm_host_batch and gptq_gemm_noalloc exist for fp16 layers only. */
+ * gptq_gemm_host and gptq_gemm_noalloc exist for fp16 layers only (gptq_gemm_host_batch_bf16 is the host-resident
+ * path). */
 #define GPTQ_FORMAT_BF16 4
 /* gptq_dequant_f32 with a format for canonical inputs (repacked = 0; GPTQ_FORMAT_GATE_UP is refused there with
  * GPTQ_ERR_LAYOUT); with repacked = 1 the trailer decides and `format` must be 0 or equal to what the layer was
@@ -277,6 +278,9 @@ typedef struct {
  * for the duration of the enqueue.  Not capturable in a CUDA graph (it records and waits on events of
  * internal streams). */
 int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
+/* The same pipeline for bfloat16 layers: every problem's x_host / y_host hold bfloat16 and its layer was repacked with
+ * GPTQ_FORMAT_BF16; each matmul is a gptq_gemm_bf16.  Arguments, ordering and errors as above. */
+int gptq_gemm_host_batch_bf16(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
 
 /* Synchronises `stream` and returns GPTQ_ERR_LAYOUT if a kernel since the last check met a layer whose tiling does
  * not fit the call (see GPTQ_FORMAT_GATE_UP), GPTQ_ERR_TIMEOUT if a kernel's bounded wait gave up (the flag is
@@ -306,7 +310,8 @@ int gptq_trace_read(unsigned long long *rows_out, int max_rows, void *stream);
 /* ---- host-only: how a problem would be launched (no CUDA call; usable without a GPU) -- */
 
 typedef struct {
-    char kernel_name[48]; /* the kernel instantiation as profilers print it, e.g. "splitk_kernel<1>" */
+    char kernel_name[48]; /* the kernel instantiation, e.g. "splitk_kernel<1,1>": a profiler prints the same integers, followed by the
+                             bfloat16 flag (false for gptq_gemm, true for gptq_gemm_bf16) */
     int kernel;       /* 1 = cluster split-K mma.sync kernel (gptq_gemm, M <= 16),
                          2 = tcgen05 kernel (gptq_gemm, M >= 17),
                          3 = stream-K mma.sync kernel (gptq_gemm_noalloc) */

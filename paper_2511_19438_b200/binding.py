@@ -82,6 +82,7 @@ _SIGNATURES = {
     "gptq_gemm_noalloc": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_noalloc_scratch_bytes": (_sz, []),
     "gptq_gemm_host_batch": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
+    "gptq_gemm_host_batch_bf16": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_check_status": (_i, [_vp]),
     "gptq_selftest_wait_timeout": (_i, [ctypes.c_uint, _vp]),
     "gptq_trace_reset": (_i, [_vp]),
@@ -246,6 +247,13 @@ def gptq_gemm_host_batch(problems, stream=None):
     """Returns (status, bad_index); `problems` comes from make_host_problems."""
     bad = ctypes.c_int(-1)
     st = _lib.gptq_gemm_host_batch(problems, len(problems), _stream(stream), ctypes.byref(bad))
+    return st, bad.value
+
+
+def gptq_gemm_host_batch_bf16(problems, stream=None):
+    """gptq_gemm_host_batch for bfloat16 layers and activations."""
+    bad = ctypes.c_int(-1)
+    st = _lib.gptq_gemm_host_batch_bf16(problems, len(problems), _stream(stream), ctypes.byref(bad))
     return st, bad.value
 
 

@@ -564,7 +564,9 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
     return GPTQ_OK;
 }
 
-int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
+} // extern "C"
+
+static int host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index, int bf16)
 {
     if (!problems || count < 0) return GPTQ_ERR_NULL;
     for (int i = 0; i < count; ++i) {
@@ -623,8 +625,8 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
                 break;
             }
         if (st) break;
-        st = gptq_gemm(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
-                       q.act_order, stream);
+        st = gemm_dispatch(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
+                           q.act_order, 0, nullptr, nullptr, nullptr, stream, bf16);
         if (st) {
             if (bad_index) *bad_index = i;
             break;
@@ -640,6 +642,18 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
     if (!st2) st2 = check(cudaEventRecord(ev_x[0], pipe->out));
     if (!st2) st2 = check(cudaStreamWaitEvent(s, ev_x[0], 0));
     return st ? st : st2;
+}
+
+extern "C" {
+
+int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
+{
+    return host_batch(problems, count, stream, bad_index, 0);
+}
+
+int gptq_gemm_host_batch_bf16(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
+{
+    return host_batch(problems, count, stream, bad_index, 1);
 }
 
 // ---- self-test of the bounded waits ------------------------------------------------------------

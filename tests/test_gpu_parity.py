@@ -1036,3 +1036,28 @@ def test_bf16_config_shapes(ws):
     cols = r.integers(0, N, 4000).astype(np.int32)
     rows[:4], cols[:4] = [0, 0, M - 1, M - 1], [0, N - 1, 0, N - 1]
     assert_close_bf16(y[rows, cols], oracle.gemm_f64_bf16_at(x_bits, L.qweight, L.qzeros, s_bits, None, 128, rows, cols), K, M)
+
+
+def test_bf16_host_batch_step(ws):
+    """Three bfloat16 matmuls (one act-order, one on the tcgen05 kernel) from pinned host memory and back."""
+    specs = [(1024, 256, 2, False), (640, 256, 5, True), (512, 384, 40, False)]
+    items, keep = [], []
+    for (K, N, M, act) in specs:
+        L = wl.make_linear(K, N, seed=wl.seed_for("bf16-batch", K, N, act), act_order=act)
+        s_bits = wl.make_scales_bf16(K // 128, N, wl.seed_for("bf16-batch-s", K))
+        D = H.upload_and_repack(L, scales_bf16_bits=s_bits)
+        x_bits = wl.make_x_bf16(M, K, wl.seed_for("bf16-batch-x", K, M))
+        xh = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+        yh = torch.zeros((M, N), dtype=torch.bfloat16).pin_memory()
+        xs = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+        ys = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        items.append((xh, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, yh, xs, ys, M, N, K, 128, act))
+        keep.append((L, s_bits, x_bits, yh, D))
+    ws.ensure(max(B.gptq_workspace_bytes(M, N, K, 128, act) for (K, N, M, act) in specs))
+    st, bad = B.gptq_gemm_host_batch_bf16(B.make_host_problems(items))
+    assert (st, bad) == (B.GPTQ_OK, -1)
+    torch.cuda.synchronize()
+    assert B.gptq_check_status() == B.GPTQ_OK
+    for (L, s_bits, x_bits, yh, _D), (K, N, M, act) in zip(keep, specs):
+        want = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, 128)
+        assert_close_bf16(H.bits_of_bf16(yh), want, K, M)
