@@ -77,8 +77,13 @@ int gptq_dequant_f32(const void *qweight, const void *qzeros, const void *scales
 
 /* Format variants.  The paper (Section 1, Section 4.2) names 4-bit GPTQ without fixing the checkpoint conventions,
  * and checkpoints of the same family differ in two of them:
- *   - group_size: 128 (all of the paper's models), 64 or 32 rows per scale / zero point.  Every tiled entry point
- *     accepts these three; gptq_gemm_noalloc and the CTA-pair switch accept 128 only.
+ *   - group_size: 128 (all of the paper's models), 64 or 32 rows per scale / zero point, or any multiple of 128 that
+ *     divides K (256, 512, ... up to K itself: one scale and zero point per output column, "per-channel").  Every tiled
+ *     entry point accepts these; the caller passes the checkpoint's group_size to all of them.  Groups coarser than 128
+ *     rows are tiled as groups of 128 rows that repeat their group's scale and zero point (the tiled scales and zero
+ *     points then take K/128 instead of K/group_size rows: gptq_repack_bytes says how much), so the kernels see a
+ *     group-128 layer and the results are those of the checkpoint's own grouping.  gptq_gemm_noalloc and the CTA-pair
+ *     switch accept 128 and coarser only.
  *   - the zero point: stored as is (default), or stored minus one (older checkpoints: the kernels add the one
  *     back, so a stored 15 means 16).  Pass GPTQ_FORMAT_ZEROS_MINUS_ONE to the _format entry points below.
  * gptq_repack_format records the flag in a 16-byte trailer behind the tiled zero points (counted in
@@ -108,11 +113,12 @@ int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void 
 
 /* Byte size of each gptq_repack output: which = 0 qweight_out, 1 qzeros_out, 2 scales_out,
  * 3 perm_out (0 bytes unless act_order).  Sizes equal the canonical ones, plus 16 bytes of format trailer
- * behind the zero points.  Returns 0 for an invalid argument. */
+ * behind the zero points (with group_size > 128: scales and zero points of K/128 groups).  Returns 0 for an invalid
+ * argument. */
 size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order);
 
 /* Re-tiles a canonical layer (what Section 3.2 / Algorithm 2 achieve with wider loads of the original layout is
- * achieved here by storing the weights in the order the kernels stream them).  Fast-path requirements: group_size 128, 64 or 32, K % 128 == 0,
+ * achieved here by storing the weights in the order the kernels stream them).  Fast-path requirements: group_size 32, 64 or a multiple of 128, K % 128 == 0,
  * N % 128 == 0 (else GPTQ_ERR_UNSUPPORTED).  With act_order != 0 the rows are stably sorted
  * by g_idx so that each group's rows are contiguous; perm_out[i] = original index of sorted
  * row i (int32[K]).  g_idx is range-checked on the device and every group must have exactly

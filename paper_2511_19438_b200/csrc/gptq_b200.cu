@@ -71,13 +71,19 @@ static int check_shape(int M, int N, int K, int group_size)
     if (K % 8 || N % 8 || K % group_size) return GPTQ_ERR_SHAPE;
     return GPTQ_OK;
 }
-static int check_fast_path(int N, int K, int group_size)
+// On success `group_size` becomes the group size of the TILED layer: a checkpoint whose groups are a multiple of 128
+// rows (256, 512, ..., K = one group per column) is tiled as groups of 128 rows that repeat their group's scales and
+// zero points, so the kernels see an ordinary group-128 layer.
+static int check_fast_path(int N, int K, int &group_size)
 {
-    if ((group_size != 128 && group_size != 64 && group_size != 32) || N % kPanel || K % kGroup)
+    const bool coarse = group_size > kGroup && group_size % kGroup == 0;
+    if ((!coarse && group_size != 128 && group_size != 64 && group_size != 32) || N % kPanel || K % kGroup)
         return GPTQ_ERR_UNSUPPORTED;
     if (N / kPanel > (int)(kTicketAreaBytes / sizeof(int))) return GPTQ_ERR_UNSUPPORTED;
+    if (coarse) group_size = kGroup;
     return GPTQ_OK;
 }
+static inline int tiled_group_size(int group_size) { return group_size > kGroup ? kGroup : group_size; }
 
 static int current_device_sms(int *dev_out, int *sms_out)
 {
@@ -162,7 +168,7 @@ const char *gptq_status_string(int status)
     case GPTQ_ERR_NULL: return "a required pointer is NULL";
     case GPTQ_ERR_SHAPE: return "invalid shape (need M>=1, K%8==0, N%8==0, K%group_size==0)";
     case GPTQ_ERR_ALIGN: return "a pointer is not 16-byte aligned";
-    case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 128, 64 or 32, N%128==0, K%128==0)";
+    case GPTQ_ERR_UNSUPPORTED: return "shape outside the tiled fast path (group_size 32, 64 or a multiple of 128, N%128==0, K%128==0)";
     case GPTQ_ERR_LAYOUT: return "invalid layout selector or flag";
     case GPTQ_ERR_GIDX: return "g_idx entry out of range, or groups of unequal size";
     case GPTQ_ERR_WORKSPACE: return "workspace missing or too small (see gptq_workspace_bytes)";
@@ -216,7 +222,7 @@ int gptq_dequant_f32_format(const void *qweight, const void *qzeros, const void 
 size_t gptq_repack_bytes(int which, int N, int K, int group_size, int act_order)
 {
     if (check_shape(1, N, K, group_size) != GPTQ_OK) return 0;
-    const size_t G = (size_t)(K / group_size);
+    const size_t G = (size_t)(K / tiled_group_size(group_size));   // coarser groups are stored once per 128 rows
     switch (which) {
     case 0: return (size_t)K / 8 * N * 4;
     case 1: return G * (N / 8) * 4 + kTrailerBytes;   // + the format trailer
@@ -243,13 +249,14 @@ int gptq_repack_format(const int32_t *qweight, const int32_t *qzeros, const void
     if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
     int st = check_shape(1, N, K, group_size);
     if (st) return st;
+    const int source_group_size = group_size;
     st = check_fast_path(N, K, group_size);
     if (st) return st;
     if (!aligned16(qweight_out) || !aligned16(qzeros_out) || !aligned16(scales_out)) return GPTQ_ERR_ALIGN;
     if (qweight_out == (const void *)qweight || qzeros_out == (const void *)qzeros || scales_out == scales)
         return GPTQ_ERR_LAYOUT;
     return launch_repack(qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, N, K,
-                         group_size, act_order, format, (cudaStream_t)stream);
+                         source_group_size, act_order, format, (cudaStream_t)stream);
 }
 
 static void set_kernel_name(gptq_plan_t *out, const char *fmt, int a, int b = 0, int c = 0, int d = 0)
@@ -579,7 +586,8 @@ static int host_batch(const gptq_host_problem_t *problems, int count, void *stre
         if (!st && (!aligned16(q.x_stage) || !aligned16(q.y_stage) || !aligned16(q.qweight) || !aligned16(q.qzeros) ||
                     !aligned16(q.scales)))
             st = GPTQ_ERR_ALIGN;
-        if (!st) st = check_fast_path(q.N, q.K, q.group_size);
+        int tiled_group = q.group_size;
+        if (!st) st = check_fast_path(q.N, q.K, tiled_group);
         if (st) {
             if (bad_index) *bad_index = i;
             return st;

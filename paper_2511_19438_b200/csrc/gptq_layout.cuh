@@ -179,7 +179,7 @@ __global__ void repack_weights_kernel(const int32_t *__restrict__ qweight, const
 // zero byte of its column pair.  Thread 0 writes the trailer behind the zero points.
 __global__ void repack_meta_kernel(const int32_t *__restrict__ qzeros, const __half *__restrict__ scales,
                                    uint8_t *__restrict__ z_out, __half *__restrict__ s_out, int N, int G,
-                                   int group_size, uint32_t flags)
+                                   int group_size, int repeat, uint32_t flags)
 {
     size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx == 0) {
@@ -187,13 +187,15 @@ __global__ void repack_meta_kernel(const int32_t *__restrict__ qzeros, const __h
         *reinterpret_cast<TiledTrailer *>(z_out + (size_t)G * (N / 2)) = tr;
     }
     if (idx >= (size_t)G * N) return;
-    // one thread per (group, tiled column nt); its values come from checkpoint column n
+    // one thread per (tiled group, tiled column nt); its values come from checkpoint column n of checkpoint group
+    // grp / repeat (repeat > 1: the checkpoint's groups span `repeat` tiled groups of 128 rows)
     int grp = (int)(idx / N), nt = (int)(idx % N);
+    const int src = grp / repeat;
     const bool gate_up = (flags & kFormatGateUp) != 0;
     int n = gate_up ? gate_up_source_column(nt, N) : nt;
-    s_out[repacked_scale_index(grp, nt, G)] = scales[(size_t)grp * N + n];
+    s_out[repacked_scale_index(grp, nt, G)] = scales[(size_t)src * N + n];
     if (((nt % 16) >> 3) == 0) {
-        const int32_t *zrow = qzeros + (size_t)grp * (N / 8);
+        const int32_t *zrow = qzeros + (size_t)src * (N / 8);
         uint32_t za = ((uint32_t)zrow[n >> 3] >> (4 * (n & 7))) & 15u;
         int nb = n + 8;     // the partner column: eight further in both numberings (halves are multiples of 64)
         uint32_t zb = ((uint32_t)zrow[nb >> 3] >> (4 * (nb & 7))) & 15u;
@@ -208,13 +210,16 @@ __global__ void repack_fence_kernel() {}
 
 int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
                   void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, int N, int K,
-                  int group_size, int act_order, int format, cudaStream_t s)
+                  int source_group_size, int act_order, int format, cudaStream_t s)
 {
+    // source_group_size: rows per group in the checkpoint; group_size: rows per group of the tiled layer (the same, or
+    // 128 when the checkpoint's groups are a multiple of 128 rows: the tiled groups then repeat their group's values)
+    const int group_size = source_group_size > kGroup ? kGroup : source_group_size;
     const int T = 256;
     int G = K / group_size;
     if (act_order) {
         int blocks = (K + T - 1) / T;
-        argsort_gidx_kernel<<<blocks, T, T * sizeof(int32_t), s>>>(g_idx, perm_out, K, G, group_size);
+        argsort_gidx_kernel<<<blocks, T, T * sizeof(int32_t), s>>>(g_idx, perm_out, K, K / source_group_size, source_group_size);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return record_cuda_error(e);
         // one-time call: read the validation result before tiling with a possibly invalid perm
@@ -237,7 +242,7 @@ int launch_repack(const int32_t *qweight, const int32_t *qzeros, const void *sca
     size_t meta = (size_t)G * N;
     repack_meta_kernel<<<(unsigned)((meta + T - 1) / T), T, 0, s>>>(qzeros, (const __half *)scales,
                                                                     (uint8_t *)qzeros_out, (__half *)scales_out, N, G,
-                                                                    group_size, (uint32_t)format);
+                                                                    group_size, source_group_size / group_size, (uint32_t)format);
     repack_fence_kernel<<<1, 32, 0, s>>>();
     return record_cuda_error(cudaGetLastError());
 }

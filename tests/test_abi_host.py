@@ -58,7 +58,7 @@ def test_gemm_validation_order_without_gpu():
     assert call(qw=A16 + 4) == B.GPTQ_ERR_ALIGN
     assert call(act_order=1, gi=A16 + 4) == B.GPTQ_ERR_ALIGN   # perm_out is read 16 bytes at a time
     assert call(group_size=16) == B.GPTQ_ERR_UNSUPPORTED   # 128, 64 and 32 have a tiled layout
-    assert call(group_size=256) == B.GPTQ_ERR_UNSUPPORTED
+    assert call(group_size=8) == B.GPTQ_ERR_UNSUPPORTED
     assert call(N=4096 + 64) == B.GPTQ_ERR_UNSUPPORTED
 
 
@@ -90,6 +90,18 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_gemm_silu_mul(A16, A16, A16, A16, None, A16, 1, 192, 128, 128, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_repack_bytes(1, 256, 512, 32, 0) == (512 // 32) * 256 // 2 + 16    # zero points + format trailer
     assert B.gptq_plan_noalloc(4, 128, 512, 64, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED
+    # groups coarser than 128 rows (multiples of 128, up to one group per column) are tiled as repeated 128-row groups
+    assert B.gptq_repack_bytes(1, 256, 512, 256, 0) == (512 // 128) * 256 // 2 + 16
+    assert B.gptq_repack_bytes(2, 256, 512, 512, 0) == (512 // 128) * 256 * 2
+    assert B.gptq_repack_bytes(0, 256, 512, 512, 0) == 512 * 256 // 2
+    for gs in (256, 1024, 4096):
+        st, pl = B.gptq_plan(8, 4096, 4096, gs, 0, 148)
+        st128, pl128 = B.gptq_plan(8, 4096, 4096, 128, 0, 148)
+        assert st == B.GPTQ_OK and B.plan_kernel_name(pl) == B.plan_kernel_name(pl128) and pl.ctas == pl128.ctas
+    assert B.gptq_plan(8, 256, 768, 192, 0, 148)[0] == B.GPTQ_ERR_UNSUPPORTED      # divides K, but no multiple of 128
+    assert B.gptq_plan(8, 256, 768, 384, 0, 148)[0] == B.GPTQ_OK
+    assert B.gptq_plan_noalloc(4, 128, 512, 512, 0, 148)[0] == B.GPTQ_OK
+    assert B.gptq_workspace_bytes(4, 256, 512, 512, 1) == B.gptq_workspace_bytes(4, 256, 512, 128, 1) > 0
     assert B.gptq_repack(A16, A16, A16, A16, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_gemm_host(None, A16, A16, A16, None, A16, A16, A16, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
 

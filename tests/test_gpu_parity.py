@@ -1061,3 +1061,50 @@ def test_bf16_host_batch_step(ws):
     for (L, s_bits, x_bits, yh, _D), (K, N, M, act) in zip(keep, specs):
         want = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, 128)
         assert_close_bf16(H.bits_of_bf16(yh), want, K, M)
+
+
+# ------------------------------------------------------------------------------- groups coarser than 128 rows
+@pytest.mark.parametrize("gs,act,zm1", [(256, False, False), (256, True, True), (1024, True, False), (1024, False, True)])
+def test_coarse_groups_dequant_bit_exact_and_sizes(gs, act, zm1):
+    """group_size 256 and group_size = K (per-channel): the tiled layer repeats each group's scale and zero point every
+    128 rows, and dequantises to the oracle's bits in both layouts."""
+    K, N = 1024, 256
+    L = wl.make_linear(K, N, seed=wl.seed_for("coarse-dq", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    want = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    gi = H.to_device(L.g_idx) if act else None
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if zm1 else 0
+    B.check(B.gptq_dequant_f32_format(H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales), gi, w,
+                                      N, K, gs, act, 0, fmt), "dequant canonical")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    D = H.upload_and_repack(L)
+    assert D.scales_t.numel() == (K // 128) * N * 2 and D.qzeros_t.numel() == (K // 128) * N // 2 + 16
+    w.zero_()
+    B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("gs,act", [(256, True), (1024, False), (1024, True)])
+@pytest.mark.parametrize("M", [1, 8, 16, 40, 300])
+def test_coarse_groups_gemm(gs, act, M, ws):
+    K, N = 1024, 384
+    L = wl.make_linear(K, N, seed=wl.seed_for("coarse", gs, act), group_size=gs, act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("coarse-x", M))
+    y, D = run_gemm(L, x, ws)
+    assert_close(y, oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs), K)
+    if M <= 16:      # the entry point without allocations takes the same layer
+        y2 = torch.zeros((M, N), dtype=torch.float16, device="cuda")
+        B.check(B.gptq_gemm_noalloc(H.to_device(x), D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y2, M, N, K, gs, act),
+                "gptq_gemm_noalloc")
+        assert B.gptq_check_status() == B.GPTQ_OK
+        assert_close(y2.cpu().numpy(), oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs), K)
+
+
+def test_per_channel_bf16_gemm(ws):
+    K, N = 1024, 384
+    L = wl.make_linear(K, N, seed=wl.seed_for("coarse-bf16"), group_size=K)
+    s_bits = wl.make_scales_bf16(1, N, wl.seed_for("coarse-bf16-s"))
+    for M in (3, 50):
+        x_bits = wl.make_x_bf16(M, K, wl.seed_for("coarse-bf16-x", M))
+        y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+        assert_close_bf16(y, oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, None, K), K, M)

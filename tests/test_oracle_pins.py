@@ -492,3 +492,23 @@ def test_bf16_sampled_outputs_equal_full_product():
         cols = np.array([0, 63, 17, 18, 40], dtype=np.int32)
         at = oracle.gemm_f64_bf16_at(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, 128, rows, cols, zeros_minus_one=zm)
         assert np.array_equal(at, full[rows, cols])
+
+
+# --------------------------------------------------------------------------- groups coarser than 128 rows
+@pytest.mark.parametrize("gs,act", [(256, False), (256, True), (512, False), (512, True)])
+def test_coarse_groups_and_per_channel_against_library_matmul(gs, act):
+    """group_size 256 and group_size = K (one scale and zero point per column): numpy's fp64 matmul over a vectorised
+    unpack, and the hand check that with one group every row of a column uses the same scale and zero point."""
+    K, N, M = 512, 64, 3
+    L = wl.make_linear(K, N, seed=wl.seed_for("pin-coarse", gs, act), group_size=gs, act_order=act)
+    assert L.scales.shape == (K // gs, N) and L.qzeros.shape == (K // gs, N // 8)
+    x = wl.make_x(M, K, wl.seed_for("pin-coarse-x", gs))
+    q, z = numpy_unpack(L.qweight, L.qzeros)
+    grp = L.g_idx if act else np.arange(K) // gs
+    w = (q - z[grp]).astype(np.float64) * L.scales[grp].astype(np.float64)
+    got_w = oracle.dequant_f32(L.qweight, L.qzeros, L.scales, L.g_idx, gs)
+    assert np.array_equal(got_w.astype(np.float64), w)
+    assert np.allclose(oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs), x.astype(np.float64) @ w,
+                       rtol=1e-12, atol=1e-12)
+    if gs == K:
+        assert np.array_equal(w, (q - z[0][None, :]) * L.scales[0].astype(np.float64)[None, :])
