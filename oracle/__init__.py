@@ -42,7 +42,8 @@ def _load():
         for name in ("oracle_unpack_q", "oracle_unpack_z", "oracle_dequant_f32",
                      "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64",
                      "oracle_add_bias_residual_f64", "oracle_dequant_f32_bf16", "oracle_gemm_f64_bf16",
-                     "oracle_gemm_f64_bf16_at"):
+                     "oracle_gemm_f64_bf16_at", "oracle_unpack_q8", "oracle_unpack_z8", "oracle_dequant_f32_w8",
+                     "oracle_gemm_f64_w8", "oracle_gemm_f64_w8_at"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -245,4 +246,74 @@ def gemm_f64_bf16_at(x_bits, qweight, qzeros, scales_bits, g_idx, group_size: in
                                     ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group_size),
                                     ctypes.c_int(1 if zeros_minus_one else 0),
                                     _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
+    return out
+
+
+# ---- 8-bit weights: qweight int32[K/4, N], qzeros int32[G, N/4] ------------------------------------------------------
+
+def unpack_q8(qweight: np.ndarray) -> np.ndarray:
+    """int32[K/4, N] -> uint8[K, N]."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    out = np.empty((R * 4, N), dtype=np.uint8)
+    _load().oracle_unpack_q8(_p(qweight), ctypes.c_int(R * 4), ctypes.c_int(N), _p(out))
+    return out
+
+
+def unpack_z8(qzeros: np.ndarray) -> np.ndarray:
+    """int32[G, N/4] -> uint8[G, N]."""
+    qzeros = _i32(qzeros)
+    G, C = qzeros.shape
+    out = np.empty((G, C * 4), dtype=np.uint8)
+    _load().oracle_unpack_z8(_p(qzeros), ctypes.c_int(G), ctypes.c_int(C * 4), _p(out))
+    return out
+
+
+def _w8_args(qweight, qzeros, scales, g_idx, group_size):
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 4
+    G = K // group_size
+    qzeros = _i32(qzeros, (G, N // 4))
+    scales = _f16(scales, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    return qweight, qzeros, scales, g, K, N
+
+
+def dequant_f32_w8(qweight, qzeros, scales, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp32[K, N] dequantised 8-bit weights."""
+    qweight, qzeros, scales, g, K, N = _w8_args(qweight, qzeros, scales, g_idx, group_size)
+    out = np.empty((K, N), dtype=np.float32)
+    _load().oracle_dequant_f32_w8(_p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(K), ctypes.c_int(N),
+                                  ctypes.c_int(group_size), ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
+    return out
+
+
+def gemm_f64_w8(x, qweight, qzeros, scales, g_idx, group_size: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp64[M, N] = x[M, K] . dequant(W8)[K, N], k ascending."""
+    qweight, qzeros, scales, g, K, N = _w8_args(qweight, qzeros, scales, g_idx, group_size)
+    x = _f16(x)
+    M = x.shape[0]
+    assert x.shape == (M, K)
+    out = np.empty((M, N), dtype=np.float64)
+    _load().oracle_gemm_f64_w8(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M), ctypes.c_int(N),
+                               ctypes.c_int(K), ctypes.c_int(group_size), ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
+    return out
+
+
+def gemm_f64_w8_at(x, qweight, qzeros, scales, g_idx, group_size: int, rows, cols, zeros_minus_one: bool = False) -> np.ndarray:
+    """The same sum as :func:`gemm_f64_w8` for chosen (row, col) outputs only."""
+    qweight, qzeros, scales, g, K, N = _w8_args(qweight, qzeros, scales, g_idx, group_size)
+    x = _f16(x)
+    M = x.shape[0]
+    assert x.shape == (M, K)
+    rows = _i32(rows)
+    cols = _i32(cols)
+    assert rows.shape == cols.shape and rows.ndim == 1
+    assert rows.min(initial=0) >= 0 and rows.max(initial=0) < M
+    assert cols.min(initial=0) >= 0 and cols.max(initial=0) < N
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _load().oracle_gemm_f64_w8_at(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M), ctypes.c_int(N),
+                                  ctypes.c_int(K), ctypes.c_int(group_size), ctypes.c_int(1 if zeros_minus_one else 0),
+                                  _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
     return out

@@ -297,3 +297,84 @@ void oracle_gemm_f64_bf16_at(const uint16_t *x, const int32_t *qweight, const in
         y_out[i] = acc;
     }
 }
+
+/* ---- format variant: 8-bit weights -------------------------------------------------------------
+ * The paper treats 4-bit GPTQ only (Section 1); the same checkpoints family also stores 8-bit
+ * weights, with the same conventions at twice the field width (this reading is pinned by hand-packed
+ * words in the tests, like the 4-bit one):
+ *   q[k][n] = byte (k mod 4) of qweight[k/4][n]   (LSB first; qweight is int32[K/4][N])
+ *   z[g][n] = byte (n mod 4) of qzeros[g][n/4]    (qzeros is int32[G][N/4]), + zeros_plus (0 or 1)
+ *   w32[k][n] = float(q - z) * float(scales[g(k)][n])   exact: |q - z| <= 256 needs 9 bits
+ *   y[m][n] = sum_{k ascending} double(x[m][k]) * double(w32[k][n]) */
+static inline unsigned byte_of(int32_t word, int i)
+{
+    return ((uint32_t)word >> (8 * i)) & 255u;
+}
+
+void oracle_unpack_q8(const int32_t *qweight, int K, int N, uint8_t *q_out)
+{
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            q_out[(size_t)k * N + n] = (uint8_t)byte_of(qweight[(size_t)(k >> 2) * N + n], k & 3);
+}
+
+void oracle_unpack_z8(const int32_t *qzeros, int G, int N, uint8_t *z_out)
+{
+    for (int g = 0; g < G; g++)
+        for (int n = 0; n < N; n++)
+            z_out[(size_t)g * N + n] = (uint8_t)byte_of(qzeros[(size_t)g * (N / 4) + (n >> 2)], n & 3);
+}
+
+static inline float dequant_one_w8(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                                   const int32_t *g_idx, int N, int group_size, int zeros_plus, int k, int n)
+{
+    int g = group_of(g_idx, k, group_size);
+    int q = (int)byte_of(qweight[(size_t)(k >> 2) * N + n], k & 3);
+    int z = (int)byte_of(qzeros[(size_t)g * (N / 4) + (n >> 2)], n & 3) + zeros_plus;
+    float s = oracle_half_to_float(scales[(size_t)g * N + n]);
+    return (float)(q - z) * s;
+}
+
+void oracle_dequant_f32_w8(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                           const int32_t *g_idx, int K, int N, int group_size, int zeros_plus, float *w_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            w_out[(size_t)k * N + n] = dequant_one_w8(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+}
+
+void oracle_gemm_f64_w8(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                        const uint16_t *scales, const int32_t *g_idx,
+                        int M, int N, int K, int group_size, int zeros_plus, double *y_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; n++) {
+        for (int m = 0; m < M; m++) {
+            double acc = 0.0;
+            for (int k = 0; k < K; k++) {
+                float w = dequant_one_w8(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+                acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+            }
+            y_out[(size_t)m * N + n] = acc;
+        }
+    }
+}
+
+void oracle_gemm_f64_w8_at(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                           const uint16_t *scales, const int32_t *g_idx,
+                           int M, int N, int K, int group_size, int zeros_plus,
+                           const int32_t *rows, const int32_t *cols, int count, double *y_out)
+{
+    (void)M;
+    #pragma omp parallel for schedule(static)
+    for (int i = 0; i < count; i++) {
+        int m = rows[i], n = cols[i];
+        double acc = 0.0;
+        for (int k = 0; k < K; k++) {
+            float w = dequant_one_w8(qweight, qzeros, scales, g_idx, N, group_size, zeros_plus, k, n);
+            acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+        }
+        y_out[i] = acc;
+    }
+}

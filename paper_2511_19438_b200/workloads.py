@@ -143,6 +143,43 @@ def make_x(M: int, K: int, seed: int) -> np.ndarray:
     return _rng(seed).standard_normal((M, K), dtype=np.float32).astype(np.float16)
 
 
+def pack8_along_k(q: np.ndarray) -> np.ndarray:
+    """uint8[K, N] bytes -> int32[K/4, N], byte i of a word = row 4r+i (8-bit weights)."""
+    K, N = q.shape
+    assert K % 4 == 0
+    q32 = q.astype(np.uint32).reshape(K // 4, 4, N)
+    w = np.zeros((K // 4, N), dtype=np.uint32)
+    for i in range(4):
+        w |= q32[:, i, :] << np.uint32(8 * i)
+    return w.view(np.int32)
+
+
+def pack8_along_n(z: np.ndarray) -> np.ndarray:
+    """uint8[G, N] bytes -> int32[G, N/4], byte j of a word = column 4c+j (8-bit zero points)."""
+    G, N = z.shape
+    assert N % 4 == 0
+    z32 = z.astype(np.uint32).reshape(G, N // 4, 4)
+    w = np.zeros((G, N // 4), dtype=np.uint32)
+    for j in range(4):
+        w |= z32[:, :, j] << np.uint32(8 * j)
+    return w.view(np.int32)
+
+
+def make_linear_w8(K: int, N: int, seed: int, group_size: int = GROUP_SIZE, act_order: bool = False,
+                   zeros_minus_one: bool = False) -> QuantLinear:
+    """Random 8-bit GPTQ layer: qweight int32[K/4, N] and qzeros int32[G, N/4] drawn as uniform 32-bit words (every
+    byte uniform on 0..255), scales and g_idx as for the 4-bit layers.  With ``zeros_minus_one`` no stored zero point
+    is 255 (its meaning, 256, has no place in the library's tiling and real checkpoints centre the zero point)."""
+    assert K % 8 == 0 and N % 8 == 0 and K % group_size == 0
+    G = K // group_size
+    r = _rng(seed)
+    qweight = r.integers(0, 1 << 32, size=(K // 4, N), dtype=np.uint32).view(np.int32)
+    z = r.integers(0, 255 if zeros_minus_one else 256, size=(G, N), dtype=np.uint32).astype(np.uint8)
+    scales = make_scales(G, N, seed ^ 0x5CA1E5)
+    g_idx = make_g_idx(K, group_size, seed ^ 0x61D7) if act_order else None
+    return QuantLinear(K, N, group_size, qweight, pack8_along_n(z), scales, g_idx, seed, zeros_minus_one)
+
+
 def bf16_bits(a: np.ndarray) -> np.ndarray:
     """Finite float values -> the bit patterns (uint16) of the nearest bfloat16, ties to even.  Inputs for the
     bfloat16 variant travel in this form because numpy has no bfloat16 type."""

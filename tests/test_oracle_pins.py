@@ -512,3 +512,111 @@ def test_coarse_groups_and_per_channel_against_library_matmul(gs, act):
                        rtol=1e-12, atol=1e-12)
     if gs == K:
         assert np.array_equal(w, (q - z[0][None, :]) * L.scales[0].astype(np.float64)[None, :])
+
+
+# --------------------------------------------------------------------------- 8-bit weights
+def local_pack_bytes(vals_4):
+    """Test-local packer for 8-bit fields: the 32-bit word digit by digit in base 256 (byte 0 least significant)."""
+    word = 0
+    for i, v in enumerate(vals_4):
+        assert 0 <= int(v) <= 255
+        word += int(v) * (256 ** i)
+    return word
+
+
+def local_pack8_k(q):
+    K, N = q.shape
+    out = np.zeros((K // 4, N), dtype=np.uint32)
+    for r in range(K // 4):
+        for n in range(N):
+            out[r, n] = local_pack_bytes(q[4 * r:4 * r + 4, n])
+    return out.view(np.int32)
+
+
+def local_pack8_n(z):
+    G, N = z.shape
+    out = np.zeros((G, N // 4), dtype=np.uint32)
+    for g in range(G):
+        for c in range(N // 4):
+            out[g, c] = local_pack_bytes(z[g, 4 * c:4 * c + 4])
+    return out.view(np.int32)
+
+
+def test_w8_unpack_hand_typed_words():
+    """Words typed as hex and decoded by hand: 0x04030201 holds rows 1, 2, 3, 4 (least significant byte first), the
+    sign bit is just the top bit of the fourth byte, and a zero-point word holds four neighbouring columns."""
+    qweight = np.array([[0x04030201, 0xFF00807F], [0x80000000, 0x12345678]], dtype=np.uint32).view(np.int32)
+    want_q = np.array([[1, 0x7F], [2, 0x80], [3, 0x00], [4, 0xFF],
+                       [0, 0x78], [0, 0x56], [0, 0x34], [0x80, 0x12]], dtype=np.uint8)
+    assert np.array_equal(oracle.unpack_q8(qweight), want_q)
+    qzeros = np.array([[0xDEADBEEF, 0x00FF0102]], dtype=np.uint32).view(np.int32)
+    assert np.array_equal(oracle.unpack_z8(qzeros), np.array([[0xEF, 0xBE, 0xAD, 0xDE, 0x02, 0x01, 0xFF, 0x00]], dtype=np.uint8))
+    # the generator's packers agree with the digit-by-digit ones
+    r = np.random.default_rng(3)
+    q = r.integers(0, 256, (16, 8)).astype(np.uint8)
+    z = r.integers(0, 256, (2, 8)).astype(np.uint8)
+    assert np.array_equal(wl.pack8_along_k(q), local_pack8_k(q)) and np.array_equal(wl.pack8_along_n(z), local_pack8_n(z))
+    assert np.array_equal(oracle.unpack_q8(local_pack8_k(q)), q) and np.array_equal(oracle.unpack_z8(local_pack8_n(z)), z)
+
+
+@pytest.mark.parametrize("act_order", [False, True])
+@pytest.mark.parametrize("zm1", [False, True])
+def test_w8_dequant_and_gemm_match_rational_brute_force(act_order, zm1):
+    K, N, M, gs = 16, 8, 2, 8
+    r = np.random.default_rng(17)
+    q = r.integers(0, 256, (K, N)).astype(np.uint8)
+    z = r.integers(0, 256, (K // gs, N)).astype(np.uint8)
+    s = np.array([[1.0, 0.5, 0.25, 2.0, 0.125, 3.0, 0.0625, 1.5], [0.5, 1.0, 2.0, 0.75, 1.0, 0.25, 4.0, 0.375]], dtype=np.float16)
+    groups = [int(g) for g in r.permutation(K) // gs] if act_order else [k // gs for k in range(K)]
+    q[0, 0], z[groups[0], 0] = 0, 255               # the extremes: -255 (or -256 with the older convention)
+    q[1, 1], z[groups[1], 1] = 255, 0
+    g_idx = np.array(groups, dtype=np.int32) if act_order else None
+    x = np.array([[1.0] * K, [0.5, -2.0, 3.0, 0.25, 1.5, -1.0, 7.0, -0.125, 2.0, 0.0, -3.0, 1.0, 0.75, -4.0, 6.0, 1.25]], dtype=np.float16)
+    qw, qz = local_pack8_k(q), local_pack8_n(z)
+    w = oracle.dequant_f32_w8(qw, qz, s, g_idx, gs, zeros_minus_one=zm1)
+    for k in range(K):
+        for n in range(N):
+            assert float(w[k, n]) == (int(q[k, n]) - int(z[groups[k], n]) - int(zm1)) * float(s[groups[k], n]), (k, n)
+    assert w[0, 0] == (-256.0 if zm1 else -255.0) * float(s[groups[0], 0])
+    want = brute_force_y(x, q.astype(np.int64), z.astype(np.int64) + int(zm1), s, groups)
+    got = oracle.gemm_f64_w8(x, qw, qz, s, g_idx, gs, zeros_minus_one=zm1)
+    for m in range(M):
+        for n in range(N):
+            assert Fraction(float(got[m, n])) == want[m][n], (m, n)
+
+
+def test_w8_with_empty_high_nibbles_is_the_4bit_layer():
+    """An 8-bit layer whose weights and zero points are all below 16 is the 4-bit layer with the same values: ties the
+    8-bit functions to the 4-bit ones, which have their own pins."""
+    K, N, M, gs = 256, 16, 3, 64
+    r = np.random.default_rng(23)
+    q = r.integers(0, 16, (K, N)).astype(np.uint8)
+    z = r.integers(0, 16, (K // gs, N)).astype(np.uint8)
+    s = wl.make_scales(K // gs, N, 5)
+    g_idx = wl.make_g_idx(K, gs, 6)
+    x = wl.make_x(M, K, 7)
+    L4 = wl.make_linear_from_values(q, z, s, gs, g_idx)
+    for zm1 in (False, True):
+        a = oracle.gemm_f64_w8(x, wl.pack8_along_k(q), wl.pack8_along_n(z), s, g_idx, gs, zeros_minus_one=zm1)
+        b = oracle.gemm_f64(x, L4.qweight, L4.qzeros, L4.scales, g_idx, gs, zeros_minus_one=zm1)
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("K,N,act,gs", [(4096, 1024, False, 128), (1024, 512, True, 128), (512, 256, True, 32)])
+def test_w8_against_library_fp64_matmul(K, N, act, gs):
+    L = wl.make_linear_w8(K, N, seed=wl.seed_for("pin-w8", K, N, act), group_size=gs, act_order=act)
+    x = wl.make_x(3, K, wl.seed_for("pin-w8-x", K))
+    sh = (8 * np.arange(4, dtype=np.uint32))
+    q = ((L.qweight.view(np.uint32)[:, None, :] >> sh[None, :, None]) & 255).reshape(K, N).astype(np.int64)
+    z = ((L.qzeros.view(np.uint32)[:, :, None] >> sh[None, None, :]) & 255).reshape(K // gs, N).astype(np.int64)
+    grp = L.g_idx if act else np.arange(K) // gs
+    w = (q - z[grp]).astype(np.float64) * L.scales[grp].astype(np.float64)
+    got = oracle.gemm_f64_w8(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs)
+    assert np.allclose(got, x.astype(np.float64) @ w, rtol=1e-11, atol=1e-9)
+    assert np.array_equal(oracle.dequant_f32_w8(L.qweight, L.qzeros, L.scales, L.g_idx, gs).astype(np.float64), w)
+    # closed-form spread: var(q - z) = 2 * (256^2 - 1) / 12
+    es2 = wl.SCALE_FLOOR ** 2 + 2 * wl.SCALE_FLOOR * wl.SCALE_SIGMA * math.sqrt(2 / math.pi) + wl.SCALE_SIGMA ** 2
+    assert abs(got.std() / math.sqrt(K * (2 * (256 ** 2 - 1) / 12) * es2) - 1) < 0.06
+    rows = np.array([0, 2, 1, 1], dtype=np.int32)
+    cols = np.array([0, N - 1, 17, 18], dtype=np.int32)
+    assert np.array_equal(oracle.gemm_f64_w8_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, rows, cols), got[rows, cols])
