@@ -221,6 +221,43 @@ int gptq_gemm_silu_mul_scatter(const void *x, const void *qweight, const void *q
  * skipped). */
 int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream);
 
+/* ---- 8-bit weights (no counterpart in the paper, which treats 4-bit GPTQ only - Section 1) ------------------------
+ * The checkpoint conventions at twice the field width: qweight int32[K/4, N], byte i of a word = row 4 r + i (least
+ * significant first); qzeros int32[G, N/4], byte j of a word = column 4 c + j; scales fp16[G, N]; g_idx int32[K].
+ * w[k,n] = (q - z) * s with q, z in 0..255 (GPTQ_FORMAT_ZEROS_MINUS_ONE: the stored byte is z - 1; a stored 255 under
+ * that convention, z = 256, is refused with GPTQ_ERR_UNSUPPORTED).
+ * An 8-bit weight is two nibbles, (q - z) s = (hi - zh) (16 s) + (lo - zl) s: gptq_repack_w8 stores the layer as a 4-bit
+ * layer of 2 K rows (rows 0..K-1 the high nibbles with scales 16 s, rows K..2K-1 the low nibbles) in the usual tiled
+ * layout, and gptq_gemm_w8 gathers x into [x | x] in that layer's row order and runs the 4-bit kernels on 2 K rows.  One
+ * byte per weight is streamed, as the format requires; scales and zero points take twice their canonical bytes.
+ * Requirements: as gptq_repack (group_size 32, 64 or a multiple of 128; K % 128 == 0; N % 128 == 0), scales < 4096. */
+
+/* Bytes of each output of gptq_repack_w8: which = 0 qweight_out, 1 qzeros_out, 2 scales_out, 3 perm_out (int32[2 K],
+ * always needed).  0 for an invalid argument. */
+size_t gptq_repack_w8_bytes(int which, int N, int K, int group_size);
+/* Bytes of the device scratch buffer gptq_repack_w8 needs (about K * N: the two planes in canonical 4-bit form). */
+size_t gptq_repack_w8_scratch_bytes(int N, int K, int group_size);
+/* One-time repack of a canonical 8-bit layer.  All pointers are device pointers; outputs 16-byte aligned, scratch
+ * 256-byte aligned and of at least gptq_repack_w8_scratch_bytes (GPTQ_ERR_WORKSPACE otherwise); it may be freed once the
+ * stream has passed the call.  g_idx may be NULL when act_order is 0.  perm_out[i] (i < 2 K) is the column of x that row i
+ * of the stacked layer multiplies.  The call synchronises the stream (it reads back the validation results: GPTQ_ERR_GIDX
+ * as for gptq_repack, GPTQ_ERR_UNSUPPORTED for a zero point of 256).  format: 0 or GPTQ_FORMAT_ZEROS_MINUS_ONE. */
+int gptq_repack_w8(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                   void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, void *scratch,
+                   size_t scratch_bytes, int N, int K, int group_size, int act_order, int format, void *stream);
+/* fp32 w[K, N] of an 8-bit layer, bit-exact (the product float(q - z) * float(s) is exact): repacked = 0 reads the
+ * canonical buffers (g_idx used when act_order != 0, format as above); repacked = 1 reads gptq_repack_w8's outputs,
+ * g_idx = its perm_out (required), and recombines the two planes. */
+int gptq_dequant_f32_w8(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx, float *w_out,
+                        int N, int K, int group_size, int act_order, int repacked, int format, void *stream);
+/* y fp16[M, N] = x fp16[M, K] . dequant(W8)[K, N] for the outputs of gptq_repack_w8 (perm = its perm_out, 16-byte
+ * aligned).  Needs the registered workspace: gptq_workspace_bytes(M, N, 2 * K, group_size, 1) bytes, for the gathered
+ * activations.  K and group_size are the checkpoint's.  Stream semantics, kernels by M, accuracy bar and error codes as
+ * for gptq_gemm with act_order = 1; up to 16 token rows the integers are exact and the scales join in fp32, above that
+ * each plane's scaled weight is rounded to fp16 once. */
+int gptq_gemm_w8(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *perm,
+                 void *y, int M, int N, int K, int group_size, void *stream);
+
 /* Process-wide switch: with enable != 0, gptq_gemm runs problems with M >= 256 and an even number
  * of 128-column panels on CTA pairs (tcgen05.mma.cta_group::2: two SMs share one 256 x 256 x 16 MMA and
  * each loads half of the x tile).  Same arithmetic and tolerance as the default kernel; it halves the

@@ -6,6 +6,7 @@
 #include "gptq_splitk.cuh"
 #include "gptq_umma.cuh"
 #include "gptq_umma2.cuh"
+#include "gptq_w8.cuh"
 
 #include <atomic>
 #include <cstdio>
@@ -473,6 +474,95 @@ int gptq_gemm_silu_mul_scatter(const void *x, const void *qweight, const void *q
     if (!out_index) return GPTQ_ERR_NULL;
     return gemm_dispatch(x, qweight, qzeros, scales, g_idx, out, M, N, K, group_size, act_order, 1, nullptr, nullptr, out_index,
                          stream);
+}
+
+// ---- 8-bit weights: two stacked 4-bit planes (gptq_w8.cuh) ----------------------------------------------------------
+
+static int check_w8(int N, int K, int &group_size, int format)
+{
+    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    return check_fast_path(N, K, group_size);     // K % 128 == 0: a 128-row tile never spans the two planes
+}
+
+size_t gptq_repack_w8_bytes(int which, int N, int K, int group_size)
+{
+    int tiled = group_size;
+    if (K < 8 || K > (1 << 29) || check_w8(N, K, tiled, 0) != GPTQ_OK) return 0;
+    return gptq_repack_bytes(which, N, 2 * K, group_size, 1);
+}
+
+size_t gptq_repack_w8_scratch_bytes(int N, int K, int group_size)
+{
+    int tiled = group_size;
+    if (K < 8 || K > (1 << 29) || check_w8(N, K, tiled, 0) != GPTQ_OK) return 0;
+    return w8_scratch_layout(N, K, group_size).total;
+}
+
+int gptq_repack_w8(const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                   void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, void *scratch,
+                   size_t scratch_bytes, int N, int K, int group_size, int act_order, int format, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out || !perm_out || !scratch)
+        return GPTQ_ERR_NULL;
+    if (act_order && !g_idx) return GPTQ_ERR_NULL;
+    if (K > (1 << 29)) return GPTQ_ERR_SHAPE;
+    int tiled = group_size;
+    int st = check_w8(N, K, tiled, format);
+    if (st) return st;
+    if (!aligned16(qweight_out) || !aligned16(qzeros_out) || !aligned16(scales_out) || !aligned16(perm_out) ||
+        (reinterpret_cast<uintptr_t>(scratch) & 255u))
+        return GPTQ_ERR_ALIGN;
+    if (scratch_bytes < w8_scratch_layout(N, K, group_size).total) return GPTQ_ERR_WORKSPACE;
+    return launch_w8_repack(qweight, qzeros, scales, act_order ? g_idx : nullptr, qweight_out, qzeros_out, scales_out,
+                            perm_out, scratch, N, K, group_size, (format & GPTQ_FORMAT_ZEROS_MINUS_ONE) ? 1 : 0,
+                            (cudaStream_t)stream);
+}
+
+int gptq_dequant_f32_w8(const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx, float *w_out,
+                        int N, int K, int group_size, int act_order, int repacked, int format, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !w_out || ((act_order || repacked) && !g_idx)) return GPTQ_ERR_NULL;
+    if (repacked != 0 && repacked != 1) return GPTQ_ERR_LAYOUT;
+    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    if (N % 4) return GPTQ_ERR_SHAPE;
+    if (repacked) {
+        st = check_fast_path(N, K, group_size);
+        if (st) return st;
+    }
+    return launch_w8_dequant_f32(qweight, qzeros, scales, (act_order || repacked) ? g_idx : nullptr, w_out, N, K,
+                                 group_size, repacked, (format & GPTQ_FORMAT_ZEROS_MINUS_ONE) ? 1 : 0, (cudaStream_t)stream);
+}
+
+int gptq_gemm_w8(const void *x, const void *qweight, const void *qzeros, const void *scales, const int32_t *perm,
+                 void *y, int M, int N, int K, int group_size, void *stream)
+{
+    if (!x || !qweight || !qzeros || !scales || !perm || !y) return GPTQ_ERR_NULL;
+    if (K > (1 << 29)) return GPTQ_ERR_SHAPE;
+    int st = check_shape(M, N, K, group_size);
+    if (st) return st;
+    if (!aligned16(x) || !aligned16(qweight) || !aligned16(qzeros) || !aligned16(scales) || !aligned16(y) || !aligned16(perm))
+        return GPTQ_ERR_ALIGN;
+    int tiled = group_size;
+    st = check_fast_path(N, K, tiled);
+    if (st) return st;
+    int dev, sms;
+    st = current_device_sms(&dev, &sms);
+    if (st) return st;
+    Workspace ws;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = g_workspace[dev];
+    }
+    if (ws.ptr == nullptr || ws.bytes < gemm_workspace_need(M, 2 * K, 1)) return GPTQ_ERR_WORKSPACE;
+    st = launch_w8_gather_x((const __half *)x, perm, (__half *)ws.ptr, M, K, (cudaStream_t)stream);
+    if (st) return st;
+    // the stacked layer, its activations already in its row order
+    return gemm_dispatch(ws.ptr, qweight, qzeros, scales, nullptr, y, M, N, 2 * K, group_size, GPTQ_ACT_ORDER_PRESORTED, 0,
+                         nullptr, nullptr, nullptr, stream);
 }
 
 int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream)

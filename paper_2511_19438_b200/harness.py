@@ -156,3 +156,35 @@ def gemm_presorted(x_sorted: torch.Tensor, D: DeviceLinear, y: torch.Tensor | No
     B.check(B.gptq_gemm(x_sorted, D.qweight_t, D.qzeros_t, D.scales_t, None, y, M, D.N, D.K, D.group_size,
                         B.GPTQ_ACT_ORDER_PRESORTED, stream), "gptq_gemm (pre-sorted)")
     return y
+
+
+# ---- 8-bit layers (stored as two stacked 4-bit planes) ----------------------------------------------------------------
+
+def upload_and_repack_w8(L: QuantLinear, keep_canonical: bool = False, device="cuda") -> DeviceLinear:
+    """Uploads a canonical 8-bit layer (qweight int32[K/4, N], qzeros int32[G, N/4]) and repacks it with gptq_repack_w8.
+    The returned DeviceLinear keeps the checkpoint's K and group size; ``perm`` is int32[2 K]."""
+    qw, qz, sc = to_device(L.qweight, device), to_device(L.qzeros, device), to_device(L.scales, device)
+    gi = to_device(L.g_idx, device) if L.act_order else None
+    outs = [torch.empty(B.gptq_repack_w8_bytes(w, L.N, L.K, L.group_size), dtype=torch.uint8, device=device) for w in range(3)]
+    perm = torch.empty(2 * L.K, dtype=torch.int32, device=device)
+    nscratch = B.gptq_repack_w8_scratch_bytes(L.N, L.K, L.group_size)
+    scratch = torch.empty(nscratch, dtype=torch.uint8, device=device)
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0
+    B.check(B.gptq_repack_w8(qw, qz, sc, gi, outs[0], outs[1], outs[2], perm, scratch, nscratch, L.N, L.K, L.group_size,
+                             L.act_order, fmt), "gptq_repack_w8")
+    torch.cuda.current_stream().synchronize()
+    canonical = (qw, qz, sc, gi) if keep_canonical else None
+    return DeviceLinear(L.K, L.N, L.group_size, L.act_order, outs[0], outs[1], outs[2], perm, canonical)
+
+
+def gemm_w8(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """y = x . dequant(W8) through gptq_gemm_w8 (the workspace must hold the gathered activations, see ensure_for_w8)."""
+    M = x.shape[0]
+    if y is None:
+        y = torch.empty((M, D.N), dtype=torch.float16, device=x.device)
+    B.check(B.gptq_gemm_w8(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, M, D.N, D.K, D.group_size, stream), "gptq_gemm_w8")
+    return y
+
+
+def ensure_for_w8(ws: "WorkspaceHolder", M: int, D: DeviceLinear) -> None:
+    ws.ensure(B.gptq_workspace_bytes(M, D.N, 2 * D.K, D.group_size, 1))

@@ -74,6 +74,21 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_repack_format(A16, A16, A16, None, A16 + 16, A16 + 32, A16 + 48, None, 128, 128, 64, 0, 8, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_dequant_f32_format(A16, A16, A16, None, A16, 128, 128, 128, 0, 0, B.GPTQ_FORMAT_GATE_UP, stream=0) == B.GPTQ_ERR_LAYOUT
     assert B.gptq_gemm_silu_mul(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
+    # the 8-bit entry points: argument checks come before any CUDA call
+    assert B.gptq_repack_w8_bytes(0, 256, 512, 128) == 512 * 256 and B.gptq_repack_w8_bytes(1, 256, 512, 128) == 2 * 4 * 128 + 16
+    assert B.gptq_repack_w8_bytes(2, 256, 512, 128) == 2 * 4 * 256 * 2 and B.gptq_repack_w8_bytes(3, 256, 512, 128) == 2 * 512 * 4
+    assert B.gptq_repack_w8_bytes(0, 256, 512, 16) == 0 and B.gptq_repack_w8_scratch_bytes(256, 512, 16) == 0
+    assert B.gptq_repack_w8_scratch_bytes(256, 512, 128) >= 512 * 256 + 2 * 4 * (128 + 512) + 2 * 512 * 4
+    assert B.gptq_repack_w8(A16, A16, A16, None, A16, A16, A16, None, A16, 1 << 30, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_repack_w8(A16, A16, A16, None, A16, A16, A16, A16, A16, 1 << 30, 128, 128, 128, 1, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_repack_w8(A16, A16, A16, None, A16, A16, A16, A16, A16, 1 << 30, 128, 128, 128, 0, 2, stream=0) == B.GPTQ_ERR_LAYOUT
+    assert B.gptq_repack_w8(A16, A16, A16, None, A16, A16, A16, A16, A16 + 16, 1 << 30, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_ALIGN
+    assert B.gptq_repack_w8(A16, A16, A16, None, A16, A16, A16, A16, A16 - A16 % 256 + 256, 10, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_WORKSPACE
+    assert B.gptq_gemm_w8(A16, A16, A16, A16, None, A16, 1, 128, 128, 128, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_w8(A16, A16, A16, A16, A16 + 4, A16, 1, 128, 128, 128, stream=0) == B.GPTQ_ERR_ALIGN
+    assert B.gptq_gemm_w8(A16, A16, A16, A16, A16, A16, 1, 128, 192, 64, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_dequant_f32_w8(A16, A16, A16, None, A16, 128, 128, 128, 0, 1, 0, stream=0) == B.GPTQ_ERR_NULL   # tiled: perm needed
+    assert B.gptq_dequant_f32_w8(A16, A16, A16, None, A16, 128, 128, 128, 0, 0, 4, stream=0) == B.GPTQ_ERR_LAYOUT
     # the bfloat16 matmul validates like gptq_gemm
     assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, A16, 1, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL

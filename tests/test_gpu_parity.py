@@ -1108,3 +1108,113 @@ def test_per_channel_bf16_gemm(ws):
         x_bits = wl.make_x_bf16(M, K, wl.seed_for("coarse-bf16-x", M))
         y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
         assert_close_bf16(y, oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, None, K), K, M)
+
+
+# ------------------------------------------------------------------------------- 8-bit weights
+W8_CASES = [(128, False, False), (128, True, True), (64, True, False), (32, False, True), (512, True, False)]
+
+
+@pytest.mark.parametrize("gs,act,zm1", W8_CASES)
+def test_w8_dequant_bit_exact(gs, act, zm1):
+    """Canonical 8-bit buffers and the repacked pair of 4-bit planes both dequantise to the oracle's bits."""
+    K, N = 512, 256
+    L = wl.make_linear_w8(K, N, seed=wl.seed_for("w8-dq", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    want = oracle.dequant_f32_w8(L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if zm1 else 0
+    D = H.upload_and_repack_w8(L, keep_canonical=True)
+    qw, qz, sc, gi = D.canonical
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    B.check(B.gptq_dequant_f32_w8(qw, qz, sc, gi, w, N, K, gs, act, 0, fmt), "dequant canonical")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    w.zero_()
+    B.check(B.gptq_dequant_f32_w8(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1, 0), "dequant tiled")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    perm = D.perm.cpu().numpy()
+    assert perm.min() >= 0 and perm.max() < K and np.array_equal(perm[:K], perm[K:])
+    assert np.array_equal(np.sort(perm[:K]), np.arange(K))
+    if not act:
+        assert np.array_equal(perm[:K], np.arange(K))
+
+
+@pytest.mark.parametrize("gs,act,zm1", W8_CASES)
+@pytest.mark.parametrize("M", [1, 8, 16, 40, 300])
+def test_w8_gemm_small_full_compare(gs, act, zm1, M, ws):
+    """8-bit layers on both kernel families.  y's spread is 16 times that of a 4-bit layer with the same scales, and so
+    is the error of the fp16-rounded weights: the absolute term of the bar scales with it (the relative term is as
+    stated)."""
+    K, N = 1024, 384
+    L = wl.make_linear_w8(K, N, seed=wl.seed_for("w8", gs, act, zm1), group_size=gs, act_order=act, zeros_minus_one=zm1)
+    x = wl.make_x(M, K, wl.seed_for("w8-x", M))
+    D = H.upload_and_repack_w8(L)
+    H.ensure_for_w8(ws, M, D)
+    y = H.gemm_w8(H.to_device(x), D).cpu().numpy().astype(np.float64)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    want = oracle.gemm_f64_w8(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+    err = np.abs(y - want)
+    finite = np.abs(want) < 60000                                  # fp16 output range
+    assert finite.mean() > 0.999
+    bound = 16 * 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(want)
+    assert np.all(err[finite] <= bound[finite]), f"max err {err[finite].max():.3e}"
+    if M <= 16:
+        tight = 16 * 1e-4 * math.sqrt(K / 4096) + 2.0 ** -11 * np.abs(want)
+        assert np.all(err[finite] <= tight[finite]), f"max err {err[finite].max():.3e}"
+
+
+def test_w8_integer_case_and_refusals(ws):
+    """Scales 1/16 and small-integer x: every term is a multiple of 1/16 and the sums are exact in fp32, so y is the
+    rounded exact product; then the argument checks of the 8-bit entry points."""
+    K, N = 512, 128
+    r = np.random.default_rng(31)
+    q = r.integers(0, 256, (K, N)).astype(np.uint8)
+    z = r.integers(0, 256, (K // 128, N)).astype(np.uint8)
+    L = wl.QuantLinear(K, N, 128, wl.pack8_along_k(q), wl.pack8_along_n(z), np.full((K // 128, N), 1 / 16, np.float16), None, 0)
+    D = H.upload_and_repack_w8(L)
+    for M in (3, 33):
+        xv = r.integers(-1, 2, (M, K)).astype(np.float16)
+        H.ensure_for_w8(ws, M, D)
+        y = H.gemm_w8(H.to_device(xv), D).cpu().numpy()
+        want = (xv.astype(np.float64) @ (q.astype(np.float64) - z[np.arange(K) // 128].astype(np.float64))) / 16
+        assert np.array_equal(oracle.gemm_f64_w8(xv, L.qweight, L.qzeros, L.scales, None, 128), want)
+        assert np.array_equal(y, want.astype(np.float16))
+    # a stored zero point of 255 under the minus-one convention means 256: refused, nothing tiled
+    zbad = z.copy()
+    zbad[1, 5] = 255
+    Lbad = wl.QuantLinear(K, N, 128, L.qweight, wl.pack8_along_n(zbad), L.scales, None, 0, True)
+    with pytest.raises(B.GptqError) as e:
+        H.upload_and_repack_w8(Lbad)
+    assert e.value.status == B.GPTQ_ERR_UNSUPPORTED
+    H.upload_and_repack_w8(wl.QuantLinear(K, N, 128, L.qweight, wl.pack8_along_n(zbad), L.scales, None, 0, False))   # fine as is
+    # argument checks
+    x = torch.zeros((2, K), dtype=torch.float16, device="cuda")
+    y = torch.zeros((2, N), dtype=torch.float16, device="cuda")
+    assert B.gptq_gemm_w8(x, D.qweight_t, D.qzeros_t, D.scales_t, None, y, 2, N, K, 128) == B.GPTQ_ERR_NULL
+    assert B.gptq_gemm_w8(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, 2, N, K, 16) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_set_workspace(None, 0) == B.GPTQ_OK
+    assert B.gptq_gemm_w8(x, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, y, 2, N, K, 128) == B.GPTQ_ERR_WORKSPACE
+    ws.buf = None
+    assert B.gptq_repack_w8_bytes(0, N, K, 128) == K * N and B.gptq_repack_w8_bytes(3, N, K, 128) == 2 * K * 4
+    assert B.gptq_repack_w8_bytes(0, N, K + 64, 64) == 0                # K % 128
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(y) == 0
+
+
+def test_w8_config_shape_sampled(ws):
+    """The 4096 x 4096 layer with 8-bit weights: M = 1 element by element, a prefill batch on sampled outputs."""
+    K, N = 4096, 4096
+    L = wl.make_linear_w8(K, N, seed=wl.seed_for("w8-config1"), act_order=True)
+    D = H.upload_and_repack_w8(L)
+    x = wl.make_x(1, K, wl.seed_for("w8-config1-x"))
+    H.ensure_for_w8(ws, 1, D)
+    y = H.gemm_w8(H.to_device(x), D).cpu().numpy().astype(np.float64)
+    want = oracle.gemm_f64_w8(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    assert np.all(np.abs(y - want) <= 16 * 1e-4 + 2.0 ** -11 * np.abs(want))
+    M = 512
+    x = wl.make_x(M, K, wl.seed_for("w8-config1-x", M))
+    H.ensure_for_w8(ws, M, D)
+    y = H.gemm_w8(H.to_device(x), D).cpu().numpy().astype(np.float64)
+    assert B.gptq_check_status() == B.GPTQ_OK
+    r = np.random.default_rng(13)
+    rows, cols = r.integers(0, M, 3000).astype(np.int32), r.integers(0, N, 3000).astype(np.int32)
+    rows[:4], cols[:4] = [0, 0, M - 1, M - 1], [0, N - 1, 0, N - 1]
+    want = oracle.gemm_f64_w8_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128, rows, cols)
+    assert np.all(np.abs(y[rows, cols] - want) <= 16 * 1e-2 + 1e-2 * np.abs(want))
