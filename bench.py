@@ -176,6 +176,13 @@ def bf16_scales(L, layer, name):
     return wl.make_scales_bf16(L.K // L.group_size, L.N, wl.seed_for("bench-bf16-scales", layer, name))
 
 
+def make_layer(spec, K, N, seed):
+    """One seeded layer of the workload: 4-bit, or 8-bit with --wbits 8."""
+    if spec.get("w8", False):
+        return wl.make_linear_w8(K, N, seed=seed, act_order=spec["act_order"])
+    return wl.make_linear(K, N, seed=seed, act_order=spec["act_order"])
+
+
 def build_problems(spec, layers, H, torch, device):
     """Uploads `layers` distinct seeded copies of every shape (repacked through the C ABI) and the
     activations; returns {M: [(D, x, y, name), ...]} in launch order (layer-major)."""
@@ -184,9 +191,12 @@ def build_problems(spec, layers, H, torch, device):
     host = {}
     for layer in range(layers):
         for name, (K, N) in spec["shapes"].items():
-            L = wl.make_linear(K, N, seed=wl.seed_for("bench", layer, name), act_order=spec["act_order"])
+            L = make_layer(spec, K, N, wl.seed_for("bench", layer, name))
             bf16 = spec.get("bf16", False)
-            D = H.upload_and_repack(L, scales_bf16_bits=bf16_scales(L, layer, name) if bf16 else None)
+            if spec.get("w8", False):
+                D = H.upload_and_repack_w8(L)
+            else:
+                D = H.upload_and_repack(L, scales_bf16_bits=bf16_scales(L, layer, name) if bf16 else None)
             if layer == 0:
                 host[name] = L
             for M in Ms:
@@ -209,7 +219,7 @@ def step_bytes_flops(spec, layers):
     f = {M: 0 for M in spec["Ms"]}
     for M in spec["Ms"]:
         for (K, N) in spec["shapes"].values():
-            b[M] += layers * wl.algorithmic_bytes(M, K, N, act_order=spec["act_order"])
+            b[M] += layers * wl.algorithmic_bytes(M, K, N, act_order=spec["act_order"], wbits=8 if spec.get("w8", False) else 4)
             f[M] += layers * wl.matmul_flops(M, K, N)
     return b, f
 
@@ -219,6 +229,10 @@ def launches_per_gemm(spec, M, name, sm_count):
     along K), plus the x gather with act-order."""
     from paper_2511_19438_b200 import binding as B
     K, N = spec["shapes"][name]
+    if spec.get("w8", False):       # the 4-bit kernels on the stacked planes (2 K rows), always behind the x gather
+        st, pl = B.gptq_plan(M, N, 2 * K, wl.GROUP_SIZE, 0, sm_count)
+        assert st == B.GPTQ_OK
+        return 2 + (1 if pl.tail_ctas > 0 else 0)
     st, pl = B.gptq_plan(M, N, K, wl.GROUP_SIZE, 1 if spec["act_order"] else 0, sm_count)
     assert st == B.GPTQ_OK
     return 1 + (1 if pl.tail_ctas > 0 else 0) + (1 if spec["act_order"] else 0)
@@ -230,6 +244,8 @@ def kernel_of(spec, M, sm_count):
     from paper_2511_19438_b200 import binding as B
     names = {}
     for (K, N) in spec["shapes"].values():
+        if spec.get("w8", False):
+            K = 2 * K
         st, pl = B.gptq_plan(M, N, K, wl.GROUP_SIZE, 1 if spec["act_order"] else 0, sm_count)
         assert st == B.GPTQ_OK
         names[B.plan_kernel_name(pl)] = names.get(B.plan_kernel_name(pl), 0) + K * N
@@ -246,8 +262,7 @@ def oracle_sample(spec, budget_s):
     small = min(shapes, key=lambda n: shapes[n][0] * shapes[n][1])
     Ms = [M for M in spec["Ms"] if M <= 16] or [16]
     ladder = [([small], Ms[:1]), (list(shapes), Ms[:1]), (list(shapes), Ms[:2]), (list(shapes), Ms)]
-    layer = {n: wl.make_linear(K, N, seed=wl.seed_for("bench", 0, n), act_order=spec["act_order"])
-             for n, (K, N) in shapes.items()}
+    layer = {n: make_layer(spec, K, N, wl.seed_for("bench", 0, n)) for n, (K, N) in shapes.items()}
     Lp = layer[small]
     bf16 = spec.get("bf16", False)
     make_x = wl.make_x_bf16 if bf16 else wl.make_x
@@ -274,10 +289,13 @@ def run_oracle_once(items, spec):
     for (L, x, M, n) in items:
         if scales is not None:
             oracle.gemm_f64_bf16(x, L.qweight, L.qzeros, scales[n], L.g_idx, L.group_size)
+        elif spec.get("w8", False):
+            oracle.gemm_f64_w8(x, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
         else:
             oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, L.group_size)
     dt = time.perf_counter() - t0
-    nbytes = sum(wl.algorithmic_bytes(M, L.K, L.N, act_order=L.act_order) for (L, x, M, n) in items)
+    nbytes = sum(wl.algorithmic_bytes(M, L.K, L.N, act_order=L.act_order, wbits=8 if spec.get("w8", False) else 4)
+                 for (L, x, M, n) in items)
     flops = sum(wl.matmul_flops(M, L.K, L.N) for (L, x, M, n) in items)
     return dt, nbytes, flops
 
@@ -357,12 +375,15 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
     need = 0
     for M, probs in per_m.items():
         for (D, x, y, _n) in probs:
+            if spec.get("w8", False):
+                need = max(need, B.gptq_workspace_bytes(M, D.N, 2 * D.K, D.group_size, 1))
             need = max(need, B.gptq_workspace_bytes(M, D.N, D.K, D.group_size, D.act_order))
     ws.ensure(need)
     bytes_m, flops_m = step_bytes_flops(spec, layers)
 
     bf16 = spec.get("bf16", False)
-    gemm = H.gemm_bf16 if bf16 else H.gemm
+    w8 = spec.get("w8", False)
+    gemm = H.gemm_bf16 if bf16 else H.gemm_w8 if w8 else H.gemm
 
     def run_m(M):
         for (D, x, y, _n) in per_m[M]:
@@ -443,7 +464,7 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
     step_problems = B.make_host_problems(step_items)
 
     def e2e_step():
-        st, bad = (B.gptq_gemm_host_batch_bf16 if bf16 else B.gptq_gemm_host_batch)(step_problems)
+        st, bad = (B.gptq_gemm_host_batch_bf16 if bf16 else B.gptq_gemm_host_batch_w8 if w8 else B.gptq_gemm_host_batch)(step_problems)
         B.check(st, f"gptq_gemm_host_batch (problem {bad})")
         stream.synchronize()   # the step's results are on the host
 
@@ -467,7 +488,7 @@ def measure_workload(name, spec, layers, steps, warmup, e2e_steps, env):
 
     sms = torch.cuda.get_device_properties(device).multi_processor_count
     launches_step = sum(launches_per_gemm(spec, M, nm, sms) for M in Ms for (_D, _x, _y, nm) in per_m[M])
-    kernels = {M: kernel_of(spec, M, sms) + (" bf16" if bf16 else "") for M in Ms}
+    kernels = {M: kernel_of(spec, M, sms) + (" bf16" if bf16 else " on 8-bit planes" if w8 else "") for M in Ms}
     out = dict(total_ms=total_ms, e2e_ms=e2e_ms, e2e_steps=e2e_steps, seg_ms=seg_ms, clocks=clocks, bytes_m=bytes_m,
                flops_m=flops_m, h2d=h2d, d2h=d2h, launches_step=launches_step, kernels=kernels,
                matmuls={M: len(per_m[M]) for M in Ms}, Ms=Ms)
@@ -486,17 +507,25 @@ def per_shape_m1(spec, env, reps=20):
     ws = H.WorkspaceHolder(device=device)
     for name, (K, N) in spec["shapes"].items():
         copies = max(2, math.ceil(600e6 / (K * N // 2)))
-        L = wl.make_linear(K, N, seed=wl.seed_for("per-shape", name), act_order=spec["act_order"])
+        w8 = spec.get("w8", False)
+        if w8:
+            copies = max(2, copies // 2)
+        L = make_layer(spec, K, N, wl.seed_for("per-shape", name))
         bf16 = spec.get("bf16", False)
-        gemm = H.gemm_bf16 if bf16 else H.gemm
-        Ds = [H.upload_and_repack(L, device=device, scales_bf16_bits=bf16_scales(L, 0, name) if bf16 else None)
-              for _ in range(copies)]
+        gemm = H.gemm_bf16 if bf16 else H.gemm_w8 if w8 else H.gemm
+        if w8:
+            Ds = [H.upload_and_repack_w8(L, device=device) for _ in range(copies)]
+        else:
+            Ds = [H.upload_and_repack(L, device=device, scales_bf16_bits=bf16_scales(L, 0, name) if bf16 else None)
+                  for _ in range(copies)]
         if bf16:
             x = H.bf16_from_bits(wl.make_x_bf16(1, K, wl.seed_for("per-shape-x", name)), device)
         else:
             x = H.to_device(wl.make_x(1, K, wl.seed_for("per-shape-x", name)), device)
         y = torch.empty((1, N), dtype=torch.bfloat16 if bf16 else torch.float16, device=device)
         ws.ensure_for(1, Ds[0])
+        if w8:
+            H.ensure_for_w8(ws, 1, Ds[0])
         with torch.cuda.stream(stream):
             for D in Ds:
                 gemm(x, D, y, stream=stream)
@@ -514,7 +543,7 @@ def per_shape_m1(spec, env, reps=20):
             e1.record(stream)
             stream.synchronize()
         us = 1e3 * e0.elapsed_time(e1) / reps / copies
-        gbs = wl.algorithmic_bytes(1, K, N) / us / 1e3
+        gbs = wl.algorithmic_bytes(1, K, N, wbits=8 if w8 else 4) / us / 1e3
         out[name] = {"K": K, "N": N, "us": round(us, 3), "GB/s": round(gbs, 1),
                      "pct_of_nominal": round(100 * gbs / NOMINAL_HBM_GBS, 2), "copies": copies}
         del Ds, g
@@ -585,12 +614,12 @@ def report_line(name, spec, layers, steps, warmup, r, world):
                    "matmuls_per_step": sum(n_matmuls[M] for M in Ms), "group_size": 128,
                    "act_order": spec["act_order"], "parallelism": f"{world} independent replica(s)",
                    "l2": f"inputs larger than L2: each M pass streams {round(bytes_m[Ms[0]] / 1e6)} MB of distinct weights",
-                   "timing": "CUDA events around CUDA-graph replays of the " + ("gptq_gemm_bf16" if spec.get("bf16", False) else "gptq_gemm") +
+                   "timing": "CUDA events around CUDA-graph replays of the " + ("gptq_gemm_bf16" if spec.get("bf16", False) else "gptq_gemm_w8" if spec.get("w8", False) else "gptq_gemm") +
                              " calls, one graph per M"},
         "clocks": clocks,
         "e2e": {"value": round(e2e_value, 2), "unit": unit, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
-                "api": ("one gptq_gemm_host_batch_bf16" if spec.get("bf16", False) else "one gptq_gemm_host_batch") +
+                "api": ("one gptq_gemm_host_batch_bf16" if spec.get("bf16", False) else "one gptq_gemm_host_batch_w8" if spec.get("w8", False) else "one gptq_gemm_host_batch") +
                        " call per step (x from pinned host memory, y back to it, per matmul)"},
         "gpu_launches": launches_step * steps,
         "per_M": per_m_report,
@@ -616,6 +645,8 @@ def main():
     ap.add_argument("--ms", default="", help="comma-separated subset of the workload's token counts (profiling small cases)")
     ap.add_argument("--cta-pairs", action="store_true", help="prefill on CTA pairs (tcgen05 cta_group::2), off by default")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--wbits", type=int, default=4, choices=[4, 8],
+                    help="8: the same workload with 8-bit GPTQ weights (gptq_repack_w8 / gptq_gemm_w8)")
     ap.add_argument("--dtype", default="f16", choices=["f16", "bf16"],
                     help="bf16: the same workload with bfloat16 activations and scales (gptq_gemm_bf16)")
     ap.add_argument("--prefill-steps", type=int, default=10,
@@ -633,6 +664,11 @@ def main():
         spec["Ms"] = tuple(int(m) for m in args.ms.split(","))
     if args.dtype == "bf16":
         spec["bf16"] = True
+    if args.wbits == 8:
+        if args.dtype == "bf16":
+            raise SystemExit("--wbits 8 runs with fp16 activations only")
+        spec["w8"] = True
+        spec["describes"] += " - with 8-bit weights (gptq_gemm_w8: two stacked 4-bit planes)"
     layers = args.layers or spec["layers"]
     if args.impl == "reference":
         run_reference(args, spec)
@@ -669,7 +705,7 @@ def main():
     # prefill workload after the decode one, and reports it as a sub-object of the same line.
     prefill = None
     if args.workload == "decode7b" and not args.ms and args.prefill_steps > 0:
-        pspec = dict(WORKLOADS["prefill7b"], bf16=spec.get("bf16", False))
+        pspec = dict(WORKLOADS["prefill7b"], bf16=spec.get("bf16", False), w8=spec.get("w8", False))
         prefill = measure_workload("prefill7b", pspec, pspec["layers"], args.prefill_steps, 3, min(args.prefill_steps, 5), env)
     shapes_m1 = None
     if args.workload == "decode7b" and not args.ms and world == 1:

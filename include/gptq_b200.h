@@ -324,6 +324,10 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
 /* The same pipeline for bfloat16 layers: every problem's x_host / y_host hold bfloat16 and its layer was repacked with
  * GPTQ_FORMAT_BF16; each matmul is a gptq_gemm_bf16.  Arguments, ordering and errors as above. */
 int gptq_gemm_host_batch_bf16(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
+/* The same pipeline for 8-bit layers (gptq_repack_w8): each matmul is a gptq_gemm_w8; a problem's g_idx is the layer's
+ * perm_out (required), act_order is ignored, K and group_size are the checkpoint's, and the registered workspace must
+ * cover the largest problem (gptq_workspace_bytes(M, N, 2 * K, group_size, 1)). */
+int gptq_gemm_host_batch_w8(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
 
 /* Synchronises `stream` and returns GPTQ_ERR_LAYOUT if a kernel since the last check met a layer whose tiling does
  * not fit the call (see GPTQ_FORMAT_GATE_UP), GPTQ_ERR_TIMEOUT if a kernel's bounded wait gave up (the flag is

@@ -88,6 +88,7 @@ _SIGNATURES = {
     "gptq_noalloc_scratch_bytes": (_sz, []),
     "gptq_gemm_host_batch": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_gemm_host_batch_bf16": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
+    "gptq_gemm_host_batch_w8": (_i, [ctypes.POINTER(gptq_host_problem_t), _i, _vp, ctypes.POINTER(_i)]),
     "gptq_check_status": (_i, [_vp]),
     "gptq_selftest_wait_timeout": (_i, [ctypes.c_uint, _vp]),
     "gptq_trace_reset": (_i, [_vp]),
@@ -284,6 +285,13 @@ def gptq_gemm_host_batch_bf16(problems, stream=None):
     """gptq_gemm_host_batch for bfloat16 layers and activations."""
     bad = ctypes.c_int(-1)
     st = _lib.gptq_gemm_host_batch_bf16(problems, len(problems), _stream(stream), ctypes.byref(bad))
+    return st, bad.value
+
+
+def gptq_gemm_host_batch_w8(problems, stream=None):
+    """gptq_gemm_host_batch for 8-bit layers (each problem's g_idx is the layer's perm_out)."""
+    bad = ctypes.c_int(-1)
+    st = _lib.gptq_gemm_host_batch_w8(problems, len(problems), _stream(stream), ctypes.byref(bad))
     return st, bad.value
 
 

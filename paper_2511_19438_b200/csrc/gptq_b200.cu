@@ -663,14 +663,15 @@ int gptq_gemm_noalloc(const void *x, const void *qweight, const void *qzeros, co
 
 } // extern "C"
 
-static int host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index, int bf16)
+// mode: 0 = fp16 layers (gptq_gemm), 1 = bfloat16 layers (gptq_gemm_bf16), 2 = 8-bit layers (gptq_gemm_w8)
+static int host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index, int mode)
 {
     if (!problems || count < 0) return GPTQ_ERR_NULL;
     for (int i = 0; i < count; ++i) {
         const gptq_host_problem_t &q = problems[i];
         int st = GPTQ_OK;
         if (!q.x_host || !q.y_host || !q.x_stage || !q.y_stage || !q.qweight || !q.qzeros || !q.scales ||
-            (q.act_order == 1 && !q.g_idx))
+            ((q.act_order == 1 || mode == 2) && !q.g_idx))
             st = GPTQ_ERR_NULL;
         if (!st) st = check_shape(q.M, q.N, q.K, q.group_size);
         if (!st && (!aligned16(q.x_stage) || !aligned16(q.y_stage) || !aligned16(q.qweight) || !aligned16(q.qzeros) ||
@@ -723,8 +724,11 @@ static int host_batch(const gptq_host_problem_t *problems, int count, void *stre
                 break;
             }
         if (st) break;
-        st = gemm_dispatch(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
-                           q.act_order, 0, nullptr, nullptr, nullptr, stream, bf16);
+        if (mode == 2)
+            st = gptq_gemm_w8(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size, stream);
+        else
+            st = gemm_dispatch(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
+                               q.act_order, 0, nullptr, nullptr, nullptr, stream, mode);
         if (st) {
             if (bad_index) *bad_index = i;
             break;
@@ -752,6 +756,11 @@ int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *s
 int gptq_gemm_host_batch_bf16(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
 {
     return host_batch(problems, count, stream, bad_index, 1);
+}
+
+int gptq_gemm_host_batch_w8(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index)
+{
+    return host_batch(problems, count, stream, bad_index, 2);
 }
 
 // ---- self-test of the bounded waits ------------------------------------------------------------

@@ -200,11 +200,11 @@ def make_scales_bf16(G: int, N: int, seed: int) -> np.ndarray:
 
 
 def algorithmic_bytes(M: int, K: int, N: int, group_size: int = GROUP_SIZE,
-                      act_order: bool = False) -> int:
+                      act_order: bool = False, wbits: int = 4) -> int:
     """Bytes the matmul must move: packed weights, scales, packed zeros,
     x, y and (act-order) the row permutation."""
     G = K // group_size
-    b = K * N // 2 + G * N * 2 + G * N // 2 + M * K * 2 + M * N * 2
+    b = K * N * wbits // 8 + G * N * 2 + G * N * wbits // 8 + M * K * 2 + M * N * 2
     if act_order:
         b += 4 * K
     return b

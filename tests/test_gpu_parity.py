@@ -1218,3 +1218,28 @@ def test_w8_config_shape_sampled(ws):
     rows[:4], cols[:4] = [0, 0, M - 1, M - 1], [0, N - 1, 0, N - 1]
     want = oracle.gemm_f64_w8_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128, rows, cols)
     assert np.all(np.abs(y[rows, cols] - want) <= 16 * 1e-2 + 1e-2 * np.abs(want))
+
+
+def test_w8_host_batch_step(ws):
+    """Three 8-bit matmuls (one act-order, one on the tcgen05 kernel) from pinned host memory and back."""
+    specs = [(1024, 256, 2, False), (640, 256, 5, True), (512, 384, 40, False)]
+    items, keep = [], []
+    for (K, N, M, act) in specs:
+        L = wl.make_linear_w8(K, N, seed=wl.seed_for("w8-batch", K, N, act), act_order=act)
+        D = H.upload_and_repack_w8(L)
+        x_np = wl.make_x(M, K, wl.seed_for("w8-batch-x", K, M))
+        xh = torch.from_numpy(x_np).pin_memory()
+        yh = torch.zeros((M, N), dtype=torch.float16).pin_memory()
+        xs = torch.empty((M, K), dtype=torch.float16, device="cuda")
+        ys = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        items.append((xh, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, yh, xs, ys, M, N, K, 128, act))
+        keep.append((L, x_np, yh, D))
+    ws.ensure(max(B.gptq_workspace_bytes(M, N, 2 * K, 128, 1) for (K, N, M, act) in specs))
+    st, bad = B.gptq_gemm_host_batch_w8(B.make_host_problems(items))
+    assert (st, bad) == (B.GPTQ_OK, -1)
+    torch.cuda.synchronize()
+    assert B.gptq_check_status() == B.GPTQ_OK
+    for (L, x_np, yh, _D), (K, N, M, act) in zip(keep, specs):
+        want = oracle.gemm_f64_w8(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+        err = np.abs(yh.numpy().astype(np.float64) - want)
+        assert np.all(err <= 16 * 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(want))
