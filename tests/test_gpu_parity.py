@@ -1243,3 +1243,24 @@ def test_w8_host_batch_step(ws):
         want = oracle.gemm_f64_w8(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
         err = np.abs(yh.numpy().astype(np.float64) - want)
         assert np.all(err <= 16 * 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(want))
+
+
+# ------------------------------------------------------------------------------- tensor-parallel shards on one GPU
+@pytest.mark.parametrize("act", [False, True])
+@pytest.mark.parametrize("M", [4, 48])
+def test_tensor_parallel_shards_run_one_after_another(act, M, ws):
+    """The shards of a layer, multiplied one after the other on this GPU: the column shards concatenate to the layer's
+    output and the row shards' partial outputs add up to it (the collectives themselves run in the gloo test)."""
+    from paper_2511_19438_b200 import tp
+    K, N, world = 1024, 512, 2
+    L = wl.make_linear(K, N, seed=wl.seed_for("tp-gpu", act), act_order=act)
+    x = wl.make_x(M, K, wl.seed_for("tp-gpu-x", M))
+    want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, 128)
+    cols = [run_gemm(tp.shard_columns(L, r, world), x, ws)[0] for r in range(world)]
+    assert_close(np.concatenate(cols, axis=1), want, K, M)
+    acc = np.zeros((M, N), dtype=np.float64)
+    for r in range(world):
+        rows = tp.row_shard_rows(L, r, world)
+        acc += run_gemm(tp.shard_rows(L, r, world), np.ascontiguousarray(x[:, rows]), ws)[0].astype(np.float64)
+    err = np.abs(acc - want)
+    assert np.all(err <= 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(want))
