@@ -1264,3 +1264,51 @@ def test_tensor_parallel_shards_run_one_after_another(act, M, ws):
         acc += run_gemm(tp.shard_rows(L, r, world), np.ascontiguousarray(x[:, rows]), ws)[0].astype(np.float64)
     err = np.abs(acc - want)
     assert np.all(err <= 1e-2 * math.sqrt(K / 4096) + 1e-2 * np.abs(want))
+
+
+# ------------------------------------------------------------------------------- seeded sweep over odd shapes
+def _sweep_cases():
+    r = np.random.default_rng(20260101)
+    cases = []
+    for i in range(60):
+        K = 128 * int(r.integers(1, 19))                 # 128 .. 2304: one group up to 18, odd group counts included
+        N = 128 * int(r.integers(1, 10))                 # 1 .. 9 panels
+        M = int(r.choice([1, 2, 3, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 257, 300]))
+        kind = ["f16", "bf16", "w8"][i % 3]
+        gs = int(r.choice([32, 64, 128, 128, 128]))
+        if r.random() < 0.15:
+            gs = K                                        # per-channel
+        cases.append((kind, K, N, M, gs, bool(r.random() < 0.5), bool(r.random() < 0.3)))
+    return cases
+
+
+@pytest.mark.parametrize("kind,K,N,M,gs,act,zm1", _sweep_cases())
+def test_seeded_shape_sweep(kind, K, N, M, gs, act, zm1, ws):
+    """Sixty seeded (format, K, N, M, group size, act-order, zero convention) combinations, single groups, single panels
+    and token counts around every tile boundary among them: each result element by element against the oracle."""
+    seed = wl.seed_for("sweep", kind, K, N, M, gs, act, zm1)
+    if kind == "w8":
+        L = wl.make_linear_w8(K, N, seed=seed, group_size=gs, act_order=act, zeros_minus_one=zm1)
+        x = wl.make_x(M, K, seed ^ 1)
+        D = H.upload_and_repack_w8(L)
+        H.ensure_for_w8(ws, M, D)
+        y = H.gemm_w8(H.to_device(x), D).cpu().numpy().astype(np.float64)
+        assert B.gptq_check_status() == B.GPTQ_OK
+        want = oracle.gemm_f64_w8(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+        assert np.all(np.abs(y - want) <= 16 * 1e-2 * max(1.0, math.sqrt(K / 4096)) + 1e-2 * np.abs(want))
+        return
+    L = wl.make_linear(K, N, seed=seed, group_size=gs, act_order=act, zeros_minus_one=zm1)
+    if kind == "bf16":
+        s_bits = wl.make_scales_bf16(K // gs, N, seed ^ 2)
+        x_bits = wl.make_x_bf16(M, K, seed ^ 1)
+        y, _ = run_gemm_bf16(L, s_bits, x_bits, ws)
+        want = oracle.gemm_f64_bf16(x_bits, L.qweight, L.qzeros, s_bits, L.g_idx, gs, zeros_minus_one=zm1)
+        got = torch.from_numpy(y.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
+        assert np.all(np.abs(got - want) <= 8e-2 * max(1.0, math.sqrt(K / 4096)) + 1e-2 * np.abs(want))
+        return
+    x = wl.make_x(M, K, seed ^ 1)
+    y, _ = run_gemm(L, x, ws)
+    want = oracle.gemm_f64(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, zeros_minus_one=zm1)
+    # below K = 4096 the stated bar shrinks faster than the error of layers with few groups does (see the header):
+    # the sweep holds the bar at its K = 4096 value there
+    assert np.all(np.abs(y.astype(np.float64) - want) <= 1e-2 * max(1.0, math.sqrt(K / 4096)) + 1e-2 * np.abs(want))
