@@ -311,15 +311,18 @@ typedef struct {
 /* A step of matmuls whose activations live in host memory (the linears of a decode step, configs of
  * Section 4's serving setting): for each problem in order, on `stream`: copy x to the device, gptq_gemm,
  * copy y back - the same results as `count` gptq_gemm_host calls, but pipelined: the copies run on two
- * internal streams (created on first use), so x of problem i+1 goes up and y of problem i-1 comes down
- * while matmul i runs; the matmuls themselves stay in order on `stream`, and `stream` completes after
- * the last copy.  Staging buffers may be shared between problems (reuse waits for the earlier user).
+ * internal streams (created on first use) in chunks of consecutive problems (up to 16, up to 2 MiB of activations and
+ * results, none sharing a staging buffer with another of the last few chunks; large problems go one by one): the x of a chunk go up, its matmuls run back to back on `stream`, its y come down, and chunk c+1 goes up
+ * while chunk c computes and chunk c-1 comes down; the matmuls themselves stay in order on `stream`, and `stream`
+ * completes after the last copy.  Staging buffers may be shared between problems (reuse waits for the earlier user;
+ * problems that share one never sit in the same chunk).
  * All problems are validated before anything is enqueued; on an invalid problem *bad_index (if not
  * NULL) receives its index and nothing runs.  If a later step fails, `stream` is still joined with the
  * internal streams before the error is returned.  The internal streams and events belong to the device:
  * concurrent calls on one device (several host threads, or several user streams) are serialised by a lock
- * for the duration of the enqueue.  Not capturable in a CUDA graph (it records and waits on events of
- * internal streams). */
+ * for the duration of the enqueue.  The call is stream-ordered (the internal streams fork from `stream` and join it
+ * again), so after one ordinary call - which creates the internal streams and events - it may be captured into a CUDA
+ * graph and replayed: every replay copies the host buffers as they are then. */
 int gptq_gemm_host_batch(const gptq_host_problem_t *problems, int count, void *stream, int *bad_index);
 /* The same pipeline for bfloat16 layers: every problem's x_host / y_host hold bfloat16 and its layer was repacked with
  * GPTQ_FORMAT_BF16; each matmul is a gptq_gemm_bf16.  Arguments, ordering and errors as above. */

@@ -11,6 +11,7 @@
 #include <atomic>
 #include <cstdio>
 #include <mutex>
+#include <unordered_map>
 #include <vector>
 
 namespace gptq {
@@ -685,7 +686,7 @@ static int host_batch(const gptq_host_problem_t *problems, int count, void *stre
         }
     }
     if (count == 0) return GPTQ_OK;
-    // Three-stage pipeline over two internal copy streams: x_i goes up while matmul i-1 runs and y_i-1 comes down.
+    // Three-stage pipeline over two internal copy streams: activations go up while earlier matmuls run and their results come down.
     int dev, sms;
     int st = current_device_sms(&dev, &sms);
     if (st) return st;
@@ -707,36 +708,89 @@ static int host_batch(const gptq_host_problem_t *problems, int count, void *stre
     if ((st = check(cudaStreamWaitEvent(pipe->in, ev_start, 0)))) return st;
     if ((st = check(cudaStreamWaitEvent(pipe->out, ev_start, 0)))) return st;
     // from here on the internal streams are forked off `stream`: every exit goes through the join below
-    for (int i = 0; i < count && !st; ++i) {
-        const gptq_host_problem_t &q = problems[i];
-        // a staging buffer shared with an earlier problem is reused only after that problem is done with it
-        for (int j = i - 1; j >= 0 && !st; --j)
-            if (problems[j].x_stage == q.x_stage) {
-                st = check(cudaStreamWaitEvent(pipe->in, ev_g[j], 0));
-                break;
+    // The problems go through the pipeline in CHUNKS: a chunk is a run of consecutive problems that share no staging
+    // buffer (at most kChunk of them).  All x of a chunk are copied up, then its matmuls run back to back on `stream`
+    // (consecutive launches overlap through programmatic dependent launch - a dependency on another stream between
+    // every two of them would cost about a microsecond each), then all its y are copied down; chunk c + 1 is copied up
+    // while chunk c computes and chunk c - 1 comes down.  Events: ev_x[c] chunk c is up, ev_g[c] computed, ev_y[c] down.
+    // A chunk that reaches back to a staging buffer used d problems earlier must wait for that problem's chunk, so the
+    // pipeline only overlaps if chunks are short against d: a chunk holds at most d / 3 problems (one problem when
+    // buffers are reused every few problems, kChunk when every problem has its own).
+    constexpr int kChunk = 16;
+    std::vector<int> reuse((size_t)count);
+    {
+        std::unordered_map<const void *, int> last_index;     // staging buffer -> the last problem that used it
+        for (int i = 0; i < count; ++i) {
+            int d = 3 * kChunk;
+            for (const void *buf : {(const void *)problems[i].x_stage, (const void *)problems[i].y_stage}) {
+                auto it = last_index.find(buf);
+                if (it != last_index.end() && i - it->second < d) d = i - it->second;
             }
-        if (!st) st = check(cudaMemcpyAsync(q.x_stage, q.x_host, (size_t)q.M * q.K * sizeof(__half), cudaMemcpyHostToDevice, pipe->in));
-        if (!st) st = check(cudaEventRecord(ev_x[i], pipe->in));
-        if (!st) st = check(cudaStreamWaitEvent(s, ev_x[i], 0));
-        for (int j = i - 1; j >= 0 && !st; --j)
-            if (problems[j].y_stage == q.y_stage) {
-                st = check(cudaStreamWaitEvent(s, ev_y[j], 0));
-                break;
-            }
-        if (st) break;
-        if (mode == 2)
-            st = gptq_gemm_w8(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size, stream);
-        else
-            st = gemm_dispatch(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
-                               q.act_order, 0, nullptr, nullptr, nullptr, stream, mode);
-        if (st) {
-            if (bad_index) *bad_index = i;
-            break;
+            reuse[(size_t)i] = d;
+            last_index[problems[i].x_stage] = i;
+            last_index[problems[i].y_stage] = i;
         }
-        st = check(cudaEventRecord(ev_g[i], s));
-        if (!st) st = check(cudaStreamWaitEvent(pipe->out, ev_g[i], 0));
-        if (!st) st = check(cudaMemcpyAsync(q.y_host, q.y_stage, (size_t)q.M * q.N * sizeof(__half), cudaMemcpyDeviceToHost, pipe->out));
-        if (!st) st = check(cudaEventRecord(ev_y[i], pipe->out));
+    }
+    // staging buffer -> the latest chunk whose matmuls read it as x / whose copies down read it as y
+    std::unordered_map<const void *, int> read_as_x, copied_as_y;
+    int n_chunks = 0;
+    for (int i0 = 0; i0 < count && !st;) {
+        // ... and at most kChunkBytes of activations and results: large problems (prefill) keep one problem per chunk,
+        // where the copies, not the dependencies, set the pace
+        constexpr size_t kChunkBytes = 2u << 20;
+        auto io_bytes = [&](int i) { return (size_t)problems[i].M * ((size_t)problems[i].K + problems[i].N) * sizeof(__half); };
+        int i1 = i0 + 1, limit = reuse[(size_t)i0] / 3;
+        size_t bytes = io_bytes(i0);
+        for (; i1 < count; ++i1) {
+            if (reuse[(size_t)i1] / 3 < limit) limit = reuse[(size_t)i1] / 3;
+            if (i1 - i0 >= limit) break;      // (also ends the chunk before a problem that shares a buffer with it)
+            bytes += io_bytes(i1);
+            if (bytes > kChunkBytes) break;
+        }
+        const int c = n_chunks++;
+        // a staging buffer used by an earlier chunk is overwritten only after that chunk is done with it: after its
+        // matmuls (ev_g) where it was their x, after its copies down (ev_y) where it was their y; the streams are in
+        // order, so the latest such chunk suffices
+        int wait_g = -1, wait_y_in = -1, wait_y = -1;
+        for (int i = i0; i < i1; ++i) {
+            auto it = read_as_x.find(problems[i].x_stage);
+            if (it != read_as_x.end() && it->second > wait_g) wait_g = it->second;
+            it = copied_as_y.find(problems[i].x_stage);
+            if (it != copied_as_y.end() && it->second > wait_y_in) wait_y_in = it->second;
+            it = copied_as_y.find(problems[i].y_stage);
+            if (it != copied_as_y.end() && it->second > wait_y) wait_y = it->second;
+        }
+        for (int i = i0; i < i1; ++i) {
+            read_as_x[problems[i].x_stage] = c;
+            copied_as_y[problems[i].y_stage] = c;
+        }
+        if (wait_y_in >= 0) st = check(cudaStreamWaitEvent(pipe->in, ev_y[wait_y_in], 0));
+        if (!st && wait_g >= 0 && wait_g > wait_y_in) st = check(cudaStreamWaitEvent(pipe->in, ev_g[wait_g], 0));
+        for (int i = i0; i < i1 && !st; ++i) {
+            const gptq_host_problem_t &q = problems[i];
+            st = check(cudaMemcpyAsync(q.x_stage, q.x_host, (size_t)q.M * q.K * sizeof(__half), cudaMemcpyHostToDevice, pipe->in));
+        }
+        if (!st) st = check(cudaEventRecord(ev_x[c], pipe->in));
+        if (!st) st = check(cudaStreamWaitEvent(s, ev_x[c], 0));
+        if (!st && wait_y >= 0) st = check(cudaStreamWaitEvent(s, ev_y[wait_y], 0));
+        for (int i = i0; i < i1 && !st; ++i) {
+            const gptq_host_problem_t &q = problems[i];
+            if (mode == 2)
+                st = gptq_gemm_w8(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size, stream);
+            else
+                st = gemm_dispatch(q.x_stage, q.qweight, q.qzeros, q.scales, q.g_idx, q.y_stage, q.M, q.N, q.K, q.group_size,
+                                   q.act_order, 0, nullptr, nullptr, nullptr, stream, mode);
+            if (st && bad_index) *bad_index = i;
+        }
+        if (st) break;
+        st = check(cudaEventRecord(ev_g[c], s));
+        if (!st) st = check(cudaStreamWaitEvent(pipe->out, ev_g[c], 0));
+        for (int i = i0; i < i1 && !st; ++i) {
+            const gptq_host_problem_t &q = problems[i];
+            st = check(cudaMemcpyAsync(q.y_host, q.y_stage, (size_t)q.M * q.N * sizeof(__half), cudaMemcpyDeviceToHost, pipe->out));
+        }
+        if (!st) st = check(cudaEventRecord(ev_y[c], pipe->out));
+        i0 = i1;
     }
     // join: `stream` finishes after the last copy of each direction, also after an error
     int st2 = check(cudaEventRecord(ev_start, pipe->in));

@@ -1312,3 +1312,73 @@ def test_seeded_shape_sweep(kind, K, N, M, gs, act, zm1, ws):
     # below K = 4096 the stated bar shrinks faster than the error of layers with few groups does (see the header):
     # the sweep holds the bar at its K = 4096 value there
     assert np.all(np.abs(y.astype(np.float64) - want) <= 1e-2 * max(1.0, math.sqrt(K / 4096)) + 1e-2 * np.abs(want))
+
+
+def test_host_batch_call_can_be_captured_in_a_cuda_graph(ws):
+    """gptq_gemm_host_batch is stream-ordered (its two copy streams fork from and join the caller's stream), so a step
+    can be captured once and replayed: every replay copies the host activations as they are then, multiplies and copies
+    the results back."""
+    specs = [(1024, 256, 2, False), (640, 256, 5, True), (512, 384, 40, False)]
+    items, keep = [], []
+    for (K, N, M, act) in specs:
+        L = wl.make_linear(K, N, seed=wl.seed_for("batch-graph", K, N, act), act_order=act)
+        D = H.upload_and_repack(L)
+        xh = torch.zeros((M, K), dtype=torch.float16).pin_memory()
+        yh = torch.zeros((M, N), dtype=torch.float16).pin_memory()
+        xs = torch.empty((M, K), dtype=torch.float16, device="cuda")
+        ys = torch.empty((M, N), dtype=torch.float16, device="cuda")
+        items.append((xh, D.qweight_t, D.qzeros_t, D.scales_t, D.perm, yh, xs, ys, M, N, K, 128, act))
+        keep.append((L, xh, yh, D))
+    ws.ensure(max(B.gptq_workspace_bytes(M, N, K, 128, act) for (K, N, M, act) in specs))
+    problems = B.make_host_problems(items)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        assert B.gptq_gemm_host_batch(problems)[0] == B.GPTQ_OK        # first use creates the copy streams and events
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            assert B.gptq_gemm_host_batch(problems)[0] == B.GPTQ_OK
+        for rnd in range(2):
+            xs_np = []
+            for (L, xh, yh, _D), (K, N, M, act) in zip(keep, specs):
+                x_np = wl.make_x(M, K, wl.seed_for("batch-graph-x", K, M, rnd))
+                xh.copy_(torch.from_numpy(x_np))
+                yh.zero_()
+                xs_np.append(x_np)
+            g.replay()
+            stream.synchronize()
+            assert B.gptq_check_status() == B.GPTQ_OK
+            for (L, xh, yh, _D), (K, N, M, act), x_np in zip(keep, specs, xs_np):
+                assert_close(yh.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, L.g_idx, 128), K)
+
+
+@pytest.mark.parametrize("pattern", ["own", "pairs", "one", "every5"])
+def test_host_batch_chunks_respect_shared_staging_buffers(pattern, ws):
+    """Forty small problems with their own activations each, whose device staging buffers are all distinct, shared by
+    neighbours, all the same, or repeating every five problems: the pipeline forms chunks of different lengths, and every
+    result must be the product of that problem's own x (a copy that overtook an earlier user of its buffer would show)."""
+    K, N, M, count = 256, 256, 3, 40
+    layers = [wl.make_linear(K, N, seed=wl.seed_for("chunks", i)) for i in range(4)]
+    Ds = [H.upload_and_repack(L) for L in layers]
+    n_bufs = {"own": count, "pairs": count // 2, "one": 1, "every5": 5}[pattern]
+    xs = [torch.empty((M, K), dtype=torch.float16, device="cuda") for _ in range(n_bufs)]
+    ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(n_bufs)]
+    slot = (lambda i: i) if pattern == "own" else (lambda i: i // 2) if pattern == "pairs" else (lambda i: i % n_bufs)
+    items, keep = [], []
+    for i in range(count):
+        x_np = wl.make_x(M, K, wl.seed_for("chunks-x", i))
+        xh = torch.from_numpy(x_np).pin_memory()
+        yh = torch.zeros((M, N), dtype=torch.float16).pin_memory()
+        D = Ds[i % 4]
+        items.append((xh, D.qweight_t, D.qzeros_t, D.scales_t, None, yh, xs[slot(i)], ys[slot(i)], M, N, K, 128, False))
+        keep.append((layers[i % 4], x_np, yh))
+    problems = B.make_host_problems(items)
+    for _ in range(3):                                   # repeated calls reuse the same events and streams
+        for (_L, _x, yh) in keep:
+            yh.zero_()
+        st, bad = B.gptq_gemm_host_batch(problems)
+        assert (st, bad) == (B.GPTQ_OK, -1)
+        torch.cuda.synchronize()
+        assert B.gptq_check_status() == B.GPTQ_OK
+        for (L, x_np, yh) in keep:
+            assert_close(yh.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, None, 128), K)
