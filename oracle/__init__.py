@@ -43,7 +43,8 @@ def _load():
                      "oracle_gemm_f64", "oracle_gemm_f64_at", "oracle_dequant_f32_v1", "oracle_gemm_f64_v1", "oracle_silu_mul_f64",
                      "oracle_add_bias_residual_f64", "oracle_dequant_f32_bf16", "oracle_gemm_f64_bf16",
                      "oracle_gemm_f64_bf16_at", "oracle_unpack_q8", "oracle_unpack_z8", "oracle_dequant_f32_w8",
-                     "oracle_gemm_f64_w8", "oracle_gemm_f64_w8_at"):
+                     "oracle_gemm_f64_w8", "oracle_gemm_f64_w8_at", "oracle_unpack_qn", "oracle_unpack_zn",
+                     "oracle_dequant_f32_wn", "oracle_gemm_f64_wn"):
             getattr(lib, name).restype = None
         _lib = lib
     return _lib
@@ -316,4 +317,60 @@ def gemm_f64_w8_at(x, qweight, qzeros, scales, g_idx, group_size: int, rows, col
     _load().oracle_gemm_f64_w8_at(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M), ctypes.c_int(N),
                                   ctypes.c_int(K), ctypes.c_int(group_size), ctypes.c_int(1 if zeros_minus_one else 0),
                                   _p(rows), _p(cols), ctypes.c_int(rows.shape[0]), _p(out))
+    return out
+
+
+# ---- 2- and 3-bit weights: qweight int32[K * bits / 32, N], qzeros int32[G, N * bits / 32] ---------------------------
+
+def unpack_qn(qweight: np.ndarray, bits: int) -> np.ndarray:
+    """int32[K * bits / 32, N] -> uint8[K, N]."""
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 32 // bits
+    out = np.empty((K, N), dtype=np.uint8)
+    _load().oracle_unpack_qn(_p(qweight), ctypes.c_int(K), ctypes.c_int(N), ctypes.c_int(bits), _p(out))
+    return out
+
+
+def unpack_zn(qzeros: np.ndarray, bits: int) -> np.ndarray:
+    """int32[G, N * bits / 32] -> uint8[G, N]."""
+    qzeros = _i32(qzeros)
+    G, C = qzeros.shape
+    N = C * 32 // bits
+    out = np.empty((G, N), dtype=np.uint8)
+    _load().oracle_unpack_zn(_p(qzeros), ctypes.c_int(G), ctypes.c_int(N), ctypes.c_int(bits), _p(out))
+    return out
+
+
+def _wn_args(qweight, qzeros, scales, g_idx, group_size, bits):
+    assert bits in (2, 3)
+    qweight = _i32(qweight)
+    R, N = qweight.shape
+    K = R * 32 // bits
+    G = K // group_size
+    qzeros = _i32(qzeros, (G, N * bits // 32))
+    scales = _f16(scales, (G, N))
+    g = None if g_idx is None else _i32(g_idx, (K,))
+    return qweight, qzeros, scales, g, K, N
+
+
+def dequant_f32_wn(qweight, qzeros, scales, g_idx, group_size: int, bits: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp32[K, N] dequantised 2- or 3-bit weights."""
+    qweight, qzeros, scales, g, K, N = _wn_args(qweight, qzeros, scales, g_idx, group_size, bits)
+    out = np.empty((K, N), dtype=np.float32)
+    _load().oracle_dequant_f32_wn(_p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(K), ctypes.c_int(N),
+                                  ctypes.c_int(group_size), ctypes.c_int(bits), ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
+    return out
+
+
+def gemm_f64_wn(x, qweight, qzeros, scales, g_idx, group_size: int, bits: int, zeros_minus_one: bool = False) -> np.ndarray:
+    """fp64[M, N] = x[M, K] . dequant(W)[K, N] for 2- or 3-bit weights, k ascending."""
+    qweight, qzeros, scales, g, K, N = _wn_args(qweight, qzeros, scales, g_idx, group_size, bits)
+    x = _f16(x)
+    M = x.shape[0]
+    assert x.shape == (M, K)
+    out = np.empty((M, N), dtype=np.float64)
+    _load().oracle_gemm_f64_wn(_p(x), _p(qweight), _p(qzeros), _p(scales), _p(g), ctypes.c_int(M), ctypes.c_int(N),
+                               ctypes.c_int(K), ctypes.c_int(group_size), ctypes.c_int(bits),
+                               ctypes.c_int(1 if zeros_minus_one else 0), _p(out))
     return out

@@ -378,3 +378,69 @@ void oracle_gemm_f64_w8_at(const uint16_t *x, const int32_t *qweight, const int3
         y_out[i] = acc;
     }
 }
+
+/* ---- format variant: 2- and 3-bit weights ------------------------------------------------------
+ * The paper treats 4-bit GPTQ only (Section 1); the checkpoint family also has 2- and 3-bit layers.
+ * Reading (pinned by hand-packed words in the tests): the values of a column (weights, along K) or
+ * of a group's row (zero points, along N) form one bit stream, value i in bits [bits*i, bits*i+bits)
+ * of the little-endian concatenation of that column's / row's 32-bit words - for 2 bits, 16 values
+ * per word; for 3 bits, 32 values per three words, values 10 and 21 straddling a word boundary.
+ *   qweight int32[K*bits/32][N], qzeros int32[G][N*bits/32], scales fp16[G][N]
+ *   w32[k][n] = float(q - z) * float(s), z = stored + zeros_plus;  y as in the 4-bit case. */
+static inline unsigned stream_field(const int32_t *words, size_t stride, int index, int bits)
+{
+    int bit = bits * index, w = bit >> 5, sh = bit & 31;
+    uint64_t two = (uint32_t)words[(size_t)w * stride];
+    if (sh + bits > 32) two |= (uint64_t)(uint32_t)words[(size_t)(w + 1) * stride] << 32;
+    return (unsigned)((two >> sh) & ((1u << bits) - 1u));
+}
+
+void oracle_unpack_qn(const int32_t *qweight, int K, int N, int bits, uint8_t *q_out)
+{
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            q_out[(size_t)k * N + n] = (uint8_t)stream_field(qweight + n, (size_t)N, k, bits);
+}
+
+void oracle_unpack_zn(const int32_t *qzeros, int G, int N, int bits, uint8_t *z_out)
+{
+    for (int g = 0; g < G; g++)
+        for (int n = 0; n < N; n++)
+            z_out[(size_t)g * N + n] = (uint8_t)stream_field(qzeros + (size_t)g * (N * bits / 32), 1, n, bits);
+}
+
+static inline float dequant_one_wn(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                                   const int32_t *g_idx, int N, int group_size, int bits, int zeros_plus, int k, int n)
+{
+    int g = group_of(g_idx, k, group_size);
+    int q = (int)stream_field(qweight + n, (size_t)N, k, bits);
+    int z = (int)stream_field(qzeros + (size_t)g * (N * bits / 32), 1, n, bits) + zeros_plus;
+    float s = oracle_half_to_float(scales[(size_t)g * N + n]);
+    return (float)(q - z) * s;
+}
+
+void oracle_dequant_f32_wn(const int32_t *qweight, const int32_t *qzeros, const uint16_t *scales,
+                           const int32_t *g_idx, int K, int N, int group_size, int bits, int zeros_plus, float *w_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; k++)
+        for (int n = 0; n < N; n++)
+            w_out[(size_t)k * N + n] = dequant_one_wn(qweight, qzeros, scales, g_idx, N, group_size, bits, zeros_plus, k, n);
+}
+
+void oracle_gemm_f64_wn(const uint16_t *x, const int32_t *qweight, const int32_t *qzeros,
+                        const uint16_t *scales, const int32_t *g_idx,
+                        int M, int N, int K, int group_size, int bits, int zeros_plus, double *y_out)
+{
+    #pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; n++) {
+        for (int m = 0; m < M; m++) {
+            double acc = 0.0;
+            for (int k = 0; k < K; k++) {
+                float w = dequant_one_wn(qweight, qzeros, scales, g_idx, N, group_size, bits, zeros_plus, k, n);
+                acc += (double)oracle_half_to_float(x[(size_t)m * K + k]) * (double)w;
+            }
+            y_out[(size_t)m * N + n] = acc;
+        }
+    }
+}

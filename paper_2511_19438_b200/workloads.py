@@ -180,6 +180,31 @@ def make_linear_w8(K: int, N: int, seed: int, group_size: int = GROUP_SIZE, act_
     return QuantLinear(K, N, group_size, qweight, pack8_along_n(z), scales, g_idx, seed, zeros_minus_one)
 
 
+def pack_bits_stream(v: np.ndarray, bits: int) -> np.ndarray:
+    """uint8[R, L] values below 2^bits -> int32[R, L * bits / 32]: each row is one bit stream, value i in bits
+    [bits * i, bits * i + bits) of the little-endian concatenation of the row's 32-bit words (2- and 3-bit layers)."""
+    R, L = v.shape
+    assert (L * bits) % 32 == 0 and int(v.max(initial=0)) < (1 << bits)
+    bit = ((v[:, :, None].astype(np.uint8) >> np.arange(bits, dtype=np.uint8)) & 1).reshape(R, L * bits)      # LSB first
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    return (bit.reshape(R, L * bits // 32, 32).astype(np.uint64) * weights).sum(axis=2).astype(np.uint32).view(np.int32)
+
+
+def make_linear_wn(K: int, N: int, seed: int, bits: int, group_size: int = GROUP_SIZE, act_order: bool = False,
+                   zeros_minus_one: bool = False) -> QuantLinear:
+    """Random 2- or 3-bit GPTQ layer: qweight int32[K * bits / 32, N] (a bit stream per column), qzeros
+    int32[G, N * bits / 32] (a bit stream per group), uniform values; scales and g_idx as for the 4-bit layers."""
+    assert bits in (2, 3) and K % 32 == 0 and N % 32 == 0 and K % group_size == 0
+    G = K // group_size
+    r = _rng(seed)
+    q = r.integers(0, 1 << bits, size=(K, N), dtype=np.uint8)
+    z = r.integers(0, 1 << bits, size=(G, N), dtype=np.uint8)
+    qweight = np.ascontiguousarray(pack_bits_stream(np.ascontiguousarray(q.T), bits).T)
+    scales = make_scales(G, N, seed ^ 0x5CA1E5)
+    g_idx = make_g_idx(K, group_size, seed ^ 0x61D7) if act_order else None
+    return QuantLinear(K, N, group_size, qweight, pack_bits_stream(z, bits), scales, g_idx, seed, zeros_minus_one)
+
+
 def bf16_bits(a: np.ndarray) -> np.ndarray:
     """Finite float values -> the bit patterns (uint16) of the nearest bfloat16, ties to even.  Inputs for the
     bfloat16 variant travel in this form because numpy has no bfloat16 type."""

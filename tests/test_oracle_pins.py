@@ -620,3 +620,85 @@ def test_w8_against_library_fp64_matmul(K, N, act, gs):
     rows = np.array([0, 2, 1, 1], dtype=np.int32)
     cols = np.array([0, N - 1, 17, 18], dtype=np.int32)
     assert np.array_equal(oracle.gemm_f64_w8_at(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, rows, cols), got[rows, cols])
+
+
+# --------------------------------------------------------------------------- 2- and 3-bit weights
+def local_pack_stream(vals, bits):
+    """Test-local packer: one big Python integer holds the bit stream (value i at bit bits * i), cut into 32-bit words."""
+    big = 0
+    for i, v in enumerate(vals):
+        assert 0 <= int(v) < (1 << bits)
+        big += int(v) << (bits * i)
+    n_words = len(vals) * bits // 32
+    return [(big >> (32 * w)) & 0xFFFFFFFF for w in range(n_words)]
+
+
+def test_wn_unpack_hand_typed_words():
+    """3 bits: the values 0..7 take 24 bits, 0xFAC688 (0 in bits 0-2, 1 in 3-5, ... 7 in 21-23); four times over they
+    fill three words, cut from the 96-bit stream 0xFAC688FAC688FAC688FAC688 at 32-bit boundaries: 0x88FAC688, 0xC688FAC6,
+    0xFAC688FA.  Value 10 (= 2) then has its low two bits at the top of word 0 and its high bit at the bottom of word 1,
+    value 21 (= 5) its low bit at the top of word 1.  2 bits: 0xE4 repeated is the sequence 0, 1, 2, 3."""
+    vals = [i % 8 for i in range(32)]
+    typed = np.array([[0x88FAC688], [0xC688FAC6], [0xFAC688FA]], dtype=np.uint32)
+    assert local_pack_stream(vals, 3) == [int(w) for w in typed[:, 0]]
+    # decode the typed words by hand rule: bit b of the stream is bit b % 32 of word b // 32
+    stream = "".join(format(int(w), "032b")[::-1] for w in typed[:, 0])
+    by_hand = [int(stream[3 * i:3 * i + 3][::-1], 2) for i in range(32)]
+    assert by_hand == vals
+    assert np.array_equal(oracle.unpack_qn(typed.view(np.int32), 3)[:, 0], np.array(vals, dtype=np.uint8))
+    assert np.array_equal(oracle.unpack_zn(typed.T.copy().view(np.int32), 3)[0], np.array(vals, dtype=np.uint8))
+    two = np.array([[0xE4E4E4E4]], dtype=np.uint32).view(np.int32)
+    assert np.array_equal(oracle.unpack_qn(two, 2)[:, 0], np.array([0, 1, 2, 3] * 4, dtype=np.uint8))
+    assert np.array_equal(oracle.unpack_zn(two, 2)[0], np.array([0, 1, 2, 3] * 4, dtype=np.uint8))
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_wn_generator_packer_agrees_with_the_big_integer_packer(bits):
+    r = np.random.default_rng(41 + bits)
+    v = r.integers(0, 1 << bits, (5, 64)).astype(np.uint8)
+    got = wl.pack_bits_stream(v, bits).view(np.uint32)
+    for row in range(5):
+        assert [int(w) for w in got[row]] == local_pack_stream(v[row], bits)
+    assert np.array_equal(oracle.unpack_zn(got.view(np.int32), bits), v)
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("act_order,zm1", [(False, False), (True, True)])
+def test_wn_dequant_and_gemm_match_rational_brute_force(bits, act_order, zm1):
+    K, N, M, gs = 32, 32, 2, 16
+    r = np.random.default_rng(50 + bits)
+    q = r.integers(0, 1 << bits, (K, N)).astype(np.uint8)
+    z = r.integers(0, 1 << bits, (K // gs, N)).astype(np.uint8)
+    s = (2.0 ** r.integers(-4, 3, (K // gs, N))).astype(np.float16) * np.where(r.random((K // gs, N)) < 0.3, 1.5, 1.0).astype(np.float16)
+    groups = [int(g) for g in r.permutation(K) // gs] if act_order else [k // gs for k in range(K)]
+    g_idx = np.array(groups, dtype=np.int32) if act_order else None
+    x = r.integers(-8, 9, (M, K)).astype(np.float16) / np.float16(4)
+    qw = np.array([local_pack_stream(q[:, n], bits) for n in range(N)], dtype=np.uint32).T.copy().view(np.int32)
+    qz = np.array([local_pack_stream(z[g], bits) for g in range(K // gs)], dtype=np.uint32).view(np.int32)
+    w = oracle.dequant_f32_wn(qw, qz, s, g_idx, gs, bits, zeros_minus_one=zm1)
+    for k in range(K):
+        for n in range(N):
+            assert float(w[k, n]) == (int(q[k, n]) - int(z[groups[k], n]) - int(zm1)) * float(s[groups[k], n]), (k, n)
+    want = brute_force_y(x, q.astype(np.int64), z.astype(np.int64) + int(zm1), s, groups)
+    got = oracle.gemm_f64_wn(x, qw, qz, s, g_idx, gs, bits, zeros_minus_one=zm1)
+    for m in range(M):
+        for n in range(N):
+            assert Fraction(float(got[m, n])) == want[m][n], (m, n)
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_wn_layer_equals_the_4bit_layer_with_the_same_values(bits):
+    """The same small values packed as a 4-bit layer must give what the (separately pinned) 4-bit functions give; and
+    numpy's fp64 matmul agrees at a larger size."""
+    K, N, M, gs = 1024, 256, 3, 128
+    L = wl.make_linear_wn(K, N, seed=wl.seed_for("pin-wn", bits), bits=bits, group_size=gs, act_order=True)
+    x = wl.make_x(M, K, wl.seed_for("pin-wn-x", bits))
+    q, z = oracle.unpack_qn(L.qweight, bits), oracle.unpack_zn(L.qzeros, bits)
+    L4 = wl.make_linear_from_values(q, z, L.scales, gs, L.g_idx)
+    for zm1 in (False, True):
+        a = oracle.gemm_f64_wn(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, bits, zeros_minus_one=zm1)
+        b = oracle.gemm_f64(x, L4.qweight, L4.qzeros, L4.scales, L.g_idx, gs, zeros_minus_one=zm1)
+        assert np.array_equal(a, b)
+    w = (q.astype(np.int64) - z.astype(np.int64)[L.g_idx]).astype(np.float64) * L.scales[L.g_idx].astype(np.float64)
+    assert np.allclose(oracle.gemm_f64_wn(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, bits), x.astype(np.float64) @ w,
+                       rtol=1e-11, atol=1e-10)
