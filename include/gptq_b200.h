@@ -221,6 +221,25 @@ int gptq_gemm_silu_mul_scatter(const void *x, const void *qweight, const void *q
  * skipped). */
 int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream);
 
+/* ---- 2- and 3-bit weights (no counterpart in the paper, which treats 4-bit GPTQ only - Section 1) -----------------
+ * Checkpoint layout: the values of a column (weights, along K) or of a group's row (zero points, along N) form one bit
+ * stream, value i in bits [bits * i, bits * i + bits) of the little-endian concatenation of that column's / row's
+ * 32-bit words: qweight int32[K * bits / 32, N], qzeros int32[G, N * bits / 32] (2 bits: 16 values per word; 3 bits: 32
+ * values per three words).  K and N must be multiples of 32 (GPTQ_ERR_SHAPE).  gptq_repack_bits widens every field to a
+ * nibble and writes an ordinary tiled 4-bit layer - same output sizes as gptq_repack (gptq_repack_bytes), same perm_out,
+ * to be used with gptq_gemm and the other 4-bit entry points with act_order as given here.  The tiled layer streams the
+ * bytes of a 4-bit layer: these widths are supported, not accelerated.  bits other than 2 or 3: GPTQ_ERR_UNSUPPORTED.
+ * format: 0 or GPTQ_FORMAT_ZEROS_MINUS_ONE (the one is added during the repack; the tiled layer stores zero points as
+ * they are).  scratch: device, 256-byte aligned, gptq_repack_bits_scratch_bytes (about K * N / 2); GPTQ_ERR_WORKSPACE if
+ * smaller; free once the stream has passed the call.  Other arguments and errors as for gptq_repack. */
+size_t gptq_repack_bits_scratch_bytes(int bits, int N, int K, int group_size);
+int gptq_repack_bits(int bits, const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                     void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, void *scratch,
+                     size_t scratch_bytes, int N, int K, int group_size, int act_order, int format, void *stream);
+/* fp32 w[K, N] of a canonical 2- or 3-bit layer, bit-exact (for the repacked layer use gptq_dequant_f32, repacked = 1). */
+int gptq_dequant_f32_bits(int bits, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                          float *w_out, int N, int K, int group_size, int act_order, int format, void *stream);
+
 /* ---- 8-bit weights (no counterpart in the paper, which treats 4-bit GPTQ only - Section 1) ------------------------
  * The checkpoint conventions at twice the field width: qweight int32[K/4, N], byte i of a word = row 4 r + i (least
  * significant first); qzeros int32[G, N/4], byte j of a word = column 4 c + j; scales fp16[G, N]; g_idx int32[K].

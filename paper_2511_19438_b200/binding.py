@@ -73,6 +73,9 @@ _SIGNATURES = {
     "gptq_set_workspace": (_i, [_vp, _sz]),
     "gptq_gemm": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_gemm_bf16": (_i, [_vp] * 6 + [_i, _i, _i, _i, _i, _vp]),
+    "gptq_repack_bits_scratch_bytes": (ctypes.c_size_t, [_i, _i, _i, _i]),
+    "gptq_repack_bits": (_i, [_i] + [_vp] * 9 + [ctypes.c_size_t, _i, _i, _i, _i, _i, _vp]),
+    "gptq_dequant_f32_bits": (_i, [_i] + [_vp] * 5 + [_i, _i, _i, _i, _i, _vp]),
     "gptq_repack_w8_bytes": (ctypes.c_size_t, [_i, _i, _i, _i]),
     "gptq_repack_w8_scratch_bytes": (ctypes.c_size_t, [_i, _i, _i]),
     "gptq_repack_w8": (_i, [_vp] * 9 + [ctypes.c_size_t, _i, _i, _i, _i, _i, _vp]),
@@ -196,6 +199,22 @@ def gptq_gemm(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_ord
 def gptq_gemm_bf16(x, qweight, qzeros, scales, g_idx, y, M, N, K, group_size, act_order, stream=None) -> int:
     return _lib.gptq_gemm_bf16(_ptr(x), _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(y), M, N, K,
                                group_size, act_order, _stream(stream))
+
+
+def gptq_repack_bits_scratch_bytes(bits, N, K, group_size) -> int:
+    return int(_lib.gptq_repack_bits_scratch_bytes(bits, N, K, group_size))
+
+
+def gptq_repack_bits(bits, qweight, qzeros, scales, g_idx, qweight_out, qzeros_out, scales_out, perm_out, scratch,
+                     scratch_bytes, N, K, group_size, act_order, fmt, stream=None) -> int:
+    return _lib.gptq_repack_bits(bits, _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(qweight_out),
+                                 _ptr(qzeros_out), _ptr(scales_out), _ptr(perm_out), _ptr(scratch), int(scratch_bytes), N, K,
+                                 group_size, int(act_order), int(fmt), _stream(stream))
+
+
+def gptq_dequant_f32_bits(bits, qweight, qzeros, scales, g_idx, w_out, N, K, group_size, act_order, fmt, stream=None) -> int:
+    return _lib.gptq_dequant_f32_bits(bits, _ptr(qweight), _ptr(qzeros), _ptr(scales), _ptr(g_idx), _ptr(w_out), N, K,
+                                      group_size, int(act_order), int(fmt), _stream(stream))
 
 
 def gptq_repack_w8_bytes(which, N, K, group_size) -> int:

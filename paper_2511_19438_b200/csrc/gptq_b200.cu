@@ -7,6 +7,7 @@
 #include "gptq_umma.cuh"
 #include "gptq_umma2.cuh"
 #include "gptq_w8.cuh"
+#include "gptq_wn.cuh"
 
 #include <atomic>
 #include <cstdio>
@@ -564,6 +565,58 @@ int gptq_gemm_w8(const void *x, const void *qweight, const void *qzeros, const v
     // the stacked layer, its activations already in its row order
     return gemm_dispatch(ws.ptr, qweight, qzeros, scales, nullptr, y, M, N, 2 * K, group_size, GPTQ_ACT_ORDER_PRESORTED, 0,
                          nullptr, nullptr, nullptr, stream);
+}
+
+// ---- 2- and 3-bit weights: widened to nibbles by the repack (gptq_wn.cuh) ------------------------------------------
+
+static int check_bits(int bits, int N, int K, int format)
+{
+    if (bits != 2 && bits != 3) return GPTQ_ERR_UNSUPPORTED;
+    if (format & ~GPTQ_FORMAT_ZEROS_MINUS_ONE) return GPTQ_ERR_LAYOUT;
+    if (K % 32 || N % 32) return GPTQ_ERR_SHAPE;     // whole words per column and per zero-point row
+    return GPTQ_OK;
+}
+
+size_t gptq_repack_bits_scratch_bytes(int bits, int N, int K, int group_size)
+{
+    int tiled = group_size;
+    if (check_shape(1, N, K, group_size) != GPTQ_OK || check_bits(bits, N, K, 0) != GPTQ_OK ||
+        check_fast_path(N, K, tiled) != GPTQ_OK)
+        return 0;
+    return wn_scratch_bytes(N, K, group_size);
+}
+
+int gptq_repack_bits(int bits, const int32_t *qweight, const int32_t *qzeros, const void *scales, const int32_t *g_idx,
+                     void *qweight_out, void *qzeros_out, void *scales_out, int32_t *perm_out, void *scratch,
+                     size_t scratch_bytes, int N, int K, int group_size, int act_order, int format, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !qweight_out || !qzeros_out || !scales_out || !scratch) return GPTQ_ERR_NULL;
+    if (act_order && (!g_idx || !perm_out)) return GPTQ_ERR_NULL;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    st = check_bits(bits, N, K, format);
+    if (st) return st;
+    int tiled = group_size;
+    st = check_fast_path(N, K, tiled);
+    if (st) return st;
+    if (!aligned16(qweight_out) || !aligned16(qzeros_out) || !aligned16(scales_out) || (reinterpret_cast<uintptr_t>(scratch) & 255u))
+        return GPTQ_ERR_ALIGN;
+    if (scratch_bytes < wn_scratch_bytes(N, K, group_size)) return GPTQ_ERR_WORKSPACE;
+    return launch_wn_repack(qweight, qzeros, scales, act_order ? g_idx : nullptr, qweight_out, qzeros_out, scales_out, perm_out,
+                            scratch, N, K, group_size, bits, act_order, (format & GPTQ_FORMAT_ZEROS_MINUS_ONE) ? 1 : 0,
+                            (cudaStream_t)stream);
+}
+
+int gptq_dequant_f32_bits(int bits, const void *qweight, const void *qzeros, const void *scales, const int32_t *g_idx,
+                          float *w_out, int N, int K, int group_size, int act_order, int format, void *stream)
+{
+    if (!qweight || !qzeros || !scales || !w_out || (act_order && !g_idx)) return GPTQ_ERR_NULL;
+    int st = check_shape(1, N, K, group_size);
+    if (st) return st;
+    st = check_bits(bits, N, K, format);
+    if (st) return st;
+    return launch_wn_dequant_f32(qweight, qzeros, scales, act_order ? g_idx : nullptr, w_out, N, K, group_size, bits,
+                                 (format & GPTQ_FORMAT_ZEROS_MINUS_ONE) ? 1 : 0, (cudaStream_t)stream);
 }
 
 int gptq_invert_perm(const int32_t *perm, int32_t *inverse, int K, void *stream)

@@ -188,3 +188,23 @@ def gemm_w8(x: torch.Tensor, D: DeviceLinear, y: torch.Tensor | None = None, str
 
 def ensure_for_w8(ws: "WorkspaceHolder", M: int, D: DeviceLinear) -> None:
     ws.ensure(B.gptq_workspace_bytes(M, D.N, 2 * D.K, D.group_size, 1))
+
+
+# ---- 2- and 3-bit layers (widened to a 4-bit layer by the repack) -----------------------------------------------------
+
+def upload_and_repack_bits(L: QuantLinear, bits: int, keep_canonical: bool = False, device="cuda") -> DeviceLinear:
+    """Uploads a canonical 2- or 3-bit layer and repacks it with gptq_repack_bits; the result is an ordinary tiled 4-bit
+    layer for :func:`gemm`."""
+    qw, qz, sc = to_device(L.qweight, device), to_device(L.qzeros, device), to_device(L.scales, device)
+    gi = to_device(L.g_idx, device) if L.act_order else None
+    outs = [torch.empty(B.gptq_repack_bytes(w, L.N, L.K, L.group_size, L.act_order), dtype=torch.uint8, device=device)
+            for w in range(3)]
+    perm = torch.empty(L.K, dtype=torch.int32, device=device) if L.act_order else None
+    nscratch = B.gptq_repack_bits_scratch_bytes(bits, L.N, L.K, L.group_size)
+    scratch = torch.empty(nscratch, dtype=torch.uint8, device=device)
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if L.zeros_minus_one else 0
+    B.check(B.gptq_repack_bits(bits, qw, qz, sc, gi, outs[0], outs[1], outs[2], perm, scratch, nscratch, L.N, L.K,
+                               L.group_size, L.act_order, fmt), "gptq_repack_bits")
+    torch.cuda.current_stream().synchronize()
+    canonical = (qw, qz, sc, gi) if keep_canonical else None
+    return DeviceLinear(L.K, L.N, L.group_size, L.act_order, outs[0], outs[1], outs[2], perm, canonical)

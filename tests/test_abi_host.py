@@ -89,6 +89,13 @@ def test_other_entry_points_validate_without_gpu():
     assert B.gptq_gemm_w8(A16, A16, A16, A16, A16, A16, 1, 128, 192, 64, stream=0) == B.GPTQ_ERR_UNSUPPORTED
     assert B.gptq_dequant_f32_w8(A16, A16, A16, None, A16, 128, 128, 128, 0, 1, 0, stream=0) == B.GPTQ_ERR_NULL   # tiled: perm needed
     assert B.gptq_dequant_f32_w8(A16, A16, A16, None, A16, 128, 128, 128, 0, 0, 4, stream=0) == B.GPTQ_ERR_LAYOUT
+    # 2- and 3-bit repack: checks before any CUDA call
+    assert B.gptq_repack_bits_scratch_bytes(3, 256, 512, 128) >= 512 * 256 // 2 and B.gptq_repack_bits_scratch_bytes(4, 256, 512, 128) == 0
+    assert B.gptq_repack_bits(5, A16, A16, A16, None, A16, A16, A16, None, A16 - A16 % 256 + 256, 1 << 30, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_UNSUPPORTED
+    assert B.gptq_repack_bits(2, A16, A16, A16, None, A16, A16, A16, None, None, 1 << 30, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_NULL
+    assert B.gptq_repack_bits(2, A16, A16, A16, None, A16, A16, A16, None, A16 - A16 % 256 + 256, 8, 128, 128, 128, 0, 0, stream=0) == B.GPTQ_ERR_WORKSPACE
+    assert B.gptq_dequant_f32_bits(3, A16, A16, A16, None, A16, 128, 136, 8, 0, 0, stream=0) == B.GPTQ_ERR_SHAPE   # K % 32
+    assert B.gptq_dequant_f32_bits(3, A16, A16, A16, None, A16, 128, 128, 128, 1, 0, stream=0) == B.GPTQ_ERR_NULL
     # the bfloat16 matmul validates like gptq_gemm
     assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, None, 1, 128, 128, 128, 0, stream=0) == B.GPTQ_ERR_NULL
     assert B.gptq_gemm_bf16(A16, A16, A16, A16, None, A16, 1, 128, 128, 128, 1, stream=0) == B.GPTQ_ERR_NULL

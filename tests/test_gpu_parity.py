@@ -1382,3 +1382,49 @@ def test_host_batch_chunks_respect_shared_staging_buffers(pattern, ws):
         assert B.gptq_check_status() == B.GPTQ_OK
         for (L, x_np, yh) in keep:
             assert_close(yh.numpy(), oracle.gemm_f64(x_np, L.qweight, L.qzeros, L.scales, None, 128), K)
+
+
+# ------------------------------------------------------------------------------- 2- and 3-bit weights
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("gs,act,zm1", [(128, False, False), (128, True, True), (32, True, False), (64, False, True), (512, False, False)])
+def test_low_bit_layers_dequant_bit_exact_and_multiply(bits, gs, act, zm1, ws):
+    """2- and 3-bit layers: the canonical buffers and the widened, tiled 4-bit layer both dequantise to the oracle's bits,
+    and gptq_gemm on the tiled layer matches the oracle's matmul on both kernel families."""
+    K, N = 512, 256
+    L = wl.make_linear_wn(K, N, seed=wl.seed_for("wn", bits, gs, act, zm1), bits=bits, group_size=gs, act_order=act,
+                          zeros_minus_one=zm1)
+    want_w = oracle.dequant_f32_wn(L.qweight, L.qzeros, L.scales, L.g_idx, gs, bits, zeros_minus_one=zm1)
+    fmt = B.GPTQ_FORMAT_ZEROS_MINUS_ONE if zm1 else 0
+    D = H.upload_and_repack_bits(L, bits, keep_canonical=True)
+    qw, qz, sc, gi = D.canonical
+    w = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    B.check(B.gptq_dequant_f32_bits(bits, qw, qz, sc, gi, w, N, K, gs, act, fmt), "dequant canonical")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want_w.view(np.uint32))
+    w.zero_()
+    B.check(B.gptq_dequant_f32(D.qweight_t, D.qzeros_t, D.scales_t, D.perm, w, N, K, gs, act, 1), "dequant tiled")
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), want_w.view(np.uint32))
+    for M in (1, 13, 40, 200):
+        x = wl.make_x(M, K, wl.seed_for("wn-x", bits, M))
+        ws.ensure_for(M, D)
+        y = H.gemm(H.to_device(x), D).cpu().numpy()
+        assert B.gptq_check_status() == B.GPTQ_OK
+        assert_close(y, oracle.gemm_f64_wn(x, L.qweight, L.qzeros, L.scales, L.g_idx, gs, bits, zeros_minus_one=zm1), K, M)
+
+
+def test_low_bit_repack_argument_checks():
+    K, N = 512, 256
+    L = wl.make_linear_wn(K, N, seed=3, bits=3)
+    qw, qz, sc = H.to_device(L.qweight), H.to_device(L.qzeros), H.to_device(L.scales)
+    outs = [torch.empty(B.gptq_repack_bytes(w, N, K, 128, 0), dtype=torch.uint8, device="cuda") for w in range(3)]
+    need = B.gptq_repack_bits_scratch_bytes(3, N, K, 128)
+    assert need >= K * N // 2 and B.gptq_repack_bits_scratch_bytes(5, N, K, 128) == 0
+    scratch = torch.empty(need, dtype=torch.uint8, device="cuda")
+    call = lambda bits=3, scr=scratch, nb=need, fmt=0, k=K: B.gptq_repack_bits(bits, qw, qz, sc, None, outs[0], outs[1], outs[2],
+                                                                              None, scr, nb, N, k, 128, 0, fmt)
+    assert call(bits=4) == B.GPTQ_ERR_UNSUPPORTED and call(bits=1) == B.GPTQ_ERR_UNSUPPORTED
+    assert call(nb=need - 1) == B.GPTQ_ERR_WORKSPACE
+    assert call(scr=None) == B.GPTQ_ERR_NULL
+    assert call(fmt=B.GPTQ_FORMAT_GATE_UP) == B.GPTQ_ERR_LAYOUT
+    assert call(k=K + 128 + 8) == B.GPTQ_ERR_SHAPE
+    assert call() == B.GPTQ_OK
+    torch.cuda.synchronize()
