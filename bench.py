@@ -50,7 +50,7 @@ NCU_TRAFFIC = {
     "splitk_kernel<1,1>": {"digest": "cafbf47bd6e61035", "ratio": 0.998, "Ms": (1, 4, 8),
                          "source": "ncu capture profiles/splitk_kernel_decode7b.md (108 launches: M = 1, 4, 8 on the four "
                                    "7B shapes): dram bytes / algorithmic bytes x algorithmic bytes per timed launch"},
-    "umma_kernel<256,4,1,2,1>": {"digest": "c94bbce5ab25a77f", "ratio": 0.928, "Ms": (512, 1024, 2048, 4096),
+    "umma_kernel<256,4,1,2,1>": {"digest": "36c16532a4b1d9c3", "ratio": 0.934, "Ms": (512, 1024, 2048, 4096),
                                "source": "ncu capture profiles/umma_kernel_prefill7b.md (161 launches: M = 512..4096 on "
                                          "the four 7B shapes, main + tail launches; y partly still in L2): ratio x "
                                          "algorithmic bytes per timed launch"},
